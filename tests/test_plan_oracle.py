@@ -1,0 +1,92 @@
+"""Pins for the tile-derivation and traffic restatements under oracle/.
+
+The register-machine derivation is pinned by the numbers the paper prints
+(Table 2, the descriptor listing, the HBM-traffic paragraph); the tensor-memory
+derivation has no printed numbers and is pinned by capacity invariants.
+"""
+import math
+
+import pytest
+
+from oracle import plan_oracle as po
+from tests.conftest import read_golden
+
+CDNA = dict(lds_bytes=64 * 1024, regs_per_thread=256, wavefront=64, atom_m=16, atom_n=16, elem_bytes=4)
+
+B200 = dict(num_units=148, local_mem_bytes=232448, regs_per_unit=65536, max_regs_per_thread=255,
+            simd_width=32, acc_mem_lanes=128, acc_mem_columns=512, atom_m=128, atom_n=16, atom_k=16,
+            atom_n_max=256, elem_bytes=2)
+
+
+def test_table2_register_use_and_feasibility():
+    for d, t_kv, t_q, regs, feasible in ((int(x) for x in row) for row in read_golden("paper_table2_tiles.txt")):
+        assert po.register_file_use(t_q, t_kv, d, 64) == regs
+        assert (regs <= 256) == bool(feasible)
+
+
+def test_table2_tiles_are_what_the_derivation_returns():
+    feasible_rows = [[int(x) for x in r] for r in read_golden("paper_table2_tiles.txt") if r[4] == "1"]
+    for d, t_kv, t_q, regs, _ in feasible_rows:
+        got = po.derive_tiles_register_machine(num_units=120, B=1, H=1, L=16384, d=d, **CDNA)
+        assert (got["tile_kv"], got["tile_q"], got["regs"], got["feasible"]) == (t_kv, t_q, regs, True)
+        # one atom step larger must not fit (the infeasible rows of the table)
+        assert po.register_file_use(t_q + 16, t_kv, d, 64) > 256
+
+
+def test_descriptor_listing_same_tiles_different_occupancy():
+    for num_cus, t_q, t_kv, printed in read_golden("paper_derive_tiles_listing.txt"):
+        got = po.derive_tiles_register_machine(num_units=int(num_cus), B=1, H=1, L=16384, d=128, **CDNA)
+        assert (got["tile_q"], got["tile_kv"]) == (int(t_q), int(t_kv))
+        assert got["tiles"] == 512
+        # the printed per-CU figure is the blocks-per-CU ratio (its fractional part for 120 CUs)
+        ratio = got["ctas_per_unit"]
+        assert min(abs(ratio - float(printed)), abs(ratio - math.floor(ratio) - float(printed))) < 0.01
+
+
+def test_traffic_figures_printed_in_the_paper():
+    g = {row[0]: (int(row[1]), float(row[2])) for row in read_golden("paper_hbm_traffic.txt")}
+    mb, gb = 1e6, 1e9
+    L, val = g["fused_mb"]
+    assert round(po.traffic_fused(1, 1, L, 128, 4) / mb) == val
+    L, val = g["unfused_mb"]
+    assert round(po.traffic_unfused(1, 1, L, 128, 4, 4) / mb) == val
+    L, val = g["score_mb"]
+    assert round(L * L * 4 / mb) == val
+    L, val = g["ratio"]
+    assert round(po.traffic_unfused(1, 1, L, 128, 4, 4) / po.traffic_fused(1, 1, L, 128, 4)) == val
+    L, val = g["unfused_gb"]
+    assert round(po.traffic_unfused(1, 1, L, 128, 4, 4) / gb) == val
+    L, val = g["savings"]
+    assert po.savings_ratio(L, 128) == val
+
+
+@pytest.mark.parametrize("B,H,L,d", [(1, 1, 256, 64), (1, 8, 2048, 128), (1, 1, 16384, 128), (1, 4, 32768, 128),
+                                     (4, 32, 4096, 128), (4, 32, 8192, 64), (1, 1, 128, 128), (2, 2, 1024, 256)])
+def test_tmem_machine_capacity_invariants(B, H, L, d):
+    t = po.derive_tiles_tmem_machine(B200, B, H, L, d)
+    assert t["feasible"]
+    n_q = t["n_q"]
+    assert t["tile_q"] == 128 * n_q and t["tile_kv"] % 16 == 0 and 32 <= t["tile_kv"] <= 256
+    assert n_q * (t["tile_kv"] + d) <= 512 <= 512 and t["tmem_columns"] <= 512       # tensor memory
+    assert t["smem_bytes"] <= B200["local_mem_bytes"]                                  # shared memory
+    assert t["smem_bytes"] == n_q * 128 * d * 2 + t["kv_stages"] * t["tile_kv"] * d * 2 + 2048
+    assert 4 <= t["kv_stages"] <= 8
+    regs_total = 128 * n_q * t["regs_softmax"] + 128 * 80 + 128 * 48                   # register file
+    assert regs_total <= 65536 and t["regs_softmax"] <= 248
+    assert t["tile_kv"] + t["tile_kv"] // 4 + 32 <= t["regs_softmax"]
+    assert t["ctas"] == t["tiles"] * t["kv_splits"]
+    assert 0 < t["wave_efficiency"] <= 1.0
+    if t["kv_splits"] > 1:
+        assert t["under_occupied"] and t["ctas"] <= 148
+        assert math.ceil(L / t["tile_kv"]) // t["kv_splits"] >= 4
+
+
+def test_tmem_machine_expected_defaults_for_the_benchmark_shapes():
+    t = po.derive_tiles_tmem_machine(B200, 1, 1, 16384, 128)
+    assert (t["tile_q"], t["tile_kv"], t["kv_stages"], t["kv_splits"], t["ctas"]) == (256, 128, 5, 2, 128)
+    assert t["under_occupied"] and abs(t["wave_efficiency"] - 128 / 148) < 1e-12
+    t = po.derive_tiles_tmem_machine(B200, 4, 32, 8192, 64)
+    assert (t["tile_q"], t["tile_kv"], t["kv_stages"], t["kv_splits"]) == (256, 128, 8, 1)
+    assert not t["under_occupied"]
+    assert not po.derive_tiles_tmem_machine(B200, 1, 1, 1024, 72)["feasible"]          # d not a multiple of 16
+    assert not po.derive_tiles_tmem_machine(B200, 1, 1, 1024, 512)["feasible"]         # d beyond the atom's N
