@@ -1,0 +1,200 @@
+/*
+ * attn.h -- C ABI of the B200 fused-attention library (libattn_b200.so).
+ *
+ * One operation: the fused attention forward pass of the paper's Section
+ * "Fused Attention",  O = softmax(Q K^T / sqrt(d)) V,  evaluated with
+ * Algorithm 1 (K/V tiles streamed through an online softmax, the L x L score
+ * matrix never written to memory), with tile sizes derived in closed form from
+ * a hardware descriptor (Sections "Hardware Model" and "Tile Derivation")
+ * instead of being searched.
+ *
+ * Conventions
+ *   - Plain C types only; no exceptions cross the boundary; every function
+ *     returns an attn_status (0 = success, negative = error) unless noted.
+ *   - q, k, v, o are DEVICE pointers to contiguous [B][H][L][d] bf16 arrays
+ *     (d fastest), 16-byte aligned.  Non-causal, no mask, scale 1/sqrt(d),
+ *     fp32 accumulation, bf16 (round-to-nearest-even) output.
+ *   - The caller owns every buffer, including the workspace.  The library
+ *     allocates no device memory and keeps no reference to q/k/v/o after a
+ *     call returns.  attn_forward* are asynchronous on `cuda_stream`
+ *     (a cudaStream_t passed as void*; NULL = the default stream) and never
+ *     synchronise.
+ *   - Supported shapes: d in {64, 128}, L a multiple of 128, B, H >= 1.
+ *   - Results are bitwise reproducible run to run (fixed merge order, no
+ *     atomics on the output).
+ */
+#ifndef ATTN_B200_H_
+#define ATTN_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum attn_status {
+  ATTN_OK = 0,
+  ATTN_ERR_INVALID_ARG = -1,       /* null pointer, non-positive size, bad struct_bytes   */
+  ATTN_ERR_UNSUPPORTED_SHAPE = -2, /* d not in {64,128} or L not a multiple of 128        */
+  ATTN_ERR_MISALIGNED = -3,        /* a device pointer is not 16-byte aligned             */
+  ATTN_ERR_ALIASING = -4,          /* o overlaps q, k or v                                */
+  ATTN_ERR_INFEASIBLE_PLAN = -5,   /* no tile choice fits; see binding_constraint         */
+  ATTN_ERR_WRONG_ARCH = -6,        /* current device is not compute capability 10.x       */
+  ATTN_ERR_NEED_WORKSPACE = -7,    /* plan splits the keys but no workspace was supplied  */
+  ATTN_ERR_CUDA = -8,              /* a CUDA runtime/driver call failed                   */
+  ATTN_ERR_DEVICE_TIMEOUT = -9,    /* a bounded device-side wait expired                  */
+  ATTN_ERR_BAD_TILES = -10         /* tile override not among the compiled variants       */
+} attn_status;
+
+/* Which capacity fixed the tile (the "binding constraint" returned by the
+ * paper's derive_tiles / FeasibilityVisitor, Section "Tile Derivation"). */
+typedef enum attn_binding {
+  ATTN_BIND_NONE = 0,
+  ATTN_BIND_SMEM = 1,  /* shared memory / local data share                       */
+  ATTN_BIND_TMEM = 2,  /* tensor-memory columns                                  */
+  ATTN_BIND_REG = 3,   /* register file                                          */
+  ATTN_BIND_ATOM = 4,  /* largest N of one matrix instruction                    */
+  ATTN_BIND_SHAPE = 5  /* problem shape not aligned to the atom                  */
+} attn_binding;
+
+/*
+ * Hardware descriptor: only the quantities the derivation uses (the paper's
+ * HardwareDescriptor / MFMAAtom listing, Section "Hardware Model").
+ * acc_mem_columns == 0 describes a machine whose accumulators live in vector
+ * registers (the paper's CDNA targets); > 0 describes tensor memory (B200).
+ * Caller-owned plain data; set struct_bytes = sizeof(attn_hw_desc).
+ */
+typedef struct attn_hw_desc {
+  int32_t struct_bytes;
+  int32_t num_units;           /* SMs / CUs                                           */
+  int32_t local_mem_bytes;     /* on-chip scratch one CTA may use (SMEM opt-in / LDS) */
+  int32_t regs_per_unit;       /* 32-bit registers per SM (0 if not modelled)         */
+  int32_t max_regs_per_thread; /* architectural per-thread limit                      */
+  int32_t simd_width;          /* warp / wavefront width                              */
+  int32_t acc_mem_lanes;       /* tensor-memory lanes (128), 0 if none                */
+  int32_t acc_mem_columns;     /* tensor-memory 32-bit columns (512), 0 if none       */
+  int32_t atom_m;              /* rows of one matrix instruction (128 | 16)           */
+  int32_t atom_n;              /* N granularity (16)                                  */
+  int32_t atom_k;              /* K of one instruction (16 | 4)                       */
+  int32_t atom_n_max;          /* largest N of one instruction (256 | 16)             */
+  int32_t elem_bytes;          /* operand element size (2 = bf16, 4 = fp32)           */
+  int32_t reserved;
+  double hbm_gbps;             /* sustained HBM bandwidth, GB/s                       */
+  double peak_tflops;          /* dense tensor peak for the operand type, TFLOP/s     */
+  double sm_clock_mhz;         /* maximum SM clock                                    */
+} attn_hw_desc;
+
+/* Result of the closed-form derivation.  Caller-owned plain data. */
+typedef struct attn_tiles {
+  int32_t tile_q;         /* Q rows per CTA = n_q * atom_m                              */
+  int32_t tile_kv;        /* K/V rows per streamed tile                                 */
+  int32_t n_q;            /* Q sub-tiles per CTA (ping-pong partners), 1 or 2           */
+  int32_t n_s;            /* score buffers per sub-tile (1)                             */
+  int32_t kv_stages;      /* depth of the shared-memory K/V ring (one K or V tile each) */
+  int32_t kv_splits;      /* CTAs sharing one Q tile along the key axis (merge operator)*/
+  int32_t smem_bytes;     /* dynamic shared memory per CTA                              */
+  int32_t tmem_columns;   /* tensor-memory columns allocated per CTA                    */
+  int32_t regs_softmax;   /* register allowance of a softmax thread                     */
+  int32_t threads;        /* threads per CTA                                            */
+  int32_t tiles;          /* B * H * ceil(L / tile_q)                                   */
+  int32_t ctas;           /* tiles * kv_splits                                          */
+  float ctas_per_unit;    /* ctas / num_units                                           */
+  float wave_efficiency;  /* ctas_per_unit / ceil(ctas_per_unit)                        */
+  int32_t feasible;       /* 1 if a tile choice fits                                    */
+  int32_t binding_constraint; /* attn_binding                                           */
+  int32_t under_occupied; /* 1 if tiles < num_units (occupancy check of the derivation) */
+  int32_t reserved;
+} attn_tiles;
+
+/* Built-in descriptor of one B200 (148 SMs, 227 KB SMEM opt-in, 64 K registers,
+ * 128 x 512 tensor memory, tcgen05 kind::f16 atom 128 x N x 16).  Host only. */
+int attn_hw_desc_b200(attn_hw_desc *out);
+
+/* Descriptor of CUDA device `device`, from cudaDeviceGetAttribute plus the
+ * per-architecture constants above.  ATTN_ERR_WRONG_ARCH unless cc 10.x. */
+int attn_hw_desc_query(int device, attn_hw_desc *out);
+
+/*
+ * Closed-form tile derivation (the paper's derive_tiles(desc, L, d); Section
+ * "Tile Derivation": capacity constraints in a fixed order, then the occupancy
+ * check, then atom alignment; Table 2 for the attention case).  Host only, no
+ * CUDA calls, no search.  Fills *out and returns ATTN_OK even when the result
+ * is infeasible (out->feasible == 0 and out->binding_constraint says why);
+ * returns ATTN_ERR_INVALID_ARG for null pointers or a bad struct_bytes.
+ */
+int attn_plan(const attn_hw_desc *desc, int B, int H, int L, int d, attn_tiles *out);
+
+/* Bytes of workspace attn_forward* needs for this plan: 0 unless kv_splits > 1
+ * (partial outputs and row statistics of the merge operator, Section "Online
+ * Softmax"). */
+size_t attn_workspace_bytes(const attn_tiles *tiles, int B, int H, int L, int d);
+
+/* Registers a caller-owned device buffer as the workspace of `device` (pass
+ * NULL, 0 to clear).  The buffer must stay valid until replaced; concurrent
+ * attn_forward calls on different streams of one device must not share it. */
+int attn_set_workspace(int device, void *dev_ptr, size_t bytes);
+
+/*
+ * Fused attention forward (Algorithm 1) with the closed-form default tiles for
+ * the current device.  Asynchronous on cuda_stream.  Errors: INVALID_ARG,
+ * UNSUPPORTED_SHAPE, MISALIGNED, ALIASING, WRONG_ARCH, INFEASIBLE_PLAN,
+ * NEED_WORKSPACE (plan has kv_splits > 1 and the registered workspace is
+ * smaller than attn_workspace_bytes), CUDA.
+ */
+int attn_forward(const void *q, const void *k, const void *v, void *o,
+                 int B, int H, int L, int d, void *cuda_stream);
+
+/* Same, with tile fields overridden (tile sweep only).  Honoured fields:
+ * n_q (1|2), tile_kv (64|128), kv_stages (2..plan maximum), kv_splits (>= 1).
+ * ATTN_ERR_BAD_TILES if the combination was not compiled or does not fit. */
+int attn_forward_tiles(const void *q, const void *k, const void *v, void *o,
+                       int B, int H, int L, int d, const attn_tiles *override_tiles,
+                       void *cuda_stream);
+
+/*
+ * Non-pipelined variant of the same algorithm: one 128-row Q tile per CTA, a
+ * single K/V stage, the two matrix products and the softmax strictly in
+ * sequence, plain global stores.  Slow; exists so that two independently
+ * scheduled kernels can be compared (the paper validates its two attention
+ * kernels against each other, Section "MFMA Kernel").  tile_kv in {64, 128}.
+ * If scores_out is non-NULL it receives the raw fp32 score tile Q_0 K_0^T of
+ * (batch 0, head 0): [128][tile_kv] floats (unscaled), for layout tests.
+ */
+int attn_forward_simple(const void *q, const void *k, const void *v, void *o,
+                        int B, int H, int L, int d, int tile_kv, float *scores_out,
+                        void *cuda_stream);
+
+/*
+ * Host-buffer form of attn_forward (the end-to-end path of Figure 2: Q, K, V
+ * come from host memory, R goes back to it).  q_host, k_host, v_host, o_host
+ * are HOST pointers (pinned memory for the copies to be asynchronous) in the
+ * same [B][H][L][d] bf16 layout; dev_scratch is a caller-owned DEVICE buffer of
+ * at least 4 * B*H*L*d*2 bytes, 256-byte aligned, that receives the device
+ * copies of q, k, v and o.  Queues three host-to-device copies, the forward
+ * pass and one device-to-host copy on cuda_stream; does not synchronise.
+ * Errors: as attn_forward, plus ATTN_ERR_INVALID_ARG if the scratch is small.
+ */
+int attn_forward_host(const void *q_host, const void *k_host, const void *v_host, void *o_host,
+                      int B, int H, int L, int d, void *dev_scratch, size_t dev_scratch_bytes,
+                      void *cuda_stream);
+
+/* Synchronises cuda_stream and reports whether any bounded device-side wait
+ * expired since the last query (ATTN_ERR_DEVICE_TIMEOUT) -- then detail[0..3]
+ * (optional, may be NULL) receive code, role/barrier/step word, CTA index and
+ * a spare word -- or ATTN_OK.  Clears the record. */
+int attn_last_device_status(void *cuda_stream, uint32_t *detail);
+
+/* Number of kernels the last attn_forward* call launched (1, or 2 with merge). */
+int attn_last_launch_count(void);
+
+/* Static description of a status code; never NULL. */
+const char *attn_status_string(int status);
+
+/* Last CUDA error text recorded by the library on this thread ("" if none). */
+const char *attn_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATTN_B200_H_ */

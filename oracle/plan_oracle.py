@@ -58,7 +58,7 @@ def derive_tiles_register_machine(lds_bytes, regs_per_thread, wavefront, num_uni
 _REGS_CORRECTION = 80      # per thread, correction/epilogue warpgroup
 _REGS_OTHER = 48           # per thread, TMA / MMA-issue warps
 _REGS_ROW_OVERHEAD = 32    # softmax thread: addresses, row statistics, loop state
-_SMEM_RESERVE = 2048       # barriers + 1 KB alignment slack
+_SMEM_RESERVE = 3072       # barriers, rescale factors, tensor-memory slot
 _MAX_STAGES = 8
 _MIN_STAGES = 4
 _MIN_TILE_KV = 32

@@ -1,0 +1,256 @@
+"""ctypes binding of libattn_b200.so: argument marshalling only.
+
+Every step of the attention path runs inside the library's CUDA kernels; this
+module turns torch tensors into device pointers, keeps the caller-owned
+workspace alive and raises on error codes.  There is no CPU fallback: if the
+shared library is missing or fails to load, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+from pathlib import Path
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libattn_b200.so"
+
+ATTN_OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_MISALIGNED, ERR_ALIASING = -1, -2, -3, -4
+ERR_INFEASIBLE_PLAN, ERR_WRONG_ARCH, ERR_NEED_WORKSPACE, ERR_CUDA = -5, -6, -7, -8
+ERR_DEVICE_TIMEOUT, ERR_BAD_TILES = -9, -10
+BIND_NAMES = ("none", "smem", "tmem", "reg", "atom", "shape")
+
+EXPORTED_SYMBOLS = (
+    "attn_hw_desc_b200", "attn_hw_desc_query", "attn_plan", "attn_workspace_bytes", "attn_set_workspace",
+    "attn_forward", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_last_device_status",
+    "attn_last_launch_count", "attn_status_string", "attn_last_cuda_error",
+)
+
+
+class AttnHwDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "struct_bytes", "num_units", "local_mem_bytes", "regs_per_unit", "max_regs_per_thread", "simd_width",
+        "acc_mem_lanes", "acc_mem_columns", "atom_m", "atom_n", "atom_k", "atom_n_max", "elem_bytes", "reserved",
+    )] + [("hbm_gbps", ctypes.c_double), ("peak_tflops", ctypes.c_double), ("sm_clock_mhz", ctypes.c_double)]
+
+
+class AttnTiles(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "tile_q", "tile_kv", "n_q", "n_s", "kv_stages", "kv_splits", "smem_bytes", "tmem_columns", "regs_softmax",
+        "threads", "tiles", "ctas",
+    )] + [("ctas_per_unit", ctypes.c_float), ("wave_efficiency", ctypes.c_float)] + [
+        (n, ctypes.c_int32) for n in ("feasible", "binding_constraint", "under_occupied", "reserved")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class AttnError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = status_string(code)
+        if code == ERR_CUDA:
+            msg += ": " + last_cuda_error()
+        super().__init__(f"{where} failed: {msg} ({code})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2609_10937_b200.build` "
+                "(there is no CPU fallback)")
+        L = ctypes.CDLL(str(LIB_PATH))
+        vp, i32 = ctypes.c_void_p, ctypes.c_int
+        L.attn_hw_desc_b200.argtypes = [ctypes.POINTER(AttnHwDesc)]
+        L.attn_hw_desc_query.argtypes = [i32, ctypes.POINTER(AttnHwDesc)]
+        L.attn_plan.argtypes = [ctypes.POINTER(AttnHwDesc), i32, i32, i32, i32, ctypes.POINTER(AttnTiles)]
+        L.attn_workspace_bytes.argtypes = [ctypes.POINTER(AttnTiles), i32, i32, i32, i32]
+        L.attn_workspace_bytes.restype = ctypes.c_size_t
+        L.attn_set_workspace.argtypes = [i32, vp, ctypes.c_size_t]
+        L.attn_forward.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+        L.attn_forward_tiles.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, ctypes.POINTER(AttnTiles), vp]
+        L.attn_forward_simple.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
+        L.attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_size_t, vp]
+        L.attn_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+        L.attn_last_launch_count.argtypes = []
+        L.attn_status_string.argtypes = [i32]
+        L.attn_status_string.restype = ctypes.c_char_p
+        L.attn_last_cuda_error.argtypes = []
+        L.attn_last_cuda_error.restype = ctypes.c_char_p
+        for name in EXPORTED_SYMBOLS:
+            getattr(L, name)
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().attn_status_string(int(code)).decode()
+
+
+def last_cuda_error() -> str:
+    return lib().attn_last_cuda_error().decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != ATTN_OK:
+        raise AttnError(code, where)
+
+
+def hw_desc_b200() -> AttnHwDesc:
+    d = AttnHwDesc()
+    _check(lib().attn_hw_desc_b200(ctypes.byref(d)), "attn_hw_desc_b200")
+    return d
+
+
+def hw_desc_query(device: int = 0) -> AttnHwDesc:
+    d = AttnHwDesc()
+    _check(lib().attn_hw_desc_query(int(device), ctypes.byref(d)), "attn_hw_desc_query")
+    return d
+
+
+def plan(desc: AttnHwDesc, B: int, H: int, L: int, d: int) -> AttnTiles:
+    t = AttnTiles()
+    _check(lib().attn_plan(ctypes.byref(desc), B, H, L, d, ctypes.byref(t)), "attn_plan")
+    return t
+
+
+def workspace_bytes(tiles: AttnTiles, B: int, H: int, L: int, d: int) -> int:
+    return int(lib().attn_workspace_bytes(ctypes.byref(tiles), B, H, L, d))
+
+
+# ---------------------------------------------------------------- torch side
+_workspaces = {}   # device index -> torch uint8 tensor registered with the library
+_descs = {}
+
+
+def _device_desc(device_index: int) -> AttnHwDesc:
+    if device_index not in _descs:
+        _descs[device_index] = hw_desc_query(device_index)
+    return _descs[device_index]
+
+
+def ensure_workspace(device_index: int, nbytes: int) -> None:
+    """Keeps a caller-side torch buffer of at least nbytes registered as the workspace."""
+    import torch
+
+    cur = _workspaces.get(device_index)
+    if nbytes <= 0 or (cur is not None and cur.numel() >= nbytes):
+        return
+    buf = torch.empty(int(nbytes), dtype=torch.uint8, device=torch.device("cuda", device_index))
+    _check(lib().attn_set_workspace(device_index, buf.data_ptr(), buf.numel()), "attn_set_workspace")
+    _workspaces[device_index] = buf
+
+
+def _prep(q, k, v, o):
+    import torch
+
+    if q.dtype != torch.bfloat16 or k.dtype != torch.bfloat16 or v.dtype != torch.bfloat16:
+        raise TypeError("q, k, v must be torch.bfloat16")
+    if q.dim() != 4 or q.shape != k.shape or q.shape != v.shape:
+        raise ValueError("q, k, v must share the shape [B, H, L, d]")
+    if not (q.is_cuda and k.is_cuda and v.is_cuda):
+        raise ValueError("q, k, v must be CUDA tensors (there is no CPU path)")
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
+        raise ValueError("q, k, v must be contiguous [B][H][L][d]")
+    if o is None:
+        o = torch.empty_like(q)
+    elif o.shape != q.shape or o.dtype != torch.bfloat16 or not o.is_contiguous() or o.device != q.device:
+        raise ValueError("o must match q in shape, dtype, device and be contiguous")
+    B, H, L, d = (int(x) for x in q.shape)
+    dev = q.device.index if q.device.index is not None else torch.cuda.current_device()
+    stream = torch.cuda.current_stream(q.device).cuda_stream
+    return o, B, H, L, d, dev, stream
+
+
+def forward(q, k, v, o=None):
+    """O = softmax(Q K^T / sqrt(d)) V with the closed-form default tiles (asynchronous)."""
+    import torch
+
+    o, B, H, L, d, dev, stream = _prep(q, k, v, o)
+    with torch.cuda.device(dev):
+        t = plan(_device_desc(dev), B, H, L, d)
+        if t.feasible and t.kv_splits > 1:
+            ensure_workspace(dev, workspace_bytes(t, B, H, L, d))
+        _check(lib().attn_forward(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d, stream),
+               "attn_forward")
+    return o
+
+
+def forward_tiles(q, k, v, o=None, *, n_q=0, tile_kv=0, kv_stages=0, kv_splits=0):
+    """Same with tile fields overridden (0 keeps the closed-form value); tile sweep only."""
+    import torch
+
+    o, B, H, L, d, dev, stream = _prep(q, k, v, o)
+    with torch.cuda.device(dev):
+        base = plan(_device_desc(dev), B, H, L, d)
+        ov = AttnTiles()
+        ov.n_q, ov.tile_kv, ov.kv_stages, ov.kv_splits = n_q, tile_kv, kv_stages, kv_splits
+        eff_nq = n_q or base.n_q
+        eff_splits = kv_splits or base.kv_splits
+        if eff_splits > 1:
+            w = AttnTiles()
+            w.feasible, w.kv_splits, w.n_q = 1, eff_splits, eff_nq
+            w.ctas = B * H * math.ceil(L / (128 * eff_nq)) * eff_splits
+            ensure_workspace(dev, workspace_bytes(w, B, H, L, d))
+        _check(lib().attn_forward_tiles(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d,
+                                        ctypes.byref(ov), stream), "attn_forward_tiles")
+    return o
+
+
+def forward_simple(q, k, v, o=None, *, tile_kv=128, scores_out=None):
+    """Non-pipelined variant; scores_out (fp32 [128, tile_kv], CUDA) receives Q_0 K_0^T of head 0."""
+    import torch
+
+    o, B, H, L, d, dev, stream = _prep(q, k, v, o)
+    sp = None
+    if scores_out is not None:
+        if scores_out.dtype != torch.float32 or scores_out.numel() < 128 * tile_kv or not scores_out.is_cuda:
+            raise ValueError("scores_out must be a CUDA fp32 tensor with at least 128*tile_kv elements")
+        sp = scores_out.data_ptr()
+    with torch.cuda.device(dev):
+        _check(lib().attn_forward_simple(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d,
+                                         int(tile_kv), sp, stream), "attn_forward_simple")
+    return o
+
+
+def forward_host(q_host, k_host, v_host, o_host, dev_scratch):
+    """Host-buffer entry point: pinned host bf16 tensors in, pinned host tensor out.
+
+    dev_scratch is a caller-owned CUDA uint8 tensor of at least 4 * q.nbytes bytes.
+    Copies and kernels are queued on the current stream; nothing is synchronised.
+    """
+    import torch
+
+    B, H, L, d = (int(x) for x in q_host.shape)
+    dev = dev_scratch.device.index
+    stream = torch.cuda.current_stream(dev_scratch.device).cuda_stream
+    with torch.cuda.device(dev):
+        t = plan(_device_desc(dev), B, H, L, d)
+        if t.feasible and t.kv_splits > 1:
+            ensure_workspace(dev, workspace_bytes(t, B, H, L, d))
+        _check(lib().attn_forward_host(q_host.data_ptr(), k_host.data_ptr(), v_host.data_ptr(), o_host.data_ptr(),
+                                       B, H, L, d, dev_scratch.data_ptr(), dev_scratch.numel(), stream),
+               "attn_forward_host")
+    return o_host
+
+
+def last_device_status(device=None):
+    """Synchronises the current stream; returns (code, detail words)."""
+    import torch
+
+    dev = torch.cuda.current_device() if device is None else device
+    detail = (ctypes.c_uint32 * 4)()
+    with torch.cuda.device(dev):
+        stream = torch.cuda.current_stream().cuda_stream
+        code = lib().attn_last_device_status(stream, detail)
+    return int(code), [int(x) for x in detail]
+
+
+def last_launch_count() -> int:
+    return int(lib().attn_last_launch_count())

@@ -1,0 +1,332 @@
+// C ABI of the fused-attention library: argument checks, closed-form plan,
+// TMA tensor maps, kernel launches.  No device memory is allocated here.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "attn.h"
+#include "attn_kernels.cuh"
+
+namespace {
+
+thread_local char t_cuda_error[256] = "";
+thread_local int t_launch_count = 0;
+
+int cuda_fail(cudaError_t e, const char* what) {
+  std::snprintf(t_cuda_error, sizeof t_cuda_error, "%s: %s", what, cudaGetErrorString(e));
+  return ATTN_ERR_CUDA;
+}
+#define ATTN_CUDA_TRY(expr)                               \
+  do {                                                    \
+    cudaError_t e__ = (expr);                             \
+    if (e__ != cudaSuccess) return cuda_fail(e__, #expr); \
+  } while (0)
+
+// ---- driver entry point for tensor-map encoding (no link-time libcuda dependency)
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// 3-D map over a contiguous [BH][L][d] bf16 tensor; box = (64 columns, box_rows rows, 1 head), 128-byte swizzle.
+int make_tmap(CUtensorMap* m, const void* base, int BH, int L, int d, int box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) {
+    std::snprintf(t_cuda_error, sizeof t_cuda_error, "cuTensorMapEncodeTiled entry point not found");
+    return ATTN_ERR_CUDA;
+  }
+  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)L, (cuuint64_t)BH};
+  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)L * (cuuint64_t)d * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    std::snprintf(t_cuda_error, sizeof t_cuda_error, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return ATTN_ERR_CUDA;
+  }
+  return ATTN_OK;
+}
+
+// ---- per-device state: workspace registry and cached descriptor
+constexpr int kMaxDevices = 64;
+struct DeviceState {
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  bool arch_checked = false;
+  bool arch_ok = false;
+  attn_hw_desc desc;
+};
+DeviceState g_dev[kMaxDevices];
+std::mutex g_mu;
+
+int device_state(DeviceState** out) {
+  int dev = 0;
+  ATTN_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return ATTN_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(g_mu);
+  DeviceState& s = g_dev[dev];
+  if (!s.arch_checked) {
+    int rc = attn_hw_desc_query(dev, &s.desc);
+    if (rc == ATTN_ERR_CUDA) return rc;
+    s.arch_ok = (rc == ATTN_OK);
+    s.arch_checked = true;
+  }
+  *out = &s;
+  return s.arch_ok ? ATTN_OK : ATTN_ERR_WRONG_ARCH;
+}
+
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+  return a0 < b0 + nb && b0 < a0 + na;
+}
+
+int check_args(const void* q, const void* k, const void* v, const void* o, int B, int H, int L, int d) {
+  if (!q || !k || !v || !o || B <= 0 || H <= 0 || L <= 0 || d <= 0) return ATTN_ERR_INVALID_ARG;
+  if ((d != 64 && d != 128) || (L % 128) != 0) return ATTN_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)B * H * (L / 128) > 0x3FFFFFFFLL) return ATTN_ERR_UNSUPPORTED_SHAPE;  // grid index range
+  if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15u) return ATTN_ERR_MISALIGNED;
+  const size_t bytes = (size_t)B * H * L * d * 2;
+  if (overlaps(o, bytes, q, bytes) || overlaps(o, bytes, k, bytes) || overlaps(o, bytes, v, bytes))
+    return ATTN_ERR_ALIASING;
+  return ATTN_OK;
+}
+
+template <int D, int TKV, int NQ>
+int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int L, const attn_tiles& t,
+               float* ws, cudaStream_t stream) {
+  using SM = attn::FwdSmem<D, TKV, NQ>;
+  const int BH = B * H;
+  CUtensorMap tq, tk, tv, to;
+  int rc;
+  if ((rc = make_tmap(&tq, q, BH, L, D, attn::kSub)) != ATTN_OK) return rc;
+  if ((rc = make_tmap(&tk, k, BH, L, D, TKV)) != ATTN_OK) return rc;
+  if ((rc = make_tmap(&tv, v, BH, L, D, TKV)) != ATTN_OK) return rc;
+  if ((rc = make_tmap(&to, o, BH, L, D, attn::kSub)) != ATTN_OK) return rc;
+
+  attn::FwdParams p;
+  p.L = L;
+  p.q_tiles = (L + NQ * attn::kSub - 1) / (NQ * attn::kSub);
+  p.n_steps = L / TKV;
+  p.kv_splits = t.kv_splits;
+  p.stages = t.kv_stages;
+  p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
+  p.ws = ws;
+  const int smem = SM::total(t.kv_stages);
+  auto kern = attn::attn_fwd_kernel<D, TKV, NQ>;
+  ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  const int grid = BH * p.q_tiles * t.kv_splits;
+  kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
+  ATTN_CUDA_TRY(cudaGetLastError());
+  t_launch_count = 1;
+  if (t.kv_splits > 1) {
+    attn::attn_merge_kernel<D, NQ><<<BH * p.q_tiles * NQ, 128, 0, stream>>>(
+        ws, reinterpret_cast<__nv_bfloat16*>(o), L, p.q_tiles, t.kv_splits);
+    ATTN_CUDA_TRY(cudaGetLastError());
+    t_launch_count = 2;
+  }
+  return ATTN_OK;
+}
+
+int dispatch_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
+                 const attn_tiles& t, float* ws, cudaStream_t s) {
+#define ATTN_CASE(D_, TKV_, NQ_) \
+  if (d == D_ && t.tile_kv == TKV_ && t.n_q == NQ_) return launch_fwd<D_, TKV_, NQ_>(q, k, v, o, B, H, L, t, ws, s);
+  ATTN_CASE(128, 128, 2)
+  ATTN_CASE(128, 64, 2)
+  ATTN_CASE(128, 128, 1)
+  ATTN_CASE(128, 64, 1)
+  ATTN_CASE(64, 128, 2)
+  ATTN_CASE(64, 64, 2)
+  ATTN_CASE(64, 128, 1)
+  ATTN_CASE(64, 64, 1)
+#undef ATTN_CASE
+  return ATTN_ERR_BAD_TILES;
+}
+
+int forward_impl(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
+                 const attn_tiles* ovr, void* cuda_stream) {
+  t_launch_count = 0;
+  int rc = check_args(q, k, v, o, B, H, L, d);
+  if (rc != ATTN_OK) return rc;
+  DeviceState* st = nullptr;
+  if ((rc = device_state(&st)) != ATTN_OK) return rc;
+  attn_tiles t;
+  if ((rc = attn_plan(&st->desc, B, H, L, d, &t)) != ATTN_OK) return rc;
+  if (!t.feasible) return ATTN_ERR_INFEASIBLE_PLAN;
+  if (ovr) {
+    if (ovr->n_q > 0) t.n_q = ovr->n_q;
+    if (ovr->tile_kv > 0) t.tile_kv = ovr->tile_kv;
+    if (t.n_q != 1 && t.n_q != 2) return ATTN_ERR_BAD_TILES;
+    if (t.tile_kv != 64 && t.tile_kv != 128) return ATTN_ERR_BAD_TILES;
+    const int q_bytes = t.n_q * 128 * d * 2, stage = t.tile_kv * d * 2;
+    int max_stages = (st->desc.local_mem_bytes - q_bytes - 3072) / stage;
+    if (max_stages > attn::kMaxStages) max_stages = attn::kMaxStages;
+    t.kv_stages = ovr->kv_stages > 0 ? ovr->kv_stages : max_stages;
+    if (t.kv_stages < 2 || t.kv_stages > max_stages) return ATTN_ERR_BAD_TILES;
+    t.tile_q = t.n_q * 128;
+    t.tiles = B * H * ((L + t.tile_q - 1) / t.tile_q);
+    if (ovr->kv_splits > 0) t.kv_splits = ovr->kv_splits;
+    if (t.kv_splits < 1 || t.kv_splits > L / t.tile_kv) return ATTN_ERR_BAD_TILES;
+    t.ctas = t.tiles * t.kv_splits;
+    t.smem_bytes = q_bytes + t.kv_stages * stage + 3072;
+  }
+  float* ws = nullptr;
+  if (t.kv_splits > 1) {
+    const size_t need = attn_workspace_bytes(&t, B, H, L, d);
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!st->ws || st->ws_bytes < need) return ATTN_ERR_NEED_WORKSPACE;
+    ws = static_cast<float*>(st->ws);
+  }
+  return dispatch_fwd(q, k, v, o, B, H, L, d, t, ws, static_cast<cudaStream_t>(cuda_stream));
+}
+
+template <int D, int TKV>
+int launch_simple(const void* q, const void* k, const void* v, void* o, int B, int H, int L, float* scores_out,
+                  cudaStream_t stream) {
+  const int BH = B * H;
+  CUtensorMap tq, tk, tv;
+  int rc;
+  if ((rc = make_tmap(&tq, q, BH, L, D, attn::kSub)) != ATTN_OK) return rc;
+  if ((rc = make_tmap(&tk, k, BH, L, D, TKV)) != ATTN_OK) return rc;
+  if ((rc = make_tmap(&tv, v, BH, L, D, TKV)) != ATTN_OK) return rc;
+  const int smem = attn::kSub * D * 2 + 2 * TKV * D * 2 + 1024;
+  auto kern = attn::attn_fwd_simple_kernel<D, TKV>;
+  ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  const char* dbg = std::getenv("ATTN_SIMPLE_DEBUG_FLAGS");
+  const int flags = dbg ? std::atoi(dbg) : 0;
+  const float scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
+  dim3 grid(L / attn::kSub, BH);
+  kern<<<grid, 128, smem, stream>>>(tq, tk, tv, reinterpret_cast<__nv_bfloat16*>(o), L, scale_log2, scores_out, flags);
+  ATTN_CUDA_TRY(cudaGetLastError());
+  t_launch_count = 1;
+  return ATTN_OK;
+}
+
+}  // namespace
+
+extern "C" int attn_hw_desc_query(int device, attn_hw_desc* out) {
+  if (!out) return ATTN_ERR_INVALID_ARG;
+  int major = 0, minor = 0, sms = 0, smem_optin = 0, regs = 0, clock_khz = 0;
+  ATTN_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
+  ATTN_CUDA_TRY(cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, device));
+  if (major != 10) return ATTN_ERR_WRONG_ARCH;
+  attn_hw_desc_b200(out);  // per-architecture constants (tensor memory, atom shapes)
+  ATTN_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+  ATTN_CUDA_TRY(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
+  ATTN_CUDA_TRY(cudaDeviceGetAttribute(&regs, cudaDevAttrMaxRegistersPerMultiprocessor, device));
+  ATTN_CUDA_TRY(cudaDeviceGetAttribute(&clock_khz, cudaDevAttrClockRate, device));
+  out->num_units = sms;
+  out->local_mem_bytes = smem_optin;
+  out->regs_per_unit = regs;
+  out->sm_clock_mhz = clock_khz / 1000.0;
+  // dense bf16: 8192 FLOP per clock per SM
+  out->peak_tflops = 8192.0 * sms * (clock_khz * 1e3) / 1e12;
+  return ATTN_OK;
+}
+
+extern "C" int attn_set_workspace(int device, void* dev_ptr, size_t bytes) {
+  if (device < 0 || device >= kMaxDevices) return ATTN_ERR_INVALID_ARG;
+  if (dev_ptr && ((uintptr_t)dev_ptr & 15u)) return ATTN_ERR_MISALIGNED;
+  std::lock_guard<std::mutex> lk(g_mu);
+  g_dev[device].ws = dev_ptr;
+  g_dev[device].ws_bytes = dev_ptr ? bytes : 0;
+  return ATTN_OK;
+}
+
+extern "C" int attn_forward(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
+                            void* cuda_stream) {
+  return forward_impl(q, k, v, o, B, H, L, d, nullptr, cuda_stream);
+}
+
+extern "C" int attn_forward_tiles(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
+                                  const attn_tiles* override_tiles, void* cuda_stream) {
+  return forward_impl(q, k, v, o, B, H, L, d, override_tiles, cuda_stream);
+}
+
+extern "C" int attn_forward_simple(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
+                                   int tile_kv, float* scores_out, void* cuda_stream) {
+  t_launch_count = 0;
+  int rc = check_args(q, k, v, o, B, H, L, d);
+  if (rc != ATTN_OK) return rc;
+  DeviceState* st = nullptr;
+  if ((rc = device_state(&st)) != ATTN_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (d == 128 && tile_kv == 128) return launch_simple<128, 128>(q, k, v, o, B, H, L, scores_out, s);
+  if (d == 128 && tile_kv == 64) return launch_simple<128, 64>(q, k, v, o, B, H, L, scores_out, s);
+  if (d == 64 && tile_kv == 128) return launch_simple<64, 128>(q, k, v, o, B, H, L, scores_out, s);
+  if (d == 64 && tile_kv == 64) return launch_simple<64, 64>(q, k, v, o, B, H, L, scores_out, s);
+  return ATTN_ERR_BAD_TILES;
+}
+
+extern "C" int attn_forward_host(const void* q_host, const void* k_host, const void* v_host, void* o_host, int B,
+                                 int H, int L, int d, void* dev_scratch, size_t dev_scratch_bytes,
+                                 void* cuda_stream) {
+  if (!q_host || !k_host || !v_host || !o_host || !dev_scratch || B <= 0 || H <= 0 || L <= 0 || d <= 0)
+    return ATTN_ERR_INVALID_ARG;
+  const size_t bytes = (size_t)B * H * L * d * 2;
+  if (dev_scratch_bytes < 4 * bytes || ((uintptr_t)dev_scratch & 255u)) return ATTN_ERR_INVALID_ARG;
+  char* base = static_cast<char*>(dev_scratch);
+  void *dq = base, *dk = base + bytes, *dv = base + 2 * bytes, *dout = base + 3 * bytes;
+  int rc = check_args(dq, dk, dv, dout, B, H, L, d);
+  if (rc != ATTN_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  ATTN_CUDA_TRY(cudaMemcpyAsync(dq, q_host, bytes, cudaMemcpyHostToDevice, s));
+  ATTN_CUDA_TRY(cudaMemcpyAsync(dk, k_host, bytes, cudaMemcpyHostToDevice, s));
+  ATTN_CUDA_TRY(cudaMemcpyAsync(dv, v_host, bytes, cudaMemcpyHostToDevice, s));
+  rc = forward_impl(dq, dk, dv, dout, B, H, L, d, nullptr, cuda_stream);
+  if (rc != ATTN_OK) return rc;
+  ATTN_CUDA_TRY(cudaMemcpyAsync(o_host, dout, bytes, cudaMemcpyDeviceToHost, s));
+  return ATTN_OK;
+}
+
+extern "C" int attn_last_device_status(void* cuda_stream, uint32_t* detail) {
+  ATTN_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+  unsigned int h[4] = {0, 0, 0, 0};
+  ATTN_CUDA_TRY(cudaMemcpyFromSymbol(h, attn::g_attn_dev_status, sizeof h));
+  if (detail)
+    for (int i = 0; i < 4; ++i) detail[i] = h[i];
+  if (h[0] == 0) return ATTN_OK;
+  unsigned int z[4] = {0, 0, 0, 0};
+  ATTN_CUDA_TRY(cudaMemcpyToSymbol(attn::g_attn_dev_status, z, sizeof z));
+  return ATTN_ERR_DEVICE_TIMEOUT;
+}
+
+extern "C" int attn_last_launch_count(void) { return t_launch_count; }
+
+extern "C" const char* attn_last_cuda_error(void) { return t_cuda_error; }
+
+extern "C" const char* attn_status_string(int status) {
+  switch (status) {
+    case ATTN_OK: return "ok";
+    case ATTN_ERR_INVALID_ARG: return "invalid argument";
+    case ATTN_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (need d in {64,128} and L a multiple of 128)";
+    case ATTN_ERR_MISALIGNED: return "device pointer not 16-byte aligned";
+    case ATTN_ERR_ALIASING: return "output overlaps an input";
+    case ATTN_ERR_INFEASIBLE_PLAN: return "no feasible tile plan";
+    case ATTN_ERR_WRONG_ARCH: return "device is not compute capability 10.x";
+    case ATTN_ERR_NEED_WORKSPACE: return "plan splits the key axis: register a workspace with attn_set_workspace";
+    case ATTN_ERR_CUDA: return "CUDA error (see attn_last_cuda_error)";
+    case ATTN_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case ATTN_ERR_BAD_TILES: return "tile override not available";
+    default: return "unknown status";
+  }
+}

@@ -1,0 +1,644 @@
+// sm_100a kernels for the fused attention forward pass (Algorithm 1 of the
+// paper: K/V tiles streamed through an online softmax; the score tile never
+// leaves the chip).
+//
+//   attn_fwd_kernel        warp-specialised, pipelined: TMA producer warp ->
+//                          shared-memory K/V ring -> one MMA-issuing thread
+//                          (tcgen05.mma, S = Q K^T into tensor memory) ->
+//                          two softmax warpgroups (one Q sub-tile each, one
+//                          thread per row) -> P as bf16 back into tensor
+//                          memory -> second tcgen05.mma (O += P V, A operand
+//                          read from tensor memory) ; a correction warpgroup
+//                          rescales O when the running maximum moved.
+//   attn_merge_kernel      merge operator of the online softmax over the
+//                          partial results of CTAs that split the key axis.
+//   attn_fwd_simple_kernel the same algorithm with nothing overlapped; used to
+//                          cross-check the pipelined kernel and the layouts.
+//
+// Every device-side wait is bounded: on expiry the CTA records an error word
+// in g_attn_dev_status, raises a CTA-wide abort flag and all roles drain.
+#pragma once
+
+#include "ptx_sm100.cuh"
+
+namespace attn {
+
+using namespace sm100;
+
+constexpr int kSub = 128;                 // rows of one Q sub-tile = tensor-memory lanes
+constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz
+
+// [0] error code (0 = none), [1] role<<24 | barrier<<16 | step, [2] CTA index, [3] spare
+__device__ unsigned int g_attn_dev_status[4];
+
+enum Role : uint32_t { kRoleLoad = 1, kRoleMma = 2, kRoleSoftmax = 3, kRoleCorrection = 4, kRoleSimple = 5 };
+enum BarId : uint32_t { kBarQ = 1, kBarKvFull = 2, kBarKvEmpty = 3, kBarSFull = 4, kBarPFull = 5, kBarOFull = 6,
+                        kBarAlpha = 7, kBarLoad = 8, kBarMma = 9, kBarSync = 10 };
+
+__device__ __noinline__ void report_timeout(uint32_t info) {
+  if (atomicCAS(&g_attn_dev_status[0], 0u, 1u) == 0u) {
+    g_attn_dev_status[1] = info;
+    g_attn_dev_status[2] = blockIdx.x + gridDim.x * blockIdx.y;
+    __threadfence();
+  }
+}
+
+// Bounded mbarrier wait.  Returns false if the CTA aborted or the limit expired.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t info) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t it = 0;
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++it & 127u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitLimitCycles) {
+        report_timeout(info);
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+// Same, for roles whose warps run warp-collective instructions afterwards: the verdict is made warp-uniform.
+__device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t info) {
+  return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_flag, info) ? 1 : 0) != 0;
+}
+__device__ __forceinline__ uint32_t wait_info(uint32_t role, uint32_t bar, uint32_t step) {
+  return (role << 24) | (bar << 16) | (step & 0xFFFFu);
+}
+
+// ---------------------------------------------------------------------------
+// Matrix-product issue helpers (one thread).
+// Q and K tiles: K-major, [rows][64] bf16 chunks with 128-byte swizzle, chunk c
+// holds head-dimension columns [64c, 64c+64).  V tile: same storage, used as
+// the MN-major B operand of the second product (N = head dimension).
+// ---------------------------------------------------------------------------
+template <int D, int TKV>
+__device__ __forceinline__ void issue_qk(uint32_t s_tmem, uint32_t q_smem, uint32_t k_smem) {
+  constexpr uint32_t idesc = make_idesc_bf16(kSub, TKV, false);
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks) {
+    const uint32_t chunk = ks >> 2, kin = ks & 3;
+    const uint64_t a = make_smem_desc_sw128(q_smem + chunk * (kSub * 128) + kin * 32, 16, 1024);
+    const uint64_t b = make_smem_desc_sw128(k_smem + chunk * (TKV * 128) + kin * 32, 16, 1024);
+    umma_ss(s_tmem, a, b, idesc, ks > 0 ? 1u : 0u);
+  }
+}
+template <int D, int TKV>
+__device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_smem, bool accumulate,
+                                         uint32_t lbo, uint32_t sbo) {
+  constexpr uint32_t idesc = make_idesc_bf16(kSub, D, true);
+#pragma unroll
+  for (int ks = 0; ks < TKV / 16; ++ks) {
+    // 16 key rows per step: two 8-row groups of 1024 bytes
+    const uint64_t b = make_smem_desc_sw128(v_smem + ks * 2048, lbo, sbo);
+    umma_ts(o_tmem, p_tmem + ks * 8, b, idesc, (accumulate || ks > 0) ? 1u : 0u);
+  }
+}
+
+struct FwdParams {
+  int L;             // sequence length
+  int q_tiles;       // Q tiles per head = ceil(L / (NQ*128))
+  int n_steps;       // KV steps per head = L / TKV
+  int kv_splits;     // CTAs per Q tile along the key axis
+  int stages;        // ring depth
+  float scale_log2;  // log2(e) / sqrt(d)
+  float* ws;         // partial results when kv_splits > 1
+};
+
+// Shared-memory footprint helpers (host and device agree through these).
+template <int D, int TKV, int NQ>
+struct FwdSmem {
+  static constexpr int kQBytes = NQ * kSub * D * 2;
+  static constexpr int kStageBytes = TKV * D * 2;
+  static constexpr int kMiscBytes = 3072;
+  __host__ __device__ static constexpr int total(int stages) { return kQBytes + stages * kStageBytes + kMiscBytes; }
+};
+
+constexpr int kMaxStages = 8;
+
+struct FwdMisc {               // lives in the last 3072 bytes of dynamic shared memory
+  float alpha[2][2][kSub];     // [sub-tile][step parity][row] rescale factor
+  uint64_t q_full;
+  uint64_t kv_full[kMaxStages];
+  uint64_t kv_empty[kMaxStages];
+  uint64_t s_full[2];
+  uint64_t p_full[2];
+  uint64_t o_full[2];
+  uint64_t alpha_full[2];
+  uint64_t epi_sync[2];        // softmax warpgroup rendezvous before the TMA store
+  uint32_t tmem_slot;
+  int abort_flag;
+};
+static_assert(sizeof(FwdMisc) <= 3072, "misc region too large");
+
+// Workspace layout for split keys: per (CTA, sub-tile): O[D/4][128][4] fp32, m[128], delta[128].
+__host__ __device__ constexpr size_t ws_floats_per_sub(int d) { return (size_t)kSub * d + 2 * kSub; }
+
+template <int D, int TKV, int NQ>
+__global__ void __launch_bounds__(512, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                const FwdParams p) {
+  static_assert(D == 64 || D == 128, "head dimension");
+  static_assert(TKV == 64 || TKV == 128, "KV tile");
+  constexpr int KCH = D / 64;                         // 64-column chunks per row
+  constexpr int S_COLS = TKV;                         // fp32 score columns per sub-tile
+  constexpr int O_COL0 = NQ * S_COLS;                 // O accumulators follow the score buffers
+  constexpr int TMEM_COLS = (NQ * (S_COLS + D) <= 32) ? 32
+                          : (NQ * (S_COLS + D) <= 64) ? 64
+                          : (NQ * (S_COLS + D) <= 128) ? 128
+                          : (NQ * (S_COLS + D) <= 256) ? 256 : 512;
+  using SM = FwdSmem<D, TKV, NQ>;
+
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = smem_u32(smem_raw);
+  const uint32_t q_smem = smem_base;
+  const uint32_t ring_smem = smem_base + SM::kQBytes;
+  FwdMisc* misc = reinterpret_cast<FwdMisc*>(smem_raw + SM::kQBytes + p.stages * SM::kStageBytes);
+  volatile int* abort_flag = &misc->abort_flag;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  // Work assignment: split fastest, then Q tile, then head, so that CTAs of one
+  // head are neighbours in launch order and share K/V through L2.
+  const int cta = blockIdx.x;
+  const int split = cta % p.kv_splits;
+  const int tile = cta / p.kv_splits;
+  const int q_tile = tile % p.q_tiles;
+  const int bh = tile / p.q_tiles;
+  const int j0 = (int)(((long long)split * p.n_steps) / p.kv_splits);
+  const int j1 = (int)(((long long)(split + 1) * p.n_steps) / p.kv_splits);
+  const int n = j1 - j0;
+  const int q_row0 = q_tile * NQ * kSub;
+
+  if (threadIdx.x == 0) {
+    misc->abort_flag = 0;
+    if (smem_base & 1023u) {                 // swizzled tiles need 1024-byte alignment
+      report_timeout(wait_info(kRoleLoad, 0, 0xFFFF));
+      misc->abort_flag = 1;
+    }
+    mbar_init(smem_u32(&misc->q_full), 1);
+    for (int s = 0; s < kMaxStages; ++s) {
+      mbar_init(smem_u32(&misc->kv_full[s]), 1);
+      mbar_init(smem_u32(&misc->kv_empty[s]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&misc->s_full[i]), 1);
+      mbar_init(smem_u32(&misc->p_full[i]), 2 * kSub);   // softmax rows + correction rows
+      mbar_init(smem_u32(&misc->o_full[i]), 1);
+      mbar_init(smem_u32(&misc->alpha_full[i]), kSub);
+      mbar_init(smem_u32(&misc->epi_sync[i]), kSub);
+    }
+    fence_mbar_init();
+    prefetch_tmap(&tm_q);
+    prefetch_tmap(&tm_k);
+    prefetch_tmap(&tm_v);
+    prefetch_tmap(&tm_o);
+  }
+  if (warp == 13) {
+    tmem_alloc(smem_u32(&misc->tmem_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = misc->tmem_slot;
+  const bool run = (*abort_flag == 0) && n > 0;
+
+  if (warp < 4 * NQ) {
+    // ===================================================== softmax warpgroup
+    setmaxnreg_inc<(NQ == 2) ? 192 : 232>();
+    const int i = warp >> 2;
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t s_tmem = lane_base + i * S_COLS;
+    const uint32_t o_tmem = lane_base + O_COL0 + i * D;
+    const uint32_t bar_s = smem_u32(&misc->s_full[i]);
+    const uint32_t bar_p = smem_u32(&misc->p_full[i]);
+    const uint32_t bar_a = smem_u32(&misc->alpha_full[i]);
+    float m_run = -INFINITY, delta = 0.f;
+    bool ok = run;
+    for (int jj = 0; ok && jj < n; ++jj) {
+      if (!wait_bar_warp(bar_s, jj & 1, abort_flag, wait_info(kRoleSoftmax, kBarSFull, jj))) { ok = false; break; }
+      tc_fence_after();
+      uint32_t s[TKV];
+#pragma unroll
+      for (int c = 0; c < TKV / 32; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+#pragma unroll
+      for (int c = 0; c < TKV / 32; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      float mx = __uint_as_float(s[0]);
+#pragma unroll
+      for (int k = 1; k < TKV; ++k) mx = fmaxf(mx, __uint_as_float(s[k]));
+      const float m_new = fmaxf(m_run, mx * p.scale_log2);
+      const float alpha = ex2_approx(m_run - m_new);     // 0 on the first step (m_run = -inf)
+      misc->alpha[i][jj & 1][row] = alpha;
+      mbar_arrive(bar_a);
+      const float neg_m = -m_new;
+      float sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < TKV / 32; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const float e0 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + 2 * k]), p.scale_log2, neg_m));
+          const float e1 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + 2 * k + 1]), p.scale_log2, neg_m));
+          sum += e0 + e1;
+          pk[k] = pack_bf16x2(e0, e1);
+        }
+        tmem_st16(s_tmem + c * 16, pk);                  // P aliases the front of the S buffer
+      }
+      delta = delta * alpha + sum;
+      m_run = m_new;
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_p);
+    }
+    // ------------------------------------------------------------- epilogue
+    if (ok) ok = wait_bar_warp(smem_u32(&misc->o_full[i]), (n - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, n));
+    if (ok) {
+      tc_fence_after();
+      if (p.kv_splits == 1) {
+        const float inv = 1.0f / delta;
+        const uint32_t stage_out = q_smem + i * (kSub * D * 2);   // Q sub-tile is dead: reuse it
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(o_tmem + c * 32, r);
+          const uint32_t chunk_base = stage_out + (c >> 1) * (kSub * 128) + row * 128;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              w[e] = pack_bf16x2(__uint_as_float(r[u * 8 + 2 * e]) * inv, __uint_as_float(r[u * 8 + 2 * e + 1]) * inv);
+            const uint32_t unit = (uint32_t)((c & 1) * 4 + u) ^ (uint32_t)(row & 7);   // 128-byte swizzle
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                         ::"r"(chunk_base + unit * 16), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+          }
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(smem_u32(&misc->epi_sync[i]));
+        if ((warp & 3) == 0 && lane == 0 &&
+            wait_bar(smem_u32(&misc->epi_sync[i]), 0, abort_flag, wait_info(kRoleSoftmax, kBarSync, n))) {
+#pragma unroll
+          for (int c = 0; c < KCH; ++c)
+            tma_store_3d(&tm_o, stage_out + c * (kSub * 128), c * 64, q_row0 + i * kSub, bh);
+          tma_store_commit();
+          tma_store_wait_read();
+        }
+      } else {
+        float* ws = p.ws + ((size_t)cta * NQ + i) * ws_floats_per_sub(D);
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(o_tmem + c * 32, r);
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            float4 v4 = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]),
+                                    __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
+            reinterpret_cast<float4*>(ws)[(size_t)(c * 8 + g) * kSub + row] = v4;
+          }
+        }
+        ws[(size_t)kSub * D + row] = m_run;
+        ws[(size_t)kSub * D + kSub + row] = delta;
+      }
+    }
+  } else if (warp >= 8 && warp < 12) {
+    // ================================================== correction warpgroup
+    setmaxnreg_dec<80>();
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    bool ok = run;
+    for (int jj = 0; ok && jj < n; ++jj) {
+#pragma unroll
+      for (int i = 0; i < NQ; ++i) {
+        if (!wait_bar_warp(smem_u32(&misc->alpha_full[i]), jj & 1, abort_flag, wait_info(kRoleCorrection, kBarAlpha, jj))) {
+          ok = false;
+          break;
+        }
+        const float a = misc->alpha[i][jj & 1][row];
+        if (jj > 0) {
+          const bool need = __any_sync(0xffffffffu, a != 1.0f);
+          if (need) {
+            if (!wait_bar_warp(smem_u32(&misc->o_full[i]), (jj - 1) & 1, abort_flag,
+                               wait_info(kRoleCorrection, kBarOFull, jj))) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t o_tmem = lane_base + O_COL0 + i * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t r[32];
+              tmem_ld32(o_tmem + c * 32, r);
+#pragma unroll
+              for (int k = 0; k < 32; ++k) r[k] = __float_as_uint(__uint_as_float(r[k]) * a);
+              tmem_st32(o_tmem + c * 32, r);
+            }
+            tmem_wait_st();
+          }
+          tc_fence_before();
+        }
+        mbar_arrive(smem_u32(&misc->p_full[i]));
+      }
+    }
+  } else if (warp == 12) {
+    // ============================================================ MMA issuer
+    setmaxnreg_dec<48>();
+    if (lane == 0 && run) {
+      bool ok = wait_bar(smem_u32(&misc->q_full), 0, abort_flag, wait_info(kRoleMma, kBarQ, 0));
+      int stage = 0;
+      uint32_t phase = 0;
+      auto advance = [&]() { if (++stage == p.stages) { stage = 0; phase ^= 1u; } };
+      if (ok) ok = wait_bar(smem_u32(&misc->kv_full[stage]), phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 0));
+      if (ok) {
+        tc_fence_after();
+#pragma unroll
+        for (int i = 0; i < NQ; ++i) {
+          issue_qk<D, TKV>(tmem_base + i * S_COLS, q_smem + i * (kSub * D * 2), ring_smem + stage * SM::kStageBytes);
+          umma_commit(smem_u32(&misc->s_full[i]));
+        }
+        umma_commit(smem_u32(&misc->kv_empty[stage]));
+        advance();
+      }
+      for (int jj = 0; ok && jj < n; ++jj) {
+        const int v_stage = stage;
+        const uint32_t v_phase = phase;
+        advance();
+        const int k_stage = stage;
+        const uint32_t k_phase = phase;
+        const bool more = (jj + 1 < n);
+        if (more) advance();
+        if (!wait_bar(smem_u32(&misc->kv_full[v_stage]), v_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 2 * jj + 1))) { ok = false; break; }
+        if (more && !wait_bar(smem_u32(&misc->kv_full[k_stage]), k_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 2 * jj + 2))) { ok = false; break; }
+#pragma unroll
+        for (int i = 0; i < NQ; ++i) {
+          if (!wait_bar(smem_u32(&misc->p_full[i]), jj & 1, abort_flag, wait_info(kRoleMma, kBarPFull, jj))) { ok = false; break; }
+          tc_fence_after();
+          issue_pv<D, TKV>(tmem_base + O_COL0 + i * D, tmem_base + i * S_COLS, ring_smem + v_stage * SM::kStageBytes,
+                           jj > 0, TKV * 128, 1024);
+          umma_commit(smem_u32(&misc->o_full[i]));
+          if (i == NQ - 1) umma_commit(smem_u32(&misc->kv_empty[v_stage]));
+          if (more) {
+            issue_qk<D, TKV>(tmem_base + i * S_COLS, q_smem + i * (kSub * D * 2), ring_smem + k_stage * SM::kStageBytes);
+            umma_commit(smem_u32(&misc->s_full[i]));
+            if (i == NQ - 1) umma_commit(smem_u32(&misc->kv_empty[k_stage]));
+          }
+        }
+      }
+    }
+  } else if (warp == 13) {
+    // ========================================================== TMA producer
+    setmaxnreg_dec<48>();
+    if (lane == 0 && run) {
+      mbar_arrive_expect_tx(smem_u32(&misc->q_full), SM::kQBytes);
+#pragma unroll
+      for (int i = 0; i < NQ; ++i)
+#pragma unroll
+        for (int c = 0; c < KCH; ++c)
+          tma_load_3d(q_smem + i * (kSub * D * 2) + c * (kSub * 128), &tm_q, c * 64, q_row0 + i * kSub, bh,
+                      smem_u32(&misc->q_full));
+      int stage = 0;
+      uint32_t phase = 0;
+      int issued = 0;
+      bool ok = true;
+      for (int t = 0; t < 2 * n; ++t) {
+        if (!wait_bar(smem_u32(&misc->kv_empty[stage]), phase ^ 1u, abort_flag, wait_info(kRoleLoad, kBarKvEmpty, t))) { ok = false; break; }
+        const uint32_t bar = smem_u32(&misc->kv_full[stage]);
+        mbar_arrive_expect_tx(bar, SM::kStageBytes);
+        const CUtensorMap* tm = (t & 1) ? &tm_v : &tm_k;
+        const int kv_row = (j0 + (t >> 1)) * TKV;
+        const uint32_t dst = ring_smem + stage * SM::kStageBytes;
+#pragma unroll
+        for (int c = 0; c < KCH; ++c) tma_load_3d(dst + c * (TKV * 128), tm, c * 64, kv_row, bh, bar);
+        ++issued;
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) {
+        // Drain: every copy this thread started must land before the CTA may exit.
+        const int first = issued > p.stages ? issued - p.stages : 0;
+        for (int t = first; t < issued; ++t) {
+          const int s = t % p.stages;
+          const uint32_t ph = (uint32_t)(t / p.stages) & 1u;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(smem_u32(&misc->kv_full[s]), ph) && clock64() - t0 < kWaitLimitCycles) {}
+        }
+        const long long t0 = clock64();
+        while (!mbar_try_wait(smem_u32(&misc->q_full), 0) && clock64() - t0 < kWaitLimitCycles) {}
+      }
+    }
+  } else {
+    setmaxnreg_dec<48>();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 13) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Merge of split-key partials: (m, delta, O)_a (+) (m, delta, O)_b applied over
+// the splits of one Q sub-tile in ascending split order, then O / delta.
+// One block of 128 threads per (tile, sub-tile); thread = row.
+// ---------------------------------------------------------------------------
+template <int D, int NQ>
+__global__ void __launch_bounds__(128) attn_merge_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o,
+                                                         int L, int q_tiles, int kv_splits) {
+  const int tile = blockIdx.x / NQ;
+  const int i = blockIdx.x % NQ;
+  const int row = threadIdx.x;
+  const int q_tile = tile % q_tiles;
+  const int bh = tile / q_tiles;
+  const int grow = q_tile * NQ * kSub + i * kSub + row;
+  const size_t per_sub = ws_floats_per_sub(D);
+  const float* base = ws + ((size_t)tile * kv_splits * NQ + i) * per_sub;
+  const size_t split_stride = (size_t)NQ * per_sub;
+
+  float m_max = -INFINITY;
+  for (int s = 0; s < kv_splits; ++s) m_max = fmaxf(m_max, base[s * split_stride + (size_t)kSub * D + row]);
+  float delta = 0.f;
+  for (int s = 0; s < kv_splits; ++s) {
+    const float* b = base + s * split_stride + (size_t)kSub * D;
+    delta += b[kSub + row] * exp2f(b[row] - m_max);
+  }
+  const float inv = 1.0f / delta;
+  if (grow >= L) return;
+  uint2* orow = reinterpret_cast<uint2*>(o + ((size_t)bh * L + grow) * D);
+  for (int g = 0; g < D / 4; ++g) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < kv_splits; ++s) {
+      const float* b = base + s * split_stride;
+      const float w = exp2f(b[(size_t)kSub * D + row] - m_max);
+      const float4 v = reinterpret_cast<const float4*>(b)[(size_t)g * kSub + row];
+      acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+    }
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    uint2 out;
+    out.x = *reinterpret_cast<uint32_t*>(&lo);
+    out.y = *reinterpret_cast<uint32_t*>(&hi);
+    orow[g] = out;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Non-pipelined kernel: one 128-row Q tile per CTA, 128 threads, one K/V stage,
+// every phase separated by a barrier.  dbg_flags bit 0 swaps the two byte
+// offsets of the V descriptor (layout diagnosis only).
+// ---------------------------------------------------------------------------
+struct SimpleMisc {
+  uint64_t load_bar;
+  uint64_t mma_bar;
+  uint64_t sync_bar;   // bounded replacement for a CTA-wide barrier inside the loop
+  uint32_t tmem_slot;
+  int abort_flag;
+};
+
+template <int D, int TKV>
+__global__ void __launch_bounds__(128, 1)
+attn_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                       const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, int L,
+                       float scale_log2, float* __restrict__ scores_out, int dbg_flags) {
+  constexpr int KCH = D / 64;
+  constexpr int TMEM_COLS = (TKV + D <= 128) ? 128 : 256;
+  constexpr int Q_BYTES = kSub * D * 2;
+  constexpr int KV_BYTES = TKV * D * 2;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = smem_u32(smem_raw);
+  const uint32_t q_smem = smem_base, k_smem = smem_base + Q_BYTES, v_smem = k_smem + KV_BYTES;
+  SimpleMisc* misc = reinterpret_cast<SimpleMisc*>(smem_raw + Q_BYTES + 2 * KV_BYTES);
+  volatile int* abort_flag = &misc->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = threadIdx.x;
+  const int q_row0 = blockIdx.x * kSub;
+  const int bh = blockIdx.y;
+  const int n = L / TKV;
+  const uint32_t bar_load = smem_u32(&misc->load_bar), bar_mma = smem_u32(&misc->mma_bar);
+  const uint32_t bar_sync = smem_u32(&misc->sync_bar);
+
+  if (threadIdx.x == 0) {
+    misc->abort_flag = (smem_base & 1023u) ? 1 : 0;
+    if (smem_base & 1023u) report_timeout(wait_info(kRoleSimple, 0, 0xFFFF));
+    mbar_init(bar_load, 1);
+    mbar_init(bar_mma, 1);
+    mbar_init(bar_sync, kSub);
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&misc->tmem_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = misc->tmem_slot;
+  const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+  const uint32_t s_tmem = lane_base, o_tmem = lane_base + TKV;
+  const uint32_t lbo = (dbg_flags & 1) ? 1024u : (uint32_t)(TKV * 128);
+  const uint32_t sbo = (dbg_flags & 1) ? (uint32_t)(TKV * 128) : 1024u;
+
+  float m_run = -INFINITY, delta = 0.f;
+  uint32_t ph_load = 0, ph_mma = 0;
+  bool ok = (*abort_flag == 0);
+  for (int j = 0; ok && j < n; ++j) {
+    if (threadIdx.x == 0) {
+      mbar_arrive_expect_tx(bar_load, (j == 0 ? Q_BYTES : 0) + 2 * KV_BYTES);
+      if (j == 0)
+        for (int c = 0; c < KCH; ++c) tma_load_3d(q_smem + c * (kSub * 128), &tm_q, c * 64, q_row0, bh, bar_load);
+      for (int c = 0; c < KCH; ++c) tma_load_3d(k_smem + c * (TKV * 128), &tm_k, c * 64, j * TKV, bh, bar_load);
+      for (int c = 0; c < KCH; ++c) tma_load_3d(v_smem + c * (TKV * 128), &tm_v, c * 64, j * TKV, bh, bar_load);
+    }
+    if (!wait_bar_warp(bar_load, ph_load, abort_flag, wait_info(kRoleSimple, kBarLoad, j))) { ok = false; break; }
+    ph_load ^= 1u;
+    if (threadIdx.x == 0) {
+      tc_fence_after();
+      issue_qk<D, TKV>(tmem_base, q_smem, k_smem);
+      umma_commit(bar_mma);
+    }
+    if (!wait_bar_warp(bar_mma, ph_mma, abort_flag, wait_info(kRoleSimple, kBarMma, 2 * j))) { ok = false; break; }
+    ph_mma ^= 1u;
+    tc_fence_after();
+
+    uint32_t s[TKV];
+#pragma unroll
+    for (int c = 0; c < TKV / 32; ++c) tmem_ld32(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+    if (scores_out != nullptr && j == 0 && blockIdx.x == 0 && blockIdx.y == 0) {
+      for (int k = 0; k < TKV; ++k) scores_out[(size_t)row * TKV + k] = __uint_as_float(s[k]);
+    }
+    float mx = __uint_as_float(s[0]);
+#pragma unroll
+    for (int k = 1; k < TKV; ++k) mx = fmaxf(mx, __uint_as_float(s[k]));
+    const float m_new = fmaxf(m_run, mx * scale_log2);
+    const float alpha = ex2_approx(m_run - m_new);
+    if (j > 0) {
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(o_tmem + c * 32, r);
+#pragma unroll
+        for (int k = 0; k < 32; ++k) r[k] = __float_as_uint(__uint_as_float(r[k]) * alpha);
+        tmem_st32(o_tmem + c * 32, r);
+      }
+    }
+    float sum = 0.f;
+#pragma unroll
+    for (int c = 0; c < TKV / 32; ++c) {
+      uint32_t pk[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const float e0 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + 2 * k]), scale_log2, -m_new));
+        const float e1 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + 2 * k + 1]), scale_log2, -m_new));
+        sum += e0 + e1;
+        pk[k] = pack_bf16x2(e0, e1);
+      }
+      tmem_st16(s_tmem + c * 16, pk);
+    }
+    delta = delta * alpha + sum;
+    m_run = m_new;
+    tmem_wait_st();
+    tc_fence_before();
+    mbar_arrive(bar_sync);
+    if (!wait_bar_warp(bar_sync, j & 1, abort_flag, wait_info(kRoleSimple, kBarSync, j))) { ok = false; break; }
+    if (threadIdx.x == 0) {
+      tc_fence_after();
+      issue_pv<D, TKV>(tmem_base + TKV, tmem_base, v_smem, j > 0, lbo, sbo);
+      umma_commit(bar_mma);
+    }
+    if (!wait_bar_warp(bar_mma, ph_mma, abort_flag, wait_info(kRoleSimple, kBarMma, 2 * j + 1))) { ok = false; break; }
+    ph_mma ^= 1u;
+    tc_fence_after();
+  }
+  if (ok) {
+    const float inv = 1.0f / delta;
+    const bool in_range = q_row0 + row < L;
+    uint4* orow = reinterpret_cast<uint4*>(o + ((size_t)bh * L + q_row0 + (in_range ? row : 0)) * D);
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld32(o_tmem + c * 32, r);          // warp-collective: every lane takes part
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        uint4 w;
+        w.x = pack_bf16x2(__uint_as_float(r[u * 8 + 0]) * inv, __uint_as_float(r[u * 8 + 1]) * inv);
+        w.y = pack_bf16x2(__uint_as_float(r[u * 8 + 2]) * inv, __uint_as_float(r[u * 8 + 3]) * inv);
+        w.z = pack_bf16x2(__uint_as_float(r[u * 8 + 4]) * inv, __uint_as_float(r[u * 8 + 5]) * inv);
+        w.w = pack_bf16x2(__uint_as_float(r[u * 8 + 6]) * inv, __uint_as_float(r[u * 8 + 7]) * inv);
+        if (in_range) orow[c * 4 + u] = w;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace attn

@@ -1,0 +1,201 @@
+// Closed-form tile derivation for fused attention (host only, no CUDA calls).
+//
+// The paper derives tiles from a hardware descriptor by applying capacity
+// constraints in a fixed order around the compute unit (Section "Tile
+// Derivation"): local memory fixes the staged tile, the register file fixes
+// the accumulator tile at the point between the two matrix products where
+// every intermediate is live, then the block count is checked against the
+// number of compute units and the result is aligned to the instruction atom.
+// Two machine models are covered:
+//   * accumulators in vector registers (the paper's CDNA targets; reproduces
+//     its Table 2), selected by acc_mem_columns == 0;
+//   * accumulators in tensor memory (B200): S/P and O live in tensor-memory
+//     columns, one S row lives in the registers of one softmax thread, K/V
+//     tiles live in a shared-memory ring.
+// No quantity is searched: each is a floor/ceil of descriptor fields.
+#include <cstdint>
+#include <cstring>
+
+#include "attn.h"
+
+namespace {
+
+// Role structure of the B200 kernel the register budget is derived for.
+constexpr int kRegsCorrection = 80;   // per thread: O-rescale / epilogue warpgroup
+constexpr int kRegsOther = 48;        // per thread: TMA and MMA-issue warps
+constexpr int kRegsRowOverhead = 32;  // softmax thread: row statistics, addresses, loop state
+constexpr int kSmemReserve = 3072;    // barriers, rescale factors, tensor-memory slot
+constexpr int kMaxStages = 8;
+constexpr int kMinStages = 4;         // K_j, V_j and one of each in flight
+constexpr int kMinTileKv = 32;
+constexpr int kMinStepsPerSplit = 4;
+
+inline int floor_to(int x, int m) { return (x / m) * m; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline int pow2_floor(int x) {
+  int p = 1;
+  if (x < 1) return 0;
+  while (p * 2 <= x) p *= 2;
+  return p;
+}
+inline int pow2_ceil(int x) {
+  int p = 1;
+  while (p < x) p *= 2;
+  return p;
+}
+
+// Registers per thread at the point between the two products on a register
+// machine: Q fragment (d), O accumulator (d), score tile (t_kv) and 8 row
+// statistics per Q row, spread over the wavefront, plus 16 of fixed overhead
+// (reproduces the four rows of the paper's Table 2).
+inline int register_machine_regs(int t_q, int t_kv, int d, int simd) {
+  return ceil_div(t_q * (2 * d + t_kv + 8), simd) + 16;
+}
+
+void plan_register_machine(const attn_hw_desc& h, int B, int H, int L, int d, attn_tiles* t) {
+  // Local memory holds K_t and V_t together.
+  const int t_kv = floor_to(h.local_mem_bytes / (2 * d * h.elem_bytes), h.atom_n);
+  const int t_q = (t_kv > 0)
+      ? floor_to(((h.max_regs_per_thread - 16) * h.simd_width) / (2 * d + t_kv + 8), h.atom_m)
+      : 0;
+  t->binding_constraint = ATTN_BIND_REG;
+  if (t_kv < h.atom_n) { t->binding_constraint = ATTN_BIND_SMEM; return; }
+  if (t_q < h.atom_m) return;
+  t->feasible = 1;
+  t->tile_q = t_q;
+  t->tile_kv = t_kv;
+  t->n_q = 1;
+  t->n_s = 1;
+  t->kv_stages = 1;
+  t->kv_splits = 1;
+  t->smem_bytes = 2 * t_kv * d * h.elem_bytes;
+  t->tmem_columns = 0;
+  t->regs_softmax = register_machine_regs(t_q, t_kv, d, h.simd_width);
+  t->threads = h.simd_width;
+  t->tiles = B * H * ceil_div(L, t_q);
+  t->ctas = t->tiles;
+  t->ctas_per_unit = (float)t->ctas / (float)h.num_units;
+  const int waves = ceil_div(t->ctas, h.num_units);
+  t->wave_efficiency = (float)((double)t->ctas / ((double)waves * h.num_units));
+  t->under_occupied = t->tiles < h.num_units;
+}
+
+void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, attn_tiles* t) {
+  const int sub = h.atom_m;  // one tensor-memory lane per Q row
+  t->binding_constraint = ATTN_BIND_SHAPE;
+  if (d % h.atom_k || d % h.atom_n || d > h.atom_n_max) return;
+
+  // 1. Sub-tiles per CTA, registers and tensor memory => tile_KV.
+  int n_q = (L > sub) ? 2 : 1;
+  int tile_kv = 0, regs_soft = 0, binding = ATTN_BIND_NONE;
+  for (;;) {
+    regs_soft = floor_to((h.regs_per_unit - 128 * kRegsCorrection - 128 * kRegsOther) / (128 * n_q), 8);
+    const int cap = floor_to(h.max_regs_per_thread, 8);
+    if (regs_soft > cap) regs_soft = cap;
+    const int c_reg = ((regs_soft - kRegsRowOverhead) * 4) / 5;  // S row + a quarter row of packed P
+    const int c_tmem = h.acc_mem_columns / n_q - d;              // S tile + O accumulator per sub-tile
+    const int c_atom = h.atom_n_max;
+    int c = c_reg < c_tmem ? c_reg : c_tmem;
+    if (c_atom < c) c = c_atom;
+    binding = (c == c_tmem) ? ATTN_BIND_TMEM : (c == c_reg ? ATTN_BIND_REG : ATTN_BIND_ATOM);
+    tile_kv = pow2_floor(c);
+    if (tile_kv >= kMinTileKv || n_q == 1) break;
+    n_q = 1;
+  }
+  t->binding_constraint = binding;
+  if (tile_kv < kMinTileKv) return;
+
+  // 2. Shared memory => depth of the K/V ring (Q tile resident, O staged in its place).
+  const int q_bytes = n_q * sub * d * h.elem_bytes;
+  int stage = 0, stages = 0;
+  for (;;) {
+    stage = tile_kv * d * h.elem_bytes;
+    stages = (h.local_mem_bytes - q_bytes - kSmemReserve) / stage;
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages >= kMinStages) break;
+    tile_kv /= 2;
+    binding = ATTN_BIND_SMEM;
+    if (tile_kv < kMinTileKv) { t->binding_constraint = ATTN_BIND_SMEM; return; }
+  }
+
+  // 3. Occupancy: blocks against compute units; split the key axis when short.
+  const int tile_q = n_q * sub;
+  const int tiles = B * H * ceil_div(L, tile_q);
+  const int steps = ceil_div(L, tile_kv);
+  const int under = tiles < h.num_units;
+  int kv_splits = 1;
+  if (under) {
+    int by_units = h.num_units / tiles;
+    int by_steps = steps / kMinStepsPerSplit;
+    kv_splits = by_units < by_steps ? by_units : by_steps;
+    if (kv_splits < 1) kv_splits = 1;
+  }
+
+  t->feasible = 1;
+  t->binding_constraint = binding;
+  t->tile_q = tile_q;
+  t->tile_kv = tile_kv;
+  t->n_q = n_q;
+  t->n_s = 1;
+  t->kv_stages = stages;
+  t->kv_splits = kv_splits;
+  t->smem_bytes = q_bytes + stages * stage + kSmemReserve;
+  t->tmem_columns = pow2_ceil(n_q * (tile_kv + d));
+  if (t->tmem_columns < 32) t->tmem_columns = 32;
+  t->regs_softmax = regs_soft;
+  t->threads = 128 * (n_q + 2);
+  t->tiles = tiles;
+  t->ctas = tiles * kv_splits;
+  t->ctas_per_unit = (float)t->ctas / (float)h.num_units;
+  const int waves = ceil_div(t->ctas, h.num_units);
+  t->wave_efficiency = (float)((double)t->ctas / ((double)waves * h.num_units));
+  t->under_occupied = under;
+}
+
+}  // namespace
+
+extern "C" int attn_hw_desc_b200(attn_hw_desc* out) {
+  if (!out) return ATTN_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  out->struct_bytes = (int32_t)sizeof(attn_hw_desc);
+  out->num_units = 148;
+  out->local_mem_bytes = 232448;  // 227 KB opt-in dynamic shared memory per block
+  out->regs_per_unit = 65536;
+  out->max_regs_per_thread = 255;
+  out->simd_width = 32;
+  out->acc_mem_lanes = 128;
+  out->acc_mem_columns = 512;
+  out->atom_m = 128;  // tcgen05.mma kind::f16, cta_group::1
+  out->atom_n = 16;
+  out->atom_k = 16;
+  out->atom_n_max = 256;
+  out->elem_bytes = 2;
+  out->hbm_gbps = 7700.0;
+  out->peak_tflops = 2250.0;
+  out->sm_clock_mhz = 1965.0;
+  return ATTN_OK;
+}
+
+extern "C" int attn_plan(const attn_hw_desc* desc, int B, int H, int L, int d, attn_tiles* out) {
+  if (!desc || !out) return ATTN_ERR_INVALID_ARG;
+  if (desc->struct_bytes != (int32_t)sizeof(attn_hw_desc)) return ATTN_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  out->binding_constraint = ATTN_BIND_SHAPE;
+  if (B <= 0 || H <= 0 || L <= 0 || d <= 0) return ATTN_OK;
+  if (desc->num_units <= 0 || desc->local_mem_bytes <= 0 || desc->atom_m <= 0 || desc->atom_n <= 0 ||
+      desc->atom_k <= 0 || desc->elem_bytes <= 0 || desc->simd_width <= 0 || desc->max_regs_per_thread <= 16)
+    return ATTN_ERR_INVALID_ARG;
+  if (desc->acc_mem_columns > 0)
+    plan_tmem_machine(*desc, B, H, L, d, out);
+  else
+    plan_register_machine(*desc, B, H, L, d, out);
+  return ATTN_OK;
+}
+
+extern "C" size_t attn_workspace_bytes(const attn_tiles* t, int B, int H, int L, int d) {
+  (void)B; (void)H; (void)L;
+  if (!t || !t->feasible || t->kv_splits <= 1 || t->n_q <= 0) return 0;
+  // Per CTA and sub-tile: 128 x d fp32 un-normalised output + 128 (m, delta) pairs.
+  const size_t per_sub = (size_t)128 * (size_t)d * 4 + (size_t)128 * 2 * 4;
+  return (size_t)t->ctas * (size_t)t->n_q * per_sub;
+}

@@ -1,0 +1,152 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every declared symbol,
+its planner equals the oracle-side restatement, and argument errors are reported
+before any CUDA call.  No kernel is launched here."""
+import ctypes
+import itertools
+import os
+import re
+
+import pytest
+
+from oracle import plan_oracle as po
+from tests.conftest import ROOT, read_golden
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2609_10937_b200 import binding as b
+    from paper_2609_10937_b200 import build
+
+    build.build()
+    b.lib()
+    return b
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "attn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(attn_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(binding):
+    names = _declared_functions()
+    assert len(names) >= 12
+    L = binding.lib()
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in include/attn.h but not exported"
+    assert set(names) == set(binding.EXPORTED_SYMBOLS)
+
+
+def test_struct_sizes_match_the_header(binding):
+    d = binding.hw_desc_b200()
+    assert d.struct_bytes == ctypes.sizeof(binding.AttnHwDesc) == 80
+    assert ctypes.sizeof(binding.AttnTiles) == 72
+
+
+def _desc_dict(d):
+    return {n: getattr(d, n) for n, _ in d._fields_}
+
+
+def test_b200_plan_equals_oracle_restatement(binding):
+    desc = binding.hw_desc_b200()
+    dd = _desc_dict(desc)
+    shapes = itertools.product([1, 4], [1, 8, 32], [128, 256, 1024, 2048, 4096, 16384, 32768], [64, 128, 256, 72])
+    for B, H, L, d in shapes:
+        got = binding.plan(desc, B, H, L, d)
+        ref = po.derive_tiles_tmem_machine(dd, B, H, L, d)
+        assert bool(got.feasible) == ref["feasible"], (B, H, L, d)
+        assert got.binding_constraint == ref["binding"]
+        if not ref["feasible"]:
+            continue
+        for key in ("tile_q", "tile_kv", "n_q", "n_s", "kv_stages", "kv_splits", "smem_bytes", "tmem_columns",
+                    "regs_softmax", "threads", "tiles", "ctas"):
+            assert getattr(got, key) == ref[key], (key, B, H, L, d)
+        assert bool(got.under_occupied) == ref["under_occupied"]
+        assert got.wave_efficiency == pytest.approx(ref["wave_efficiency"], rel=1e-6)
+        assert got.ctas_per_unit == pytest.approx(ref["ctas_per_unit"], rel=1e-6)
+
+
+def test_other_descriptors_rerun_the_same_derivation(binding):
+    """Changing the descriptor re-runs the derivation with no code change (the paper's portability claim)."""
+    desc = binding.hw_desc_b200()
+    for field, value in (("local_mem_bytes", 101376), ("num_units", 74), ("acc_mem_columns", 256),
+                         ("regs_per_unit", 32768)):
+        setattr(desc, field, value)
+        for B, H, L, d in [(1, 1, 16384, 128), (4, 32, 4096, 64), (1, 8, 2048, 128)]:
+            got = binding.plan(desc, B, H, L, d)
+            ref = po.derive_tiles_tmem_machine(_desc_dict(desc), B, H, L, d)
+            assert bool(got.feasible) == ref["feasible"]
+            if ref["feasible"]:
+                assert (got.tile_q, got.tile_kv, got.kv_stages, got.kv_splits, got.smem_bytes) == (
+                    ref["tile_q"], ref["tile_kv"], ref["kv_stages"], ref["kv_splits"], ref["smem_bytes"])
+                assert got.smem_bytes <= desc.local_mem_bytes
+            assert got.binding_constraint == ref["binding"]
+
+
+def _cdna_desc(binding, num_cus):
+    d = binding.AttnHwDesc()
+    d.struct_bytes = ctypes.sizeof(binding.AttnHwDesc)
+    d.num_units, d.local_mem_bytes, d.max_regs_per_thread, d.simd_width = num_cus, 64 * 1024, 256, 64
+    d.atom_m, d.atom_n, d.atom_k, d.atom_n_max, d.elem_bytes = 16, 16, 4, 16, 4
+    return d
+
+
+def test_register_machine_plan_reproduces_the_paper_table(binding):
+    """The C planner fed the paper's CDNA descriptor returns the tiles of its Table 2."""
+    for d, t_kv, t_q, regs, feasible in ([int(x) for x in r] for r in read_golden("paper_table2_tiles.txt")):
+        if not feasible:
+            continue
+        got = binding.plan(_cdna_desc(binding, 120), 1, 1, 16384, d)
+        assert (got.feasible, got.tile_kv, got.tile_q, got.regs_softmax) == (1, t_kv, t_q, regs)
+        assert got.binding_constraint == po.BIND_REG
+    for num_cus, t_q, t_kv, _ in read_golden("paper_derive_tiles_listing.txt"):
+        got = binding.plan(_cdna_desc(binding, int(num_cus)), 1, 1, 16384, 128)
+        assert (got.tile_q, got.tile_kv, got.tiles) == (int(t_q), int(t_kv), 512)
+
+
+def test_plan_argument_errors(binding):
+    desc = binding.hw_desc_b200()
+    t = binding.AttnTiles()
+    L = binding.lib()
+    assert L.attn_plan(None, 1, 1, 128, 64, ctypes.byref(t)) == binding.ERR_INVALID_ARG
+    desc.struct_bytes = 12
+    assert L.attn_plan(ctypes.byref(desc), 1, 1, 128, 64, ctypes.byref(t)) == binding.ERR_INVALID_ARG
+    desc = binding.hw_desc_b200()
+    assert L.attn_plan(ctypes.byref(desc), 1, 1, 0, 64, ctypes.byref(t)) == 0 and t.feasible == 0
+    assert t.binding_constraint == po.BIND_SHAPE
+
+
+def test_workspace_bytes(binding):
+    desc = binding.hw_desc_b200()
+    t = binding.plan(desc, 1, 1, 16384, 128)
+    assert t.kv_splits == 2
+    assert binding.workspace_bytes(t, 1, 1, 16384, 128) == t.ctas * 2 * (128 * 128 + 256) * 4
+    t1 = binding.plan(desc, 4, 32, 4096, 128)
+    assert binding.workspace_bytes(t1, 4, 32, 4096, 128) == 0
+
+
+def test_forward_argument_errors_come_before_any_cuda_call(binding):
+    L = binding.lib()
+    p = ctypes.c_void_p
+    a, b, c, o = 0x10000, 0x20000000, 0x40000000, 0x60000000    # never dereferenced: checks fail first
+    assert L.attn_forward(None, p(b), p(c), p(o), 1, 1, 128, 64, None) == binding.ERR_INVALID_ARG
+    assert L.attn_forward(p(a), p(b), p(c), p(o), 0, 1, 128, 64, None) == binding.ERR_INVALID_ARG
+    assert L.attn_forward(p(a), p(b), p(c), p(o), 1, 1, 128, 96, None) == binding.ERR_UNSUPPORTED_SHAPE
+    assert L.attn_forward(p(a), p(b), p(c), p(o), 1, 1, 100, 64, None) == binding.ERR_UNSUPPORTED_SHAPE
+    assert L.attn_forward(p(a + 8), p(b), p(c), p(o), 1, 1, 128, 64, None) == binding.ERR_MISALIGNED
+    assert L.attn_forward(p(a), p(b), p(c), p(a + 1024), 1, 1, 128, 64, None) == binding.ERR_ALIASING
+    assert L.attn_forward_simple(p(a), p(b), p(c), p(b), 1, 1, 128, 64, 128, None, None) == binding.ERR_ALIASING
+    assert L.attn_forward_host(p(a), p(b), p(c), p(o), 1, 1, 128, 64, p(0x7000000), 16, None) == binding.ERR_INVALID_ARG
+    assert "aligned" in binding.status_string(binding.ERR_MISALIGNED)
+    assert binding.status_string(12345) == "unknown status"
+
+
+def test_product_does_not_reach_the_oracle():
+    """The product package must not import, read or execute anything under oracle/."""
+    pkg = os.path.join(ROOT, "paper_2609_10937_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".cpp", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                for pat in (r"import\s+oracle", r"from\s+oracle", r"oracle[/\\.]", r"attn_oracle", r"plan_oracle"):
+                    assert not re.search(pat, text), f"{f} reaches into oracle/ ({pat})"
