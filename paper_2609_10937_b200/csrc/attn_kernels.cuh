@@ -26,7 +26,7 @@ namespace attn {
 using namespace sm100;
 
 constexpr int kSub = 128;                 // rows of one Q sub-tile = tensor-memory lanes
-constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz
+constexpr long long kWaitLimitCycles = 1000000000LL;  // ~0.5 s at 1.9 GHz
 
 // [0] error code (0 = none), [1] role<<24 | barrier<<16 | step, [2] CTA index, [3] spare
 __device__ unsigned int g_attn_dev_status[4];
