@@ -1,0 +1,304 @@
+#!/usr/bin/env python
+"""Benchmark of the fused-attention forward pass (one JSON line on stdout).
+
+Metric: attention TFLOP/s = 4*B*H*L^2*d / time at the paper's headline shape
+B=1, H=1, L=16384, d=128 (bf16 in/out, fp32 accumulate, non-causal), with the
+closed-form default tiles.  A "step" is one whole forward pass (main kernel and,
+when the plan splits the key axis, the merge kernel) over one synthetic batch.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 (under torchrun): every rank runs its own copy of the workload (weak
+scaling, independent problems, no data-path collective); value is the total
+work of all ranks over the slowest rank's time.
+
+--impl reference times the fp64 CPU oracle on the host cores on a bounded row
+sample of the same workload (rank 0 only).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+WORKLOAD = "cfg3"
+METRIC = "fused_attention_fwd_tflops_L16384_d128"
+UNIT = "TFLOP/s"
+L2_FLUSH_BYTES = 256 << 20
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"bf16_tflops": float(p["bf16_tflops"]), "bf16_tflops_sustained": float(p["bf16_tflops_sustained"]),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.lines = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        chosen = [l for t, l in self.lines if t0 - 0.05 <= t <= t1 + 0.1] or [l for _, l in self.lines]
+        for line in chosen:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def cpu_baseline(case, q, k, v, target_seconds=12.0):
+    """The fp64 oracle, as it stands, on the host cores, on a bounded row sample."""
+    from oracle import attn_oracle as orc
+
+    cores = orc.threads()
+    probe = np.arange(0, case.L, max(1, case.L // 256), dtype=np.int32)[:256]
+    t0 = time.perf_counter()
+    orc.attention_rows(q, k, v, case.B, case.H, case.L, case.d, probe)
+    dt = max(time.perf_counter() - t0, 1e-6)
+    n_rows = int(min(case.L, max(256, len(probe) * target_seconds / dt)))
+    rows = np.unique(np.linspace(0, case.L - 1, n_rows).astype(np.int32))
+    t0 = time.perf_counter()
+    orc.attention_rows(q, k, v, case.B, case.H, case.L, case.d, rows)
+    dt = time.perf_counter() - t0
+    flops = 4.0 * case.B * case.H * len(rows) * case.L * case.d
+    return {"value": flops / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{len(rows)} of {case.L} query rows per head, all keys, fp64, {dt:.2f} s",
+            "seconds": dt}
+
+
+def run_reference(args):
+    """Reference arm: the fp64 CPU oracle on the host cores (rank 0 only)."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return 0
+    from oracle import attn_oracle as orc
+    from paper_2609_10937_b200 import synth
+
+    case = synth.CONFIGS[WORKLOAD]
+    q, k, v = synth.make_qkv(case, seed=0)
+    cores = orc.threads()
+    rows = np.unique(np.linspace(0, case.L - 1, 2048).astype(np.int32))   # bounded sample per step
+    flops = 4.0 * case.B * case.H * len(rows) * case.L * case.d
+    for _ in range(args.warmup):
+        orc.attention_rows(q, k, v, case.B, case.H, case.L, case.d, rows[:256])
+    times = []
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        orc.attention_rows(q, k, v, case.B, case.H, case.L, case.d, rows)
+        times.append(time.perf_counter() - t0)
+    ms = 1e3 * sum(times) / len(times)
+    value = flops / (ms * 1e-3) / 1e12
+    sample = f"{len(rows)} of {case.L} query rows per head per step, all keys, fp64 (extrapolates linearly in rows)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "cfg3: attention fwd B=1,H=1,L=16384,d=128, non-causal, bf16 inputs N(0,1), seed 0"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def run_ours(args):
+    import torch
+
+    from paper_2609_10937_b200 import binding, synth, traffic
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    binding.lib()
+    case = synth.CONFIGS[WORKLOAD]
+    q, k, v = synth.make_qkv(case, seed=rank)       # every rank its own problem of the same shape
+    as_t = lambda b: torch.from_numpy(b.view(np.int16)).view(torch.bfloat16)
+    hq, hk, hv = (as_t(x).pin_memory() for x in (q, k, v))
+    ho = torch.empty_like(hq).pin_memory()
+    dq, dk, dv = (x.cuda(non_blocking=True) for x in (hq, hk, hv))
+    do = torch.empty_like(dq)
+    scratch = torch.empty(4 * dq.numel() * 2, dtype=torch.uint8, device="cuda")
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    plan = binding.plan(binding.hw_desc_query(local), case.B, case.H, case.L, case.d)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            flush.fill_(1)
+            fn()
+        barrier()
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        t0 = time.time()
+        for i in range(steps):
+            flush.fill_(i & 0xFF)                  # L2 flush between timed steps, outside the step's events
+            starts[i].record(stream)
+            fn()
+            ends[i].record(stream)
+        barrier()
+        t1 = time.time()
+        per = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+        ms = sum(per) / len(per)
+        if dist is not None:
+            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, per, t0, t1
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.15)
+    ms, per, t0, t1 = timed(lambda: binding.forward(dq, dk, dv, do), args.steps, args.warmup)
+    launches_per_step = binding.last_launch_count()
+    clocks = sampler.stop(t0, t1) if sampler else None
+    code, detail = binding.last_device_status()
+    if code != 0:
+        raise RuntimeError(f"device-side wait expired: {detail}")
+    e2e_steps = max(3, min(args.steps, 10))
+    e2e_ms, _, _, _ = timed(lambda: binding.forward_host(hq, hk, hv, ho, scratch), e2e_steps, 3)
+
+    flops = case.flops
+    value = world * flops / (ms * 1e-3) / 1e12
+    e2e_value = world * flops / (e2e_ms * 1e-3) / 1e12
+    nbytes = dq.numel() * 2
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    peaks = load_peaks()
+    achieved = flops / (ms * 1e-3) / 1e12
+    traffic_note = traffic.measured_dram_bytes_per_launch(ROOT)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {
+            "workload": "cfg3: attention fwd B=1,H=1,L=16384,d=128, non-causal, bf16 N(0,1), scale 1/sqrt(d), "
+                        "fp32 accumulate (one such problem per GPU)",
+            "tiles": {"tile_q": plan.tile_q, "tile_kv": plan.tile_kv, "kv_stages": plan.kv_stages,
+                      "kv_splits": plan.kv_splits, "ctas": plan.ctas, "closed_form_default": True},
+            "l2": f"{L2_FLUSH_BYTES >> 20} MiB device write between timed steps (outside the step's events)",
+            "timing": "CUDA events on the launching stream around every step; mean of per-step times; max over ranks",
+            "ms_per_step_min": min(per), "ms_per_step_max": max(per),
+        },
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes,
+                "ms_per_step": e2e_ms, "steps": e2e_steps,
+                "path": "attn_forward_host: pinned host q,k,v -> device, forward, o -> pinned host, all in the timed region"},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {
+            "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": UNIT,
+            "frac": achieved / peaks["bf16_tflops"], "traffic": traffic_note,
+            "peak_source": f"{peaks['source']} cuBLAS bf16 burst (kernel timed alone)",
+            "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+            "frac_of_nominal_2250": achieved / 2250.0,
+            "kernel": "attn_fwd_kernel<128,128,2> (+ attn_merge_kernel when kv_splits > 1; whole step timed)",
+            "algorithmic_flops_per_launch": flops,
+            "unfused_traffic_bytes_bf16_scores": traffic.unfused_bytes(case.B, case.H, case.L, case.d, 2, 2),
+            "compulsory_traffic_bytes": traffic.fused_bytes(case.B, case.H, case.L, case.d, 2),
+        },
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = {k_: v_ for k_, v_ in cpu_baseline(case, q, k, v).items() if k_ != "seconds"}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        if args.steps > 10:
+            args.steps = 10
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -150,3 +150,17 @@ def test_product_does_not_reach_the_oracle():
                 text = open(os.path.join(dirpath, f)).read()
                 for pat in (r"import\s+oracle", r"from\s+oracle", r"oracle[/\\.]", r"attn_oracle", r"plan_oracle"):
                     assert not re.search(pat, text), f"{f} reaches into oracle/ ({pat})"
+
+
+def test_traffic_model_matches_the_paper_figures():
+    """The product-side traffic calculator against the figures the paper prints."""
+    from paper_2609_10937_b200 import traffic
+
+    g = {row[0]: (int(row[1]), float(row[2])) for row in read_golden("paper_hbm_traffic.txt")}
+    L = g["fused_mb"][0]
+    assert round(traffic.fused_bytes(1, 1, L, 128, 4) / 1e6) == g["fused_mb"][1]
+    assert round(traffic.unfused_bytes(1, 1, L, 128, 4, 4) / 1e6) == g["unfused_mb"][1]
+    assert round(traffic.unfused_bytes(1, 1, L, 128, 4, 4) / traffic.fused_bytes(1, 1, L, 128, 4)) == g["ratio"][1]
+    assert round(traffic.unfused_bytes(1, 1, g["unfused_gb"][0], 128, 4, 4) / 1e9) == g["unfused_gb"][1]
+    assert traffic.savings(L, 128) == g["savings"][1]
+    assert traffic.unfused_bytes(1, 1, L, 128, 4, 4) == po.traffic_unfused(1, 1, L, 128, 4, 4)
