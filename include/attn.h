@@ -126,13 +126,15 @@ int attn_hw_desc_query(int device, attn_hw_desc *out);
 int attn_plan(const attn_hw_desc *desc, int B, int H, int L, int d, attn_tiles *out);
 
 /* Bytes of workspace attn_forward* needs for this plan: 0 unless kv_splits > 1
- * (partial outputs and row statistics of the merge operator, Section "Online
- * Softmax"). */
+ * (64 KB of arrival counters, then the partial outputs and row statistics of
+ * the merge operator, Section "Online Softmax"). */
 size_t attn_workspace_bytes(const attn_tiles *tiles, int B, int H, int L, int d);
 
 /* Registers a caller-owned device buffer as the workspace of `device` (pass
- * NULL, 0 to clear).  The buffer must stay valid until replaced; concurrent
- * attn_forward calls on different streams of one device must not share it. */
+ * NULL, 0 to clear) and zeroes its first 64 KB (the arrival counters) with a
+ * synchronous cudaMemset on the current device, which must be `device`.  The
+ * buffer must stay valid until replaced; concurrent attn_forward calls on
+ * different streams of one device must not share it. */
 int attn_set_workspace(int device, void *dev_ptr, size_t bytes);
 
 /*
@@ -185,7 +187,7 @@ int attn_forward_host(const void *q_host, const void *k_host, const void *v_host
  * a spare word -- or ATTN_OK.  Clears the record. */
 int attn_last_device_status(void *cuda_stream, uint32_t *detail);
 
-/* Number of kernels the last attn_forward* call launched (1, or 2 with merge). */
+/* Number of kernels the last attn_forward* call on this thread launched. */
 int attn_last_launch_count(void);
 
 /* Static description of a status code; never NULL. */

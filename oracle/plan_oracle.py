@@ -55,8 +55,8 @@ def derive_tiles_register_machine(lds_bytes, regs_per_thread, wavefront, num_uni
 
 
 # Role structure of the B200 kernel that the derivation budgets for.
-_REGS_CORRECTION = 80      # per thread, correction/epilogue warpgroup
-_REGS_OTHER = 48           # per thread, TMA / MMA-issue warps
+_REGS_CORRECTION = 64      # per thread, correction warpgroup
+_REGS_OTHER = 64           # per thread, TMA / MMA-issue warpgroup
 _REGS_ROW_OVERHEAD = 32    # softmax thread: addresses, row statistics, loop state
 _SMEM_RESERVE = 3072       # barriers, rescale factors, tensor-memory slot
 _MAX_STAGES = 8

@@ -129,7 +129,10 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   p.kv_splits = t.kv_splits;
   p.stages = t.kv_stages;
   p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
-  p.ws = ws;
+  p.counters = reinterpret_cast<unsigned int*>(ws);                   // head of the workspace
+  p.ws = ws ? ws + attn::kCounterBytes / sizeof(float) : nullptr;    // partial results follow
+  if (t.kv_splits > 1 && (size_t)BH * p.q_tiles * NQ > attn::kCounterBytes / sizeof(unsigned int))
+    return ATTN_ERR_BAD_TILES;
   const int smem = SM::total(t.kv_stages);
   auto kern = attn::attn_fwd_kernel<D, TKV, NQ>;
   ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -137,12 +140,6 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
   ATTN_CUDA_TRY(cudaGetLastError());
   t_launch_count = 1;
-  if (t.kv_splits > 1) {
-    attn::attn_merge_kernel<D, NQ><<<BH * p.q_tiles * NQ, 128, 0, stream>>>(
-        ws, reinterpret_cast<__nv_bfloat16*>(o), L, p.q_tiles, t.kv_splits);
-    ATTN_CUDA_TRY(cudaGetLastError());
-    t_launch_count = 2;
-  }
   return ATTN_OK;
 }
 
@@ -246,6 +243,10 @@ extern "C" int attn_hw_desc_query(int device, attn_hw_desc* out) {
 extern "C" int attn_set_workspace(int device, void* dev_ptr, size_t bytes) {
   if (device < 0 || device >= kMaxDevices) return ATTN_ERR_INVALID_ARG;
   if (dev_ptr && ((uintptr_t)dev_ptr & 15u)) return ATTN_ERR_MISALIGNED;
+  if (dev_ptr && bytes >= (size_t)attn::kCounterBytes) {
+    // arrival counters at the head of the workspace start at zero; kernels leave them at zero
+    ATTN_CUDA_TRY(cudaMemset(dev_ptr, 0, attn::kCounterBytes));
+  }
   std::lock_guard<std::mutex> lk(g_mu);
   g_dev[device].ws = dev_ptr;
   g_dev[device].ws_bytes = dev_ptr ? bytes : 0;
@@ -307,8 +308,25 @@ extern "C" int attn_last_device_status(void* cuda_stream, uint32_t* detail) {
   if (h[0] == 0) return ATTN_OK;
   unsigned int z[4] = {0, 0, 0, 0};
   ATTN_CUDA_TRY(cudaMemcpyToSymbol(attn::g_attn_dev_status, z, sizeof z));
+  {
+    // an aborted launch may have left arrival counters non-zero
+    int dev = 0;
+    ATTN_CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (dev >= 0 && dev < kMaxDevices && g_dev[dev].ws && g_dev[dev].ws_bytes >= (size_t)attn::kCounterBytes)
+      ATTN_CUDA_TRY(cudaMemset(g_dev[dev].ws, 0, attn::kCounterBytes));
+  }
   return ATTN_ERR_DEVICE_TIMEOUT;
 }
+
+#ifdef ATTN_TRACE
+// Debug builds only: copies the timeline of CTA 0 (5 roles x 16 steps x 8 events, clock64 values).
+extern "C" int attn_debug_read_trace(long long* out) {
+  ATTN_CUDA_TRY(cudaDeviceSynchronize());
+  ATTN_CUDA_TRY(cudaMemcpyFromSymbol(out, attn::g_attn_trace, sizeof(long long) * 5 * 16 * 8));
+  return ATTN_OK;
+}
+#endif
 
 extern "C" int attn_last_launch_count(void) { return t_launch_count; }
 

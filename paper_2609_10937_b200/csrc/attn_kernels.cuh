@@ -10,8 +10,9 @@
 //                          memory -> second tcgen05.mma (O += P V, A operand
 //                          read from tensor memory) ; a correction warpgroup
 //                          rescales O when the running maximum moved.
-//   attn_merge_kernel      merge operator of the online softmax over the
-//                          partial results of CTAs that split the key axis.
+//                          When CTAs split the key axis, each writes its partial
+//                          (O, m, delta) and the last one to finish merges them
+//                          with the merge operator of the online softmax.
 //   attn_fwd_simple_kernel the same algorithm with nothing overlapped; used to
 //                          cross-check the pipelined kernel and the layouts.
 //
@@ -34,6 +35,21 @@ __device__ unsigned int g_attn_dev_status[4];
 enum Role : uint32_t { kRoleLoad = 1, kRoleMma = 2, kRoleSoftmax = 3, kRoleCorrection = 4, kRoleSimple = 5 };
 enum BarId : uint32_t { kBarQ = 1, kBarKvFull = 2, kBarKvEmpty = 3, kBarSFull = 4, kBarPFull = 5, kBarOFull = 6,
                         kBarAlpha = 7, kBarLoad = 8, kBarMma = 9, kBarSync = 10 };
+
+// Optional timeline instrumentation (debug builds only, -DATTN_TRACE): CTA 0 records clock64()
+// at fixed points of each role for KV steps [kTraceStep0, kTraceStep0 + 16).
+#ifdef ATTN_TRACE
+constexpr int kTraceStep0 = 8;
+__device__ long long g_attn_trace[5][16][8];
+#define ATTN_TRACE_EVENT(role_slot, step, ev)                                                   \
+  do {                                                                                          \
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (step) >= kTraceStep0 && (step) < kTraceStep0 + 16) \
+      g_attn_trace[role_slot][(step) - kTraceStep0][ev] = clock64();                            \
+  } while (0)
+#else
+constexpr int kTraceStep0 = 0;
+#define ATTN_TRACE_EVENT(role_slot, step, ev) do {} while (0)
+#endif
 
 __device__ __noinline__ void report_timeout(uint32_t info) {
   if (atomicCAS(&g_attn_dev_status[0], 0u, 1u) == 0u) {
@@ -74,37 +90,59 @@ __device__ __forceinline__ uint32_t wait_info(uint32_t role, uint32_t bar, uint3
 // holds head-dimension columns [64c, 64c+64).  V tile: same storage, used as
 // the MN-major B operand of the second product (N = head dimension).
 // ---------------------------------------------------------------------------
+// Descriptor words are split so that the issuing thread only adds a constant to the low
+// word per k-step: low = (address >> 4) | (LBO >> 4) << 16, high = (SBO >> 4) | version | swizzle.
+__device__ __forceinline__ uint64_t desc_from_words(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+__host__ __device__ constexpr uint32_t desc_hi_sw128(uint32_t sbo_bytes) {
+  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
+}
+__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+  return ((smem_addr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+
 template <int D, int TKV>
 __device__ __forceinline__ void issue_qk(uint32_t s_tmem, uint32_t q_smem, uint32_t k_smem) {
   constexpr uint32_t idesc = make_idesc_bf16(kSub, TKV, false);
+  constexpr uint32_t hi = desc_hi_sw128(1024);
+  const uint32_t a_lo = desc_lo(q_smem, 16), b_lo = desc_lo(k_smem, 16);
 #pragma unroll
   for (int ks = 0; ks < D / 16; ++ks) {
     const uint32_t chunk = ks >> 2, kin = ks & 3;
-    const uint64_t a = make_smem_desc_sw128(q_smem + chunk * (kSub * 128) + kin * 32, 16, 1024);
-    const uint64_t b = make_smem_desc_sw128(k_smem + chunk * (TKV * 128) + kin * 32, 16, 1024);
-    umma_ss(s_tmem, a, b, idesc, ks > 0 ? 1u : 0u);
+    const uint64_t a = desc_from_words(a_lo + ((chunk * (kSub * 128) + kin * 32) >> 4), hi);
+    const uint64_t b = desc_from_words(b_lo + ((chunk * (TKV * 128) + kin * 32) >> 4), hi);
+    if (ks == 0) umma_ss_c<0>(s_tmem, a, b, idesc);
+    else umma_ss_c<1>(s_tmem, a, b, idesc);
   }
 }
 template <int D, int TKV>
 __device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_smem, bool accumulate,
-                                         uint32_t lbo, uint32_t sbo) {
+                                         uint32_t lbo, uint32_t sbo, int ks_begin = 0, int ks_end = TKV / 16) {
   constexpr uint32_t idesc = make_idesc_bf16(kSub, D, true);
+  const uint32_t hi = ((sbo >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
+  const uint32_t b_lo = desc_lo(v_smem, lbo);
 #pragma unroll
   for (int ks = 0; ks < TKV / 16; ++ks) {
+    if (ks < ks_begin || ks >= ks_end) continue;
     // 16 key rows per step: two 8-row groups of 1024 bytes
-    const uint64_t b = make_smem_desc_sw128(v_smem + ks * 2048, lbo, sbo);
-    umma_ts(o_tmem, p_tmem + ks * 8, b, idesc, (accumulate || ks > 0) ? 1u : 0u);
+    const uint64_t b = desc_from_words(b_lo + ((ks * 2048) >> 4), hi);
+    if (ks == 0) umma_ts(o_tmem, p_tmem + ks * 8, b, idesc, accumulate ? 1u : 0u);
+    else umma_ts_c<1>(o_tmem, p_tmem + ks * 8, b, idesc);
   }
 }
 
 struct FwdParams {
-  int L;             // sequence length
-  int q_tiles;       // Q tiles per head = ceil(L / (NQ*128))
-  int n_steps;       // KV steps per head = L / TKV
-  int kv_splits;     // CTAs per Q tile along the key axis
-  int stages;        // ring depth
-  float scale_log2;  // log2(e) / sqrt(d)
-  float* ws;         // partial results when kv_splits > 1
+  int L;                   // sequence length
+  int q_tiles;             // Q tiles per head = ceil(L / (NQ*128))
+  int n_steps;             // KV steps per head = L / TKV
+  int kv_splits;           // CTAs per Q tile along the key axis
+  int stages;              // ring depth
+  float scale_log2;        // log2(e) / sqrt(d)
+  float* ws;               // partial results when kv_splits > 1
+  unsigned int* counters;  // one arrival counter per (Q tile, sub-tile); zero between launches
 };
 
 // Shared-memory footprint helpers (host and device agree through these).
@@ -117,6 +155,9 @@ struct FwdSmem {
 };
 
 constexpr int kMaxStages = 8;
+constexpr float kRescaleThreshold = 8.0f;   // log2 units: P stays below 2^8
+constexpr float kDominanceFactor = 16.0f;   // a new maximum heavier than delta/16 moves the reference
+constexpr int kCounterBytes = 65536;   // head of the workspace: 16384 arrival counters
 
 struct FwdMisc {               // lives in the last 3072 bytes of dynamic shared memory
   float alpha[2][2][kSub];     // [sub-tile][step parity][row] rescale factor
@@ -124,10 +165,12 @@ struct FwdMisc {               // lives in the last 3072 bytes of dynamic shared
   uint64_t kv_full[kMaxStages];
   uint64_t kv_empty[kMaxStages];
   uint64_t s_full[2];
-  uint64_t p_full[2];
+  uint64_t p_full[2];          // first half of P written and O rescaled
+  uint64_t p_half[2];          // second half of P written
   uint64_t o_full[2];
   uint64_t alpha_full[2];
-  uint64_t epi_sync[2];        // softmax warpgroup rendezvous before the TMA store
+  uint64_t epi_sync[2];        // softmax warpgroup rendezvous in the epilogue
+  uint32_t ticket[2];          // arrival order of this CTA among the splits of its Q sub-tile
   uint32_t tmem_slot;
   int abort_flag;
 };
@@ -135,6 +178,47 @@ static_assert(sizeof(FwdMisc) <= 3072, "misc region too large");
 
 // Workspace layout for split keys: per (CTA, sub-tile): O[D/4][128][4] fp32, m[128], delta[128].
 __host__ __device__ constexpr size_t ws_floats_per_sub(int d) { return (size_t)kSub * d + 2 * kSub; }
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// max of s[B..E) as one dependency chain of 3-input maxima
+template <int B, int E>
+__device__ __forceinline__ float chain_max(const uint32_t* s) {
+  float m = __uint_as_float(s[B]);
+#pragma unroll
+  for (int k = B + 1; k + 1 < E; k += 2) m = max3(m, __uint_as_float(s[k]), __uint_as_float(s[k + 1]));
+  if (((E - B - 1) & 1) != 0) m = fmaxf(m, __uint_as_float(s[E - 1]));
+  return m;
+}
+// P = exp2(s * scale - m) for 32 consecutive scores, packed to bf16 pairs; returns their fp32 sum.
+__device__ __forceinline__ float exp_chunk(const uint32_t* s, float scale, float neg_m, uint32_t (&pk)[16]) {
+  float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+    const float e0 = ex2_approx(fmaf(__uint_as_float(s[2 * k]), scale, neg_m));
+    const float e1 = ex2_approx(fmaf(__uint_as_float(s[2 * k + 1]), scale, neg_m));
+    sum0 += e0;
+    sum1 += e1;
+    pk[k] = pack_bf16x2(e0, e1);
+  }
+  return sum0 + sum1;
+}
+// 32 fp32 values of one output row -> bf16, written into a 128-byte-swizzled [128][64] staging chunk.
+__device__ __forceinline__ void stage_row_chunk(uint32_t stage_out, int c, int row, const float (&val)[32]) {
+  const uint32_t chunk_base = stage_out + (c >> 1) * (kSub * 128) + row * 128;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) w[e] = pack_bf16x2(val[u * 8 + 2 * e], val[u * 8 + 2 * e + 1]);
+    const uint32_t unit = (uint32_t)((c & 1) * 4 + u) ^ (uint32_t)(row & 7);   // 128-byte swizzle
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                 ::"r"(chunk_base + unit * 16), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+  }
+}
 
 template <int D, int TKV, int NQ>
 __global__ void __launch_bounds__(512, 1)
@@ -146,6 +230,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   constexpr int KCH = D / 64;                         // 64-column chunks per row
   constexpr int S_COLS = TKV;                         // fp32 score columns per sub-tile
   constexpr int O_COL0 = NQ * S_COLS;                 // O accumulators follow the score buffers
+  constexpr int NCH = TKV / 32;                       // 32-column chunks of one score row
   constexpr int TMEM_COLS = (NQ * (S_COLS + D) <= 32) ? 32
                           : (NQ * (S_COLS + D) <= 64) ? 64
                           : (NQ * (S_COLS + D) <= 128) ? 128
@@ -188,6 +273,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&misc->s_full[i]), 1);
       mbar_init(smem_u32(&misc->p_full[i]), 2 * kSub);   // softmax rows + correction rows
+      mbar_init(smem_u32(&misc->p_half[i]), kSub);
       mbar_init(smem_u32(&misc->o_full[i]), 1);
       mbar_init(smem_u32(&misc->alpha_full[i]), kSub);
       mbar_init(smem_u32(&misc->epi_sync[i]), kSub);
@@ -198,7 +284,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     prefetch_tmap(&tm_v);
     prefetch_tmap(&tm_o);
   }
-  if (warp == 13) {
+  if (warp == 15) {
     tmem_alloc(smem_u32(&misc->tmem_slot), TMEM_COLS);
     tmem_relinquish();
   }
@@ -218,79 +304,94 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t o_tmem = lane_base + O_COL0 + i * D;
     const uint32_t bar_s = smem_u32(&misc->s_full[i]);
     const uint32_t bar_p = smem_u32(&misc->p_full[i]);
+    const uint32_t bar_h = smem_u32(&misc->p_half[i]);
     const uint32_t bar_a = smem_u32(&misc->alpha_full[i]);
+    const float scale = p.scale_log2;
     float m_run = -INFINITY, delta = 0.f;
     bool ok = run;
     for (int jj = 0; ok && jj < n; ++jj) {
       if (!wait_bar_warp(bar_s, jj & 1, abort_flag, wait_info(kRoleSoftmax, kBarSFull, jj))) { ok = false; break; }
       tc_fence_after();
+      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 0);
       uint32_t s[TKV];
 #pragma unroll
-      for (int c = 0; c < TKV / 32; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      for (int c = 0; c < NCH; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
 #pragma unroll
-      for (int c = 0; c < TKV / 32; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-      float mx = __uint_as_float(s[0]);
-#pragma unroll
-      for (int k = 1; k < TKV; ++k) mx = fmaxf(mx, __uint_as_float(s[k]));
-      const float m_new = fmaxf(m_run, mx * p.scale_log2);
-      const float alpha = ex2_approx(m_run - m_new);     // 0 on the first step (m_run = -inf)
+      for (int c = 0; c < NCH; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 1);
+      // row maximum: four independent chains of 3-input maxima
+      const float mx = fmaxf(fmaxf(chain_max<0, TKV / 4>(s), chain_max<TKV / 4, TKV / 2>(s)),
+                             fmaxf(chain_max<TKV / 2, 3 * TKV / 4>(s), chain_max<3 * TKV / 4, TKV>(s)));
+      // Lazy rescale.  The reference maximum m_run moves (and O, delta are rescaled by alpha) only
+      //  (a) when the row maximum grew by more than kRescaleThreshold (log2 units), which bounds
+      //      P = exp2(s - m_run) by 2^threshold, or
+      //  (b) when the new maximum is a dominant key: its weight 2^gap is more than 1/16 of the
+      //      running denominator.  Then P of that key is exactly 1 and carries no bf16 rounding
+      //      error; a stale reference would put the rounding error of the heaviest weight on the
+      //      whole row.  For flat score distributions (b) stops firing after the first few tiles.
+      // Otherwise the reference stays stale, which changes nothing in exact arithmetic because
+      // delta and O carry the same factor.  First step: m_run = -inf, gap = +inf, alpha = 0.
+      const float m_cand = fmaxf(m_run, mx * scale);
+      const float gap = m_cand - m_run;
+      const bool move = (gap > kRescaleThreshold) ||
+                        (gap > 0.f && ex2_approx(gap) * kDominanceFactor > delta);
+      const float m_new = move ? m_cand : m_run;
+      const float alpha = move ? ex2_approx(m_run - m_new) : 1.0f;
       misc->alpha[i][jj & 1][row] = alpha;
       mbar_arrive(bar_a);
+      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 2);
       const float neg_m = -m_new;
       float sum = 0.f;
+      uint32_t pk[16];
+      // first half of the row: the second product may start on it while the rest is computed
 #pragma unroll
-      for (int c = 0; c < TKV / 32; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const float e0 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + 2 * k]), p.scale_log2, neg_m));
-          const float e1 = ex2_approx(fmaf(__uint_as_float(s[c * 32 + 2 * k + 1]), p.scale_log2, neg_m));
-          sum += e0 + e1;
-          pk[k] = pack_bf16x2(e0, e1);
-        }
+      for (int c = 0; c < NCH / 2; ++c) {
+        sum += exp_chunk(&s[c * 32], scale, neg_m, pk);
         tmem_st16(s_tmem + c * 16, pk);                  // P aliases the front of the S buffer
       }
-      delta = delta * alpha + sum;
-      m_run = m_new;
+      uint32_t pk2[16];
+      float sum2 = exp_chunk(&s[(NCH / 2) * 32], scale, neg_m, pk2);
+      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 3);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar_p);
+      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 4);
+      tmem_st16(s_tmem + (NCH / 2) * 16, pk2);
+#pragma unroll
+      for (int c = NCH / 2 + 1; c < NCH; ++c) {
+        sum2 += exp_chunk(&s[c * 32], scale, neg_m, pk);
+        tmem_st16(s_tmem + c * 16, pk);
+      }
+      delta = delta * alpha + (sum + sum2);
+      m_run = m_new;
+      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 5);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_h);
+      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 6);
     }
     // ------------------------------------------------------------- epilogue
+    const uint32_t bar_e = smem_u32(&misc->epi_sync[i]);
+    uint32_t ep_phase = 0;
+    auto wg_sync = [&](uint32_t tag) -> bool {          // all 128 threads of this warpgroup, bounded
+      mbar_arrive(bar_e);
+      const bool r = wait_bar_warp(bar_e, ep_phase, abort_flag, wait_info(kRoleSoftmax, kBarSync, tag));
+      ep_phase ^= 1u;
+      return r;
+    };
     if (ok) ok = wait_bar_warp(smem_u32(&misc->o_full[i]), (n - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, n));
     if (ok) {
       tc_fence_after();
-      if (p.kv_splits == 1) {
-        const float inv = 1.0f / delta;
-        const uint32_t stage_out = q_smem + i * (kSub * D * 2);   // Q sub-tile is dead: reuse it
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(o_tmem + c * 32, r);
-          const uint32_t chunk_base = stage_out + (c >> 1) * (kSub * 128) + row * 128;
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            uint32_t w[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-              w[e] = pack_bf16x2(__uint_as_float(r[u * 8 + 2 * e]) * inv, __uint_as_float(r[u * 8 + 2 * e + 1]) * inv);
-            const uint32_t unit = (uint32_t)((c & 1) * 4 + u) ^ (uint32_t)(row & 7);   // 128-byte swizzle
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                         ::"r"(chunk_base + unit * 16), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-          }
-        }
-        fence_proxy_async_smem();
-        mbar_arrive(smem_u32(&misc->epi_sync[i]));
-        if ((warp & 3) == 0 && lane == 0 &&
-            wait_bar(smem_u32(&misc->epi_sync[i]), 0, abort_flag, wait_info(kRoleSoftmax, kBarSync, n))) {
-#pragma unroll
-          for (int c = 0; c < KCH; ++c)
-            tma_store_3d(&tm_o, stage_out + c * (kSub * 128), c * 64, q_row0 + i * kSub, bh);
-          tma_store_commit();
-          tma_store_wait_read();
-        }
-      } else {
-        float* ws = p.ws + ((size_t)cta * NQ + i) * ws_floats_per_sub(D);
+      const bool direct = (p.kv_splits == 1);
+      bool do_store = direct;
+      float inv = 1.0f / delta;
+      float m_all = 0.f;
+      const size_t per_sub = ws_floats_per_sub(D);
+      const float* tile_ws = p.ws + ((size_t)tile * p.kv_splits * NQ + i) * per_sub;   // split 0 of this sub-tile
+      const size_t split_stride = (size_t)NQ * per_sub;
+      if (!direct) {
+        // un-normalised partial (O, m, delta) of this key range
+        float* ws = p.ws + ((size_t)cta * NQ + i) * per_sub;
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
           uint32_t r[32];
@@ -304,11 +405,75 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         ws[(size_t)kSub * D + row] = m_run;
         ws[(size_t)kSub * D + kSub + row] = delta;
+        __threadfence();
+        ok = wg_sync(1);
+        if (ok) {
+          if (row == 0) misc->ticket[i] = atomicAdd(&p.counters[tile * NQ + i], 1u);
+          ok = wg_sync(2);
+        }
+        if (ok) {
+          do_store = (*reinterpret_cast<volatile uint32_t*>(&misc->ticket[i]) == (uint32_t)(p.kv_splits - 1));
+          if (do_store) {
+            // Last CTA of this Q sub-tile to finish: merge all splits in ascending order
+            // (the merge operator of the online softmax), independent of arrival order.
+            if (row == 0) p.counters[tile * NQ + i] = 0u;
+            __threadfence();
+            m_all = -INFINITY;
+            for (int sp = 0; sp < p.kv_splits; ++sp)
+              m_all = fmaxf(m_all, __ldcg(tile_ws + sp * split_stride + (size_t)kSub * D + row));
+            float d_all = 0.f;
+            for (int sp = 0; sp < p.kv_splits; ++sp) {
+              const float* b = tile_ws + sp * split_stride + (size_t)kSub * D;
+              d_all += __ldcg(b + kSub + row) * exp2f(__ldcg(b + row) - m_all);
+            }
+            inv = 1.0f / d_all;
+          }
+        }
+      }
+      if (ok && do_store) {
+        const uint32_t stage_out = q_smem + i * (kSub * D * 2);   // Q sub-tile is dead: reuse it
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          float val[32];
+          if (direct) {
+            uint32_t r[32];
+            tmem_ld32(o_tmem + c * 32, r);
+#pragma unroll
+            for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(r[k]) * inv;
+          } else {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) val[k] = 0.f;
+            for (int sp = 0; sp < p.kv_splits; ++sp) {
+              const float* b = tile_ws + sp * split_stride;
+              const float w = exp2f(__ldcg(b + (size_t)kSub * D + row) - m_all);
+#pragma unroll
+              for (int g = 0; g < 8; ++g) {
+                const float4 v4 = __ldcg(reinterpret_cast<const float4*>(b) + (size_t)(c * 8 + g) * kSub + row);
+                val[g * 4 + 0] += w * v4.x;
+                val[g * 4 + 1] += w * v4.y;
+                val[g * 4 + 2] += w * v4.z;
+                val[g * 4 + 3] += w * v4.w;
+              }
+            }
+#pragma unroll
+            for (int k = 0; k < 32; ++k) val[k] *= inv;
+          }
+          stage_row_chunk(stage_out, c, row, val);
+        }
+        fence_proxy_async_smem();
+        ok = wg_sync(3);
+        if (ok && (warp & 3) == 0 && lane == 0) {
+#pragma unroll
+          for (int c = 0; c < KCH; ++c)
+            tma_store_3d(&tm_o, stage_out + c * (kSub * 128), c * 64, q_row0 + i * kSub, bh);
+          tma_store_commit();
+          tma_store_wait_read();
+        }
       }
     }
   } else if (warp >= 8 && warp < 12) {
     // ================================================== correction warpgroup
-    setmaxnreg_dec<80>();
+    setmaxnreg_dec<64>();
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     bool ok = run;
@@ -320,8 +485,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           break;
         }
         const float a = misc->alpha[i][jj & 1][row];
+        if (warp == 8) ATTN_TRACE_EVENT(2, jj, i * 4 + 0);
         if (jj > 0) {
           const bool need = __any_sync(0xffffffffu, a != 1.0f);
+          if (warp == 8 && need) ATTN_TRACE_EVENT(2, jj, i * 4 + 1);
           if (need) {
             if (!wait_bar_warp(smem_u32(&misc->o_full[i]), (jj - 1) & 1, abort_flag,
                                wait_info(kRoleCorrection, kBarOFull, jj))) {
@@ -343,25 +510,34 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tc_fence_before();
         }
         mbar_arrive(smem_u32(&misc->p_full[i]));
+        if (warp == 8) ATTN_TRACE_EVENT(2, jj, i * 4 + 2);
       }
     }
   } else if (warp == 12) {
     // ============================================================ MMA issuer
-    setmaxnreg_dec<48>();
-    if (lane == 0 && run) {
-      bool ok = wait_bar(smem_u32(&misc->q_full), 0, abort_flag, wait_info(kRoleMma, kBarQ, 0));
+    // The whole warp walks the loop and the waits (converged control flow keeps descriptors and
+    // counters in the uniform datapath); one elected lane issues the matrix instructions and the
+    // commits.  Sub-tiles are served strictly in turn: that order is what keeps the two softmax
+    // warpgroups half a step apart, so that one computes exponentials while the tensor pipe works
+    // for the other.  (setmaxnreg is warpgroup-aligned: warps 12-15 request the same count.)
+    setmaxnreg_dec<64>();
+    if (run) {
+      bool ok = wait_bar_warp(smem_u32(&misc->q_full), 0, abort_flag, wait_info(kRoleMma, kBarQ, 0));
       int stage = 0;
       uint32_t phase = 0;
       auto advance = [&]() { if (++stage == p.stages) { stage = 0; phase ^= 1u; } };
-      if (ok) ok = wait_bar(smem_u32(&misc->kv_full[stage]), phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 0));
+      if (ok) ok = wait_bar_warp(smem_u32(&misc->kv_full[stage]), phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 0));
       if (ok) {
         tc_fence_after();
+        if (elect_one()) {
 #pragma unroll
-        for (int i = 0; i < NQ; ++i) {
-          issue_qk<D, TKV>(tmem_base + i * S_COLS, q_smem + i * (kSub * D * 2), ring_smem + stage * SM::kStageBytes);
-          umma_commit(smem_u32(&misc->s_full[i]));
+          for (int i = 0; i < NQ; ++i) {
+            issue_qk<D, TKV>(tmem_base + i * S_COLS, q_smem + i * (kSub * D * 2), ring_smem + stage * SM::kStageBytes);
+            umma_commit(smem_u32(&misc->s_full[i]));
+          }
+          umma_commit(smem_u32(&misc->kv_empty[stage]));
         }
-        umma_commit(smem_u32(&misc->kv_empty[stage]));
+        __syncwarp();
         advance();
       }
       for (int jj = 0; ok && jj < n; ++jj) {
@@ -372,28 +548,45 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t k_phase = phase;
         const bool more = (jj + 1 < n);
         if (more) advance();
-        if (!wait_bar(smem_u32(&misc->kv_full[v_stage]), v_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 2 * jj + 1))) { ok = false; break; }
-        if (more && !wait_bar(smem_u32(&misc->kv_full[k_stage]), k_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 2 * jj + 2))) { ok = false; break; }
+        const uint32_t v_smem = ring_smem + v_stage * SM::kStageBytes;
+        const uint32_t k_smem = ring_smem + k_stage * SM::kStageBytes;
+        if (!wait_bar_warp(smem_u32(&misc->kv_full[v_stage]), v_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 2 * jj + 1))) { ok = false; break; }
 #pragma unroll
         for (int i = 0; i < NQ; ++i) {
-          if (!wait_bar(smem_u32(&misc->p_full[i]), jj & 1, abort_flag, wait_info(kRoleMma, kBarPFull, jj))) { ok = false; break; }
+          const uint32_t s_acc = tmem_base + i * S_COLS;
+          const uint32_t o_acc = tmem_base + O_COL0 + i * D;
+          if (!wait_bar_warp(smem_u32(&misc->p_full[i]), jj & 1, abort_flag, wait_info(kRoleMma, kBarPFull, jj))) { ok = false; break; }
           tc_fence_after();
-          issue_pv<D, TKV>(tmem_base + O_COL0 + i * D, tmem_base + i * S_COLS, ring_smem + v_stage * SM::kStageBytes,
-                           jj > 0, TKV * 128, 1024);
-          umma_commit(smem_u32(&misc->o_full[i]));
-          if (i == NQ - 1) umma_commit(smem_u32(&misc->kv_empty[v_stage]));
-          if (more) {
-            issue_qk<D, TKV>(tmem_base + i * S_COLS, q_smem + i * (kSub * D * 2), ring_smem + k_stage * SM::kStageBytes);
-            umma_commit(smem_u32(&misc->s_full[i]));
-            if (i == NQ - 1) umma_commit(smem_u32(&misc->kv_empty[k_stage]));
+          ATTN_TRACE_EVENT(3, jj, i * 4 + 0);
+          if (elect_one()) issue_pv<D, TKV>(o_acc, s_acc, v_smem, jj > 0, TKV * 128, 1024, 0, TKV / 32);
+          __syncwarp();
+          ATTN_TRACE_EVENT(3, jj, i * 4 + 1);
+          if (!wait_bar_warp(smem_u32(&misc->p_half[i]), jj & 1, abort_flag, wait_info(kRoleMma, kBarPFull, 0x8000 | jj))) { ok = false; break; }
+          tc_fence_after();
+          ATTN_TRACE_EVENT(3, jj, i * 4 + 2);
+          if (more && i == 0) {
+            if (!wait_bar_warp(smem_u32(&misc->kv_full[k_stage]), k_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 2 * jj + 2))) { ok = false; break; }
+            tc_fence_after();
           }
+          if (elect_one()) {
+            issue_pv<D, TKV>(o_acc, s_acc, v_smem, true, TKV * 128, 1024, TKV / 32, TKV / 16);
+            umma_commit(smem_u32(&misc->o_full[i]));
+            if (i == NQ - 1) umma_commit(smem_u32(&misc->kv_empty[v_stage]));
+            if (more) {
+              issue_qk<D, TKV>(s_acc, q_smem + i * (kSub * D * 2), k_smem);
+              umma_commit(smem_u32(&misc->s_full[i]));
+              if (i == NQ - 1) umma_commit(smem_u32(&misc->kv_empty[k_stage]));
+            }
+          }
+          __syncwarp();
+          ATTN_TRACE_EVENT(3, jj, i * 4 + 3);
         }
       }
     }
   } else if (warp == 13) {
     // ========================================================== TMA producer
-    setmaxnreg_dec<48>();
-    if (lane == 0 && run) {
+    setmaxnreg_dec<64>();
+    if (run && elect_one()) {
       mbar_arrive_expect_tx(smem_u32(&misc->q_full), SM::kQBytes);
 #pragma unroll
       for (int i = 0; i < NQ; ++i)
@@ -414,6 +607,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t dst = ring_smem + stage * SM::kStageBytes;
 #pragma unroll
         for (int c = 0; c < KCH; ++c) tma_load_3d(dst + c * (TKV * 128), tm, c * 64, kv_row, bh, bar);
+        ATTN_TRACE_EVENT(4, t >> 1, (t & 1));
         ++issued;
         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
       }
@@ -431,59 +625,29 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
     }
   } else {
-    setmaxnreg_dec<48>();
+    setmaxnreg_dec<64>();
+#ifdef ATTN_TRACE
+    // completion times of the matrix products, observed by an otherwise idle warp
+    if (warp == 15 && lane == 0 && run && blockIdx.x == 0) {
+      for (int jj = 0; jj < n && jj < kTraceStep0 + 16; ++jj) {
+        for (int i = 0; i < NQ; ++i) {
+          if (!wait_bar(smem_u32(&misc->o_full[i]), jj & 1, abort_flag, 0)) break;
+          ATTN_TRACE_EVENT(4, jj, 2 + i * 2);
+          if (jj + 1 < n) {
+            if (!wait_bar(smem_u32(&misc->s_full[i]), (jj + 1) & 1, abort_flag, 0)) break;
+            ATTN_TRACE_EVENT(4, jj, 3 + i * 2);
+          }
+        }
+      }
+    }
+#endif
   }
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 13) {
+  if (warp == 15) {
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
-  }
-}
-
-// ---------------------------------------------------------------------------
-// Merge of split-key partials: (m, delta, O)_a (+) (m, delta, O)_b applied over
-// the splits of one Q sub-tile in ascending split order, then O / delta.
-// One block of 128 threads per (tile, sub-tile); thread = row.
-// ---------------------------------------------------------------------------
-template <int D, int NQ>
-__global__ void __launch_bounds__(128) attn_merge_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o,
-                                                         int L, int q_tiles, int kv_splits) {
-  const int tile = blockIdx.x / NQ;
-  const int i = blockIdx.x % NQ;
-  const int row = threadIdx.x;
-  const int q_tile = tile % q_tiles;
-  const int bh = tile / q_tiles;
-  const int grow = q_tile * NQ * kSub + i * kSub + row;
-  const size_t per_sub = ws_floats_per_sub(D);
-  const float* base = ws + ((size_t)tile * kv_splits * NQ + i) * per_sub;
-  const size_t split_stride = (size_t)NQ * per_sub;
-
-  float m_max = -INFINITY;
-  for (int s = 0; s < kv_splits; ++s) m_max = fmaxf(m_max, base[s * split_stride + (size_t)kSub * D + row]);
-  float delta = 0.f;
-  for (int s = 0; s < kv_splits; ++s) {
-    const float* b = base + s * split_stride + (size_t)kSub * D;
-    delta += b[kSub + row] * exp2f(b[row] - m_max);
-  }
-  const float inv = 1.0f / delta;
-  if (grow >= L) return;
-  uint2* orow = reinterpret_cast<uint2*>(o + ((size_t)bh * L + grow) * D);
-  for (int g = 0; g < D / 4; ++g) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < kv_splits; ++s) {
-      const float* b = base + s * split_stride;
-      const float w = exp2f(b[(size_t)kSub * D + row] - m_max);
-      const float4 v = reinterpret_cast<const float4*>(b)[(size_t)g * kSub + row];
-      acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
-    }
-    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-    __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-    uint2 out;
-    out.x = *reinterpret_cast<uint32_t*>(&lo);
-    out.y = *reinterpret_cast<uint32_t*>(&hi);
-    orow[g] = out;
   }
 }
 

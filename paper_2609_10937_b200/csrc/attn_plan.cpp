@@ -21,8 +21,8 @@
 namespace {
 
 // Role structure of the B200 kernel the register budget is derived for.
-constexpr int kRegsCorrection = 80;   // per thread: O-rescale / epilogue warpgroup
-constexpr int kRegsOther = 48;        // per thread: TMA and MMA-issue warps
+constexpr int kRegsCorrection = 64;   // per thread: O-rescale warpgroup
+constexpr int kRegsOther = 64;        // per thread: TMA and MMA-issue warpgroup
 constexpr int kRegsRowOverhead = 32;  // softmax thread: row statistics, addresses, loop state
 constexpr int kSmemReserve = 3072;    // barriers, rescale factors, tensor-memory slot
 constexpr int kMaxStages = 8;
@@ -195,7 +195,8 @@ extern "C" int attn_plan(const attn_hw_desc* desc, int B, int H, int L, int d, a
 extern "C" size_t attn_workspace_bytes(const attn_tiles* t, int B, int H, int L, int d) {
   (void)B; (void)H; (void)L;
   if (!t || !t->feasible || t->kv_splits <= 1 || t->n_q <= 0) return 0;
-  // Per CTA and sub-tile: 128 x d fp32 un-normalised output + 128 (m, delta) pairs.
+  // 64 KB of arrival counters, then per CTA and sub-tile: 128 x d fp32 un-normalised
+  // output + 128 (m, delta) pairs.
   const size_t per_sub = (size_t)128 * (size_t)d * 4 + (size_t)128 * 2 * 4;
-  return (size_t)t->ctas * (size_t)t->n_q * per_sub;
+  return (size_t)65536 + (size_t)t->ctas * (size_t)t->n_q * per_sub;
 }

@@ -120,7 +120,7 @@ def test_workspace_bytes(binding):
     desc = binding.hw_desc_b200()
     t = binding.plan(desc, 1, 1, 16384, 128)
     assert t.kv_splits == 2
-    assert binding.workspace_bytes(t, 1, 1, 16384, 128) == t.ctas * 2 * (128 * 128 + 256) * 4
+    assert binding.workspace_bytes(t, 1, 1, 16384, 128) == 65536 + t.ctas * 2 * (128 * 128 + 256) * 4
     t1 = binding.plan(desc, 4, 32, 4096, 128)
     assert binding.workspace_bytes(t1, 4, 32, 4096, 128) == 0
 

@@ -71,7 +71,7 @@ def test_tmem_machine_capacity_invariants(B, H, L, d):
     assert t["smem_bytes"] <= B200["local_mem_bytes"]                                  # shared memory
     assert t["smem_bytes"] == n_q * 128 * d * 2 + t["kv_stages"] * t["tile_kv"] * d * 2 + 3072
     assert 4 <= t["kv_stages"] <= 8
-    regs_total = 128 * n_q * t["regs_softmax"] + 128 * 80 + 128 * 48                   # register file
+    regs_total = 128 * n_q * t["regs_softmax"] + 128 * 64 + 128 * 64                   # register file
     assert regs_total <= 65536 and t["regs_softmax"] <= 248
     assert t["tile_kv"] + t["tile_kv"] // 4 + 32 <= t["regs_softmax"]
     assert t["ctas"] == t["tiles"] * t["kv_splits"]
