@@ -170,6 +170,7 @@ struct FwdMisc {               // lives in the last 3072 bytes of dynamic shared
   uint64_t o_full[2];
   uint64_t alpha_full[2];
   uint64_t epi_sync[2];        // softmax warpgroup rendezvous in the epilogue
+  uint64_t dbg_bar[2];         // trace builds only: completion of the first half of P V
   uint32_t ticket[2];          // arrival order of this CTA among the splits of its Q sub-tile
   uint32_t tmem_slot;
   int abort_flag;
@@ -193,18 +194,64 @@ __device__ __forceinline__ float chain_max(const uint32_t* s) {
   if (((E - B - 1) & 1) != 0) m = fmaxf(m, __uint_as_float(s[E - 1]));
   return m;
 }
-// P = exp2(s * scale - m) for 32 consecutive scores, packed to bf16 pairs; returns their fp32 sum.
-__device__ __forceinline__ float exp_chunk(const uint32_t* s, float scale, float neg_m, uint32_t (&pk)[16]) {
-  float sum0 = 0.f, sum1 = 0.f;
+// Constants of the exponential evaluation, packed once per thread.
+struct ExpConsts {
+  uint64_t scale2, magic2, neg_magic2, minus_one2, c3, c2, c1, c0;
+};
+__device__ __forceinline__ ExpConsts make_exp_consts(float scale) {
+  ExpConsts k;
+  k.scale2 = pack_f32x2(scale, scale);
+  k.magic2 = pack_f32x2(12582912.0f, 12582912.0f);          // 1.5 * 2^23: adding it rounds to an integer
+  k.neg_magic2 = pack_f32x2(-12582912.0f, -12582912.0f);
+  k.minus_one2 = pack_f32x2(-1.0f, -1.0f);
+  // minimax cubic for 2^f on [-0.5, 0.5], relative error 7.6e-5 (bf16 rounding of P is 2e-3)
+  k.c3 = pack_f32x2(0.055168043822050095f, 0.055168043822050095f);
+  k.c2 = pack_f32x2(0.24260213971138f, 0.24260213971138f);
+  k.c1 = pack_f32x2(0.6932607889175415f, 0.6932607889175415f);
+  k.c0 = pack_f32x2(0.9999286532402039f, 0.9999286532402039f);
+  return k;
+}
+// exp2 of a packed pair on the FMA/ALU pipes (no MUFU): x = n + f with n integer, f in [-0.5, 0.5];
+// 2^f by the cubic, 2^n by adding n to the exponent field.  x is clamped at -126 (result ~1e-38).
+__device__ __forceinline__ void exp2_poly_pair(uint64_t x2, const ExpConsts& k, float& e0, float& e1) {
+  float x0, x1;
+  unpack_f32x2(x2, x0, x1);
+  x0 = fmaxf(x0, -126.0f);
+  x1 = fmaxf(x1, -126.0f);
+  const uint64_t xc = pack_f32x2(x0, x1);
+  const uint64_t r2 = add_f32x2(xc, k.magic2);
+  const uint64_t n2 = add_f32x2(r2, k.neg_magic2);
+  const uint64_t f2 = fma_f32x2(n2, k.minus_one2, xc);
+  uint64_t p2 = fma_f32x2(f2, k.c3, k.c2);
+  p2 = fma_f32x2(p2, f2, k.c1);
+  p2 = fma_f32x2(p2, f2, k.c0);
+  float p0, p1, r0, r1;
+  unpack_f32x2(p2, p0, p1);
+  unpack_f32x2(r2, r0, r1);
+  e0 = __int_as_float(__float_as_int(p0) + (__float_as_int(r0) << 23));
+  e1 = __int_as_float(__float_as_int(p1) + (__float_as_int(r1) << 23));
+}
+// P = exp2(s * scale - m) for 32 consecutive scores, packed to bf16 pairs; adds them to the packed
+// partial sums.  Of every eight pairs, kPolyPairsPer8 are evaluated by the polynomial and the rest
+// by MUFU ex2, which balances the two pipes (MUFU alone would take as long as the matrix products).
+constexpr int kPolyPairsPer8 = 3;
+__device__ __forceinline__ void exp_chunk(const uint32_t* s, const ExpConsts& k, uint64_t neg_m2, uint64_t& sum2,
+                                          uint32_t (&pk)[16]) {
 #pragma unroll
-  for (int k = 0; k < 16; ++k) {
-    const float e0 = ex2_approx(fmaf(__uint_as_float(s[2 * k]), scale, neg_m));
-    const float e1 = ex2_approx(fmaf(__uint_as_float(s[2 * k + 1]), scale, neg_m));
-    sum0 += e0;
-    sum1 += e1;
-    pk[k] = pack_bf16x2(e0, e1);
+  for (int j = 0; j < 16; ++j) {
+    const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[2 * j]), __uint_as_float(s[2 * j + 1])), k.scale2, neg_m2);
+    float e0, e1;
+    if ((j & 7) < kPolyPairsPer8) {
+      exp2_poly_pair(x2, k, e0, e1);
+    } else {
+      float x0, x1;
+      unpack_f32x2(x2, x0, x1);
+      e0 = ex2_approx(x0);
+      e1 = ex2_approx(x1);
+    }
+    sum2 = add_f32x2(sum2, pack_f32x2(e0, e1));
+    pk[j] = pack_bf16x2(e0, e1);
   }
-  return sum0 + sum1;
 }
 // 32 fp32 values of one output row -> bf16, written into a 128-byte-swizzled [128][64] staging chunk.
 __device__ __forceinline__ void stage_row_chunk(uint32_t stage_out, int c, int row, const float (&val)[32]) {
@@ -277,6 +324,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(smem_u32(&misc->o_full[i]), 1);
       mbar_init(smem_u32(&misc->alpha_full[i]), kSub);
       mbar_init(smem_u32(&misc->epi_sync[i]), kSub);
+      mbar_init(smem_u32(&misc->dbg_bar[i]), 1);
     }
     fence_mbar_init();
     prefetch_tmap(&tm_q);
@@ -307,6 +355,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t bar_h = smem_u32(&misc->p_half[i]);
     const uint32_t bar_a = smem_u32(&misc->alpha_full[i]);
     const float scale = p.scale_log2;
+    const ExpConsts ek = make_exp_consts(scale);
     float m_run = -INFINITY, delta = 0.f;
     bool ok = run;
     for (int jj = 0; ok && jj < n; ++jj) {
@@ -320,8 +369,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       for (int c = 0; c < NCH; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
       if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 1);
       // row maximum: four independent chains of 3-input maxima
-      const float mx = fmaxf(fmaxf(chain_max<0, TKV / 4>(s), chain_max<TKV / 4, TKV / 2>(s)),
-                             fmaxf(chain_max<TKV / 2, 3 * TKV / 4>(s), chain_max<3 * TKV / 4, TKV>(s)));
+      const float mx = fmaxf(
+          max3(chain_max<0, TKV / 8>(s), chain_max<TKV / 8, TKV / 4>(s), chain_max<TKV / 4, 3 * TKV / 8>(s)),
+          max3(chain_max<3 * TKV / 8, TKV / 2>(s), chain_max<TKV / 2, 5 * TKV / 8>(s),
+               fmaxf(chain_max<5 * TKV / 8, 3 * TKV / 4>(s),
+                     fmaxf(chain_max<3 * TKV / 4, 7 * TKV / 8>(s), chain_max<7 * TKV / 8, TKV>(s)))));
       // Lazy rescale.  The reference maximum m_run moves (and O, delta are rescaled by alpha) only
       //  (a) when the row maximum grew by more than kRescaleThreshold (log2 units), which bounds
       //      P = exp2(s - m_run) by 2^threshold, or
@@ -340,17 +392,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       misc->alpha[i][jj & 1][row] = alpha;
       mbar_arrive(bar_a);
       if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 2);
-      const float neg_m = -m_new;
-      float sum = 0.f;
+      const uint64_t neg_m2 = pack_f32x2(-m_new, -m_new);
+      uint64_t sum_a = 0ull, sum_b = 0ull;               // packed (0.f, 0.f)
       uint32_t pk[16];
       // first half of the row: the second product may start on it while the rest is computed
 #pragma unroll
       for (int c = 0; c < NCH / 2; ++c) {
-        sum += exp_chunk(&s[c * 32], scale, neg_m, pk);
+        exp_chunk(&s[c * 32], ek, neg_m2, sum_a, pk);
         tmem_st16(s_tmem + c * 16, pk);                  // P aliases the front of the S buffer
       }
       uint32_t pk2[16];
-      float sum2 = exp_chunk(&s[(NCH / 2) * 32], scale, neg_m, pk2);
+      exp_chunk(&s[(NCH / 2) * 32], ek, neg_m2, sum_b, pk2);
       if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 3);
       tmem_wait_st();
       tc_fence_before();
@@ -359,9 +411,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tmem_st16(s_tmem + (NCH / 2) * 16, pk2);
 #pragma unroll
       for (int c = NCH / 2 + 1; c < NCH; ++c) {
-        sum2 += exp_chunk(&s[c * 32], scale, neg_m, pk);
+        exp_chunk(&s[c * 32], ek, neg_m2, sum_b, pk);
         tmem_st16(s_tmem + c * 16, pk);
       }
+      float sa0, sa1, sb0, sb1;
+      unpack_f32x2(sum_a, sa0, sa1);
+      unpack_f32x2(sum_b, sb0, sb1);
+      const float sum = sa0 + sa1, sum2 = sb0 + sb1;
       delta = delta * alpha + (sum + sum2);
       m_run = m_new;
       if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 5);
@@ -558,7 +614,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (!wait_bar_warp(smem_u32(&misc->p_full[i]), jj & 1, abort_flag, wait_info(kRoleMma, kBarPFull, jj))) { ok = false; break; }
           tc_fence_after();
           ATTN_TRACE_EVENT(3, jj, i * 4 + 0);
-          if (elect_one()) issue_pv<D, TKV>(o_acc, s_acc, v_smem, jj > 0, TKV * 128, 1024, 0, TKV / 32);
+          if (elect_one()) {
+            issue_pv<D, TKV>(o_acc, s_acc, v_smem, jj > 0, TKV * 128, 1024, 0, TKV / 32);
+#ifdef ATTN_TRACE
+            umma_commit(smem_u32(&misc->dbg_bar[i]));
+#endif
+          }
           __syncwarp();
           ATTN_TRACE_EVENT(3, jj, i * 4 + 1);
           if (!wait_bar_warp(smem_u32(&misc->p_half[i]), jj & 1, abort_flag, wait_info(kRoleMma, kBarPFull, 0x8000 | jj))) { ok = false; break; }
@@ -607,7 +668,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t dst = ring_smem + stage * SM::kStageBytes;
 #pragma unroll
         for (int c = 0; c < KCH; ++c) tma_load_3d(dst + c * (TKV * 128), tm, c * 64, kv_row, bh, bar);
-        ATTN_TRACE_EVENT(4, t >> 1, (t & 1));
         ++issued;
         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
       }
@@ -631,6 +691,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (warp == 15 && lane == 0 && run && blockIdx.x == 0) {
       for (int jj = 0; jj < n && jj < kTraceStep0 + 16; ++jj) {
         for (int i = 0; i < NQ; ++i) {
+          if (!wait_bar(smem_u32(&misc->dbg_bar[i]), jj & 1, abort_flag, 0)) break;
+          ATTN_TRACE_EVENT(4, jj, i);          // overwrites the loader's K/V issue slots
           if (!wait_bar(smem_u32(&misc->o_full[i]), jj & 1, abort_flag, 0)) break;
           ATTN_TRACE_EVENT(4, jj, 2 + i * 2);
           if (jj + 1 < n) {
