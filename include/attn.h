@@ -44,7 +44,8 @@ typedef enum attn_status {
   ATTN_ERR_NEED_WORKSPACE = -7,    /* plan splits the keys but no workspace was supplied  */
   ATTN_ERR_CUDA = -8,              /* a CUDA runtime/driver call failed                   */
   ATTN_ERR_DEVICE_TIMEOUT = -9,    /* a bounded device-side wait expired                  */
-  ATTN_ERR_BAD_TILES = -10         /* tile override not among the compiled variants       */
+  ATTN_ERR_BAD_TILES = -10,        /* tile override not among the compiled variants       */
+  ATTN_ERR_SCRATCH_LIMIT = -11     /* problem needs more than the built-in scratch array  */
 } attn_status;
 
 /* Which capacity fixed the tile (the "binding constraint" returned by the
@@ -180,6 +181,39 @@ int attn_forward_simple(const void *q, const void *k, const void *v, void *o,
 int attn_forward_host(const void *q_host, const void *k_host, const void *v_host, void *o_host,
                       int B, int H, int L, int d, void *dev_scratch, size_t dev_scratch_bytes,
                       void *cuda_stream);
+
+/*
+ * Allocation-free form of attn_forward.  (The paper has no counterpart: this is a
+ * packaging variant of the same kernel, not another algorithm.)
+ *
+ * Who it is for: callers that are not allowed to obtain device memory at the
+ * point where they run attention -- a serving loop whose memory budget was
+ * fixed at start-up, code running under an allocator that must not be
+ * re-entered, a plug-in that only ever receives its input and output buffers.
+ * attn_forward needs a caller-supplied workspace whenever the plan splits the
+ * key axis; such callers have nowhere to get one from.  Here the partial
+ * results and arrival counters live in an array that is part of the library
+ * image itself: ATTN_STATIC_SCRATCH_BYTES (about 18.9 MiB) of device memory,
+ * held by every GPU that loads the library until the process exits.
+ *
+ * q, k, v, o, shapes, stream and results are exactly those of attn_forward (same
+ * kernel, same closed-form plan, bitwise the same output).  The call makes no
+ * cudaMalloc / cudaFree and calls no allocating library routine.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current) and remembers it; make that first call outside any
+ *     stream capture.
+ *   - Every call on a device shares the one array, and the array keeps whatever
+ *     the previous call left in it: the counters that must start at zero are
+ *     cleared on `cuda_stream` before each launch.  Two calls that overlap in
+ *     time on one GPU (different streams, or another thread) race on it and give
+ *     wrong results; serialise them.
+ *   - ATTN_ERR_SCRATCH_LIMIT if the plan for this shape needs more scratch than
+ *     ATTN_STATIC_SCRATCH_BYTES (never the case for the built-in B200 descriptor
+ *     with d <= 128); other errors as attn_forward.
+ */
+#define ATTN_STATIC_SCRATCH_BYTES 19767296
+int attn_forward_static_scratch(const void *q, const void *k, const void *v, void *o,
+                                int B, int H, int L, int d, void *cuda_stream);
 
 /* Synchronises cuda_stream and reports whether any bounded device-side wait
  * expired since the last query (ATTN_ERR_DEVICE_TIMEOUT) -- then detail[0..3]

@@ -17,12 +17,13 @@ LIB_PATH = _PKG / "libattn_b200.so"
 ATTN_OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_MISALIGNED, ERR_ALIASING = -1, -2, -3, -4
 ERR_INFEASIBLE_PLAN, ERR_WRONG_ARCH, ERR_NEED_WORKSPACE, ERR_CUDA = -5, -6, -7, -8
-ERR_DEVICE_TIMEOUT, ERR_BAD_TILES = -9, -10
+ERR_DEVICE_TIMEOUT, ERR_BAD_TILES, ERR_SCRATCH_LIMIT = -9, -10, -11
 BIND_NAMES = ("none", "smem", "tmem", "reg", "atom", "shape")
 
 EXPORTED_SYMBOLS = (
     "attn_hw_desc_b200", "attn_hw_desc_query", "attn_plan", "attn_workspace_bytes", "attn_set_workspace",
-    "attn_forward", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_last_device_status",
+    "attn_forward", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_static_scratch",
+    "attn_last_device_status",
     "attn_last_launch_count", "attn_status_string", "attn_last_cuda_error",
 )
 
@@ -77,6 +78,7 @@ def lib() -> ctypes.CDLL:
         L.attn_forward_tiles.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, ctypes.POINTER(AttnTiles), vp]
         L.attn_forward_simple.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
         L.attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_size_t, vp]
+        L.attn_forward_static_scratch.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
         L.attn_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.attn_last_launch_count.argtypes = []
         L.attn_status_string.argtypes = [i32]
@@ -179,6 +181,20 @@ def forward(q, k, v, o=None):
             ensure_workspace(dev, workspace_bytes(t, B, H, L, d))
         _check(lib().attn_forward(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d, stream),
                "attn_forward")
+    return o
+
+
+def forward_static_scratch(q, k, v, o):
+    """attn_forward without any allocation: the output tensor must be supplied, and the split-key
+    scratch is the array built into the library (shared by all calls on a device; do not overlap calls)."""
+    import torch
+
+    if o is None:
+        raise ValueError("the allocation-free entry point needs a caller-supplied output tensor")
+    o, B, H, L, d, dev, stream = _prep(q, k, v, o)
+    with torch.cuda.device(dev):
+        _check(lib().attn_forward_static_scratch(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                                 B, H, L, d, stream), "attn_forward_static_scratch")
     return o
 
 

@@ -299,6 +299,56 @@ extern "C" int attn_forward_host(const void* q_host, const void* k_host, const v
   return ATTN_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Allocation-free entry point.  The scratch that a split plan needs (arrival counters followed by
+// the partial outputs) is this file-scope device array instead of a caller-supplied workspace.
+// In host code the name below is only a handle: its device address is obtained once per device
+// with cudaGetSymbolAddress and that pointer is what the kernel receives.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_attn_static_scratch[ATTN_STATIC_SCRATCH_BYTES];
+
+namespace {
+void* g_static_scratch_ptr[kMaxDevices] = {};
+std::mutex g_static_mu;
+
+// Device address of the array on the current device, looked up on first use.
+int static_scratch_address(void** out) {
+  int dev = 0;
+  ATTN_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return ATTN_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(g_static_mu);
+  if (!g_static_scratch_ptr[dev]) {
+    void* ptr = nullptr;
+    ATTN_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_attn_static_scratch));
+    if (!ptr) return ATTN_ERR_CUDA;
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return ATTN_OK;
+}
+}  // namespace
+
+extern "C" int attn_forward_static_scratch(const void* q, const void* k, const void* v, void* o, int B, int H, int L,
+                                           int d, void* cuda_stream) {
+  t_launch_count = 0;
+  int rc = check_args(q, k, v, o, B, H, L, d);
+  if (rc != ATTN_OK) return rc;
+  DeviceState* st = nullptr;
+  if ((rc = device_state(&st)) != ATTN_OK) return rc;
+  attn_tiles t;
+  if ((rc = attn_plan(&st->desc, B, H, L, d, &t)) != ATTN_OK) return rc;
+  if (!t.feasible) return ATTN_ERR_INFEASIBLE_PLAN;
+  void* scratch = nullptr;
+  if ((rc = static_scratch_address(&scratch)) != ATTN_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (t.kv_splits > 1) {
+    if (attn_workspace_bytes(&t, B, H, L, d) > (size_t)ATTN_STATIC_SCRATCH_BYTES) return ATTN_ERR_SCRATCH_LIMIT;
+    // the array keeps the previous call's contents: the arrival counters must start at zero
+    ATTN_CUDA_TRY(cudaMemsetAsync(scratch, 0, attn::kCounterBytes, stream));
+  }
+  return dispatch_fwd(q, k, v, o, B, H, L, d, t, static_cast<float*>(scratch), stream);
+}
+
 extern "C" int attn_last_device_status(void* cuda_stream, uint32_t* detail) {
   ATTN_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
   unsigned int h[4] = {0, 0, 0, 0};
@@ -345,6 +395,7 @@ extern "C" const char* attn_status_string(int status) {
     case ATTN_ERR_CUDA: return "CUDA error (see attn_last_cuda_error)";
     case ATTN_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
     case ATTN_ERR_BAD_TILES: return "tile override not available";
+    case ATTN_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the library's built-in array holds";
     default: return "unknown status";
   }
 }
