@@ -234,7 +234,15 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, const ExpConsts& k, 
 // P = exp2(s * scale - m) for 32 consecutive scores, packed to bf16 pairs; adds them to the packed
 // partial sums.  Of every eight pairs, kPolyPairsPer8 are evaluated by the polynomial and the rest
 // by MUFU ex2, which balances the two pipes (MUFU alone would take as long as the matrix products).
-constexpr int kPolyPairsPer8 = 3;
+// Two of eight measured best on B200: more polynomial work costs issue slots that the other warps
+// of the scheduler partition (and the MMA-issuing warp) need.
+#ifndef ATTN_POLY_PAIRS_D128
+#define ATTN_POLY_PAIRS_D128 2
+#endif
+#ifndef ATTN_POLY_PAIRS_D64
+#define ATTN_POLY_PAIRS_D64 2
+#endif
+template <int kPolyPairsPer8>
 __device__ __forceinline__ void exp_chunk(const uint32_t* s, const ExpConsts& k, uint64_t neg_m2, uint64_t& sum2,
                                           uint32_t (&pk)[16]) {
 #pragma unroll
@@ -278,6 +286,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   constexpr int S_COLS = TKV;                         // fp32 score columns per sub-tile
   constexpr int O_COL0 = NQ * S_COLS;                 // O accumulators follow the score buffers
   constexpr int NCH = TKV / 32;                       // 32-column chunks of one score row
+  constexpr int kPoly = (D == 128) ? ATTN_POLY_PAIRS_D128 : ATTN_POLY_PAIRS_D64;   // polynomial pairs per 8
   constexpr int TMEM_COLS = (NQ * (S_COLS + D) <= 32) ? 32
                           : (NQ * (S_COLS + D) <= 64) ? 64
                           : (NQ * (S_COLS + D) <= 128) ? 128
@@ -363,17 +372,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tc_fence_after();
       if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 0);
       uint32_t s[TKV];
+      // load the row in two halves: the maximum of the first half is taken while the second is in flight
 #pragma unroll
-      for (int c = 0; c < NCH; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      for (int c = 0; c < NCH / 2; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
 #pragma unroll
-      for (int c = 0; c < NCH; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      for (int c = 0; c < NCH / 2; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+#pragma unroll
+      for (int c = NCH / 2; c < NCH; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      const float mx_a = fmaxf(fmaxf(chain_max<0, TKV / 8>(s), chain_max<TKV / 8, TKV / 4>(s)),
+                               fmaxf(chain_max<TKV / 4, 3 * TKV / 8>(s), chain_max<3 * TKV / 8, TKV / 2>(s)));
+#pragma unroll
+      for (int c = NCH / 2; c < NCH; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
       if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 1);
-      // row maximum: four independent chains of 3-input maxima
-      const float mx = fmaxf(
-          max3(chain_max<0, TKV / 8>(s), chain_max<TKV / 8, TKV / 4>(s), chain_max<TKV / 4, 3 * TKV / 8>(s)),
-          max3(chain_max<3 * TKV / 8, TKV / 2>(s), chain_max<TKV / 2, 5 * TKV / 8>(s),
-               fmaxf(chain_max<5 * TKV / 8, 3 * TKV / 4>(s),
-                     fmaxf(chain_max<3 * TKV / 4, 7 * TKV / 8>(s), chain_max<7 * TKV / 8, TKV>(s)))));
+      const float mx_b = fmaxf(fmaxf(chain_max<TKV / 2, 5 * TKV / 8>(s), chain_max<5 * TKV / 8, 3 * TKV / 4>(s)),
+                               fmaxf(chain_max<3 * TKV / 4, 7 * TKV / 8>(s), chain_max<7 * TKV / 8, TKV>(s)));
+      const float mx = fmaxf(mx_a, mx_b);
       // Lazy rescale.  The reference maximum m_run moves (and O, delta are rescaled by alpha) only
       //  (a) when the row maximum grew by more than kRescaleThreshold (log2 units), which bounds
       //      P = exp2(s - m_run) by 2^threshold, or
@@ -385,10 +398,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // delta and O carry the same factor.  First step: m_run = -inf, gap = +inf, alpha = 0.
       const float m_cand = fmaxf(m_run, mx * scale);
       const float gap = m_cand - m_run;
-      const bool move = (gap > kRescaleThreshold) ||
-                        (gap > 0.f && ex2_approx(gap) * kDominanceFactor > delta);
+      const float shrink = ex2_approx(-gap);             // 2^-gap: the rescale factor if the reference moves
+      const bool move = (gap > kRescaleThreshold) || (gap > 0.f && kDominanceFactor > delta * shrink);
       const float m_new = move ? m_cand : m_run;
-      const float alpha = move ? ex2_approx(m_run - m_new) : 1.0f;
+      const float alpha = move ? shrink : 1.0f;
       misc->alpha[i][jj & 1][row] = alpha;
       mbar_arrive(bar_a);
       if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 2);
@@ -398,11 +411,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // first half of the row: the second product may start on it while the rest is computed
 #pragma unroll
       for (int c = 0; c < NCH / 2; ++c) {
-        exp_chunk(&s[c * 32], ek, neg_m2, sum_a, pk);
+        exp_chunk<kPoly>(&s[c * 32], ek, neg_m2, sum_a, pk);
         tmem_st16(s_tmem + c * 16, pk);                  // P aliases the front of the S buffer
       }
       uint32_t pk2[16];
-      exp_chunk(&s[(NCH / 2) * 32], ek, neg_m2, sum_b, pk2);
+      exp_chunk<kPoly>(&s[(NCH / 2) * 32], ek, neg_m2, sum_b, pk2);
       if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 3);
       tmem_wait_st();
       tc_fence_before();
@@ -411,7 +424,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tmem_st16(s_tmem + (NCH / 2) * 16, pk2);
 #pragma unroll
       for (int c = NCH / 2 + 1; c < NCH; ++c) {
-        exp_chunk(&s[c * 32], ek, neg_m2, sum_b, pk);
+        exp_chunk<kPoly>(&s[c * 32], ek, neg_m2, sum_b, pk);
         tmem_st16(s_tmem + c * 16, pk);
       }
       float sa0, sa1, sb0, sb1;
