@@ -93,13 +93,13 @@ typedef struct attn_tiles {
   int32_t n_q;            /* Q sub-tiles per CTA (ping-pong partners), 1 or 2           */
   int32_t n_s;            /* score buffers per sub-tile (1)                             */
   int32_t kv_stages;      /* depth of the shared-memory K/V ring (one K or V tile each) */
-  int32_t kv_splits;      /* CTAs sharing one Q tile along the key axis (merge operator)*/
+  int32_t kv_splits;      /* most CTAs sharing one Q tile along the key axis = ceil(ctas / tiles) */
   int32_t smem_bytes;     /* dynamic shared memory per CTA                              */
   int32_t tmem_columns;   /* tensor-memory columns allocated per CTA                    */
   int32_t regs_softmax;   /* register allowance of a softmax thread                     */
   int32_t threads;        /* threads per CTA                                            */
   int32_t tiles;          /* B * H * ceil(L / tile_q)                                   */
-  int32_t ctas;           /* tiles * kv_splits                                          */
+  int32_t ctas;           /* grid size: tiles, or min(num_units, tiles*steps/4) if under-occupied */
   float ctas_per_unit;    /* ctas / num_units                                           */
   float wave_efficiency;  /* ctas_per_unit / ceil(ctas_per_unit)                        */
   int32_t feasible;       /* 1 if a tile choice fits                                    */
@@ -126,9 +126,9 @@ int attn_hw_desc_query(int device, attn_hw_desc *out);
  */
 int attn_plan(const attn_hw_desc *desc, int B, int H, int L, int d, attn_tiles *out);
 
-/* Bytes of workspace attn_forward* needs for this plan: 0 unless kv_splits > 1
- * (64 KB of arrival counters, then the partial outputs and row statistics of
- * the merge operator, Section "Online Softmax"). */
+/* Bytes of workspace attn_forward* needs for this plan: 0 unless ctas > tiles
+ * (64 KB of arrival counters, then ctas + tiles slots of partial outputs and row
+ * statistics for the merge operator, Section "Online Softmax"). */
 size_t attn_workspace_bytes(const attn_tiles *tiles, int B, int H, int L, int d);
 
 /* Registers a caller-owned device buffer as the workspace of `device` (pass
@@ -148,9 +148,11 @@ int attn_set_workspace(int device, void *dev_ptr, size_t bytes);
 int attn_forward(const void *q, const void *k, const void *v, void *o,
                  int B, int H, int L, int d, void *cuda_stream);
 
-/* Same, with tile fields overridden (tile sweep only).  Honoured fields:
- * n_q (1|2), tile_kv (64|128), kv_stages (2..plan maximum), kv_splits (>= 1).
- * ATTN_ERR_BAD_TILES if the combination was not compiled or does not fit. */
+/* Same, with tile fields overridden (tile sweep only).  Honoured fields (0 keeps
+ * the closed-form value): n_q (1|2), tile_kv (64|128), kv_stages (2..plan maximum),
+ * kv_splits (that many CTAs per Q tile) or ctas (the grid size itself, from the
+ * number of Q tiles up to tiles * KV steps).  ATTN_ERR_BAD_TILES if the combination
+ * was not compiled or does not fit. */
 int attn_forward_tiles(const void *q, const void *k, const void *v, void *o,
                        int B, int H, int L, int d, const attn_tiles *override_tiles,
                        void *cuda_stream);
@@ -193,7 +195,7 @@ int attn_forward_host(const void *q_host, const void *k_host, const void *v_host
  * attn_forward needs a caller-supplied workspace whenever the plan splits the
  * key axis; such callers have nowhere to get one from.  Here the partial
  * results and arrival counters live in an array that is part of the library
- * image itself: ATTN_STATIC_SCRATCH_BYTES (about 18.9 MiB) of device memory,
+ * image itself: ATTN_STATIC_SCRATCH_BYTES (about 37.5 MiB) of device memory,
  * held by every GPU that loads the library until the process exits.
  *
  * q, k, v, o, shapes, stream and results are exactly those of attn_forward (same
@@ -211,7 +213,7 @@ int attn_forward_host(const void *q_host, const void *k_host, const void *v_host
  *     ATTN_STATIC_SCRATCH_BYTES (never the case for the built-in B200 descriptor
  *     with d <= 128); other errors as attn_forward.
  */
-#define ATTN_STATIC_SCRATCH_BYTES 19767296
+#define ATTN_STATIC_SCRATCH_BYTES 39335936
 int attn_forward_static_scratch(const void *q, const void *k, const void *v, void *o,
                                 int B, int H, int L, int d, void *cuda_stream);
 

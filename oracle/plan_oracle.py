@@ -63,6 +63,7 @@ _MAX_STAGES = 8
 _MIN_STAGES = 4
 _MIN_TILE_KV = 32
 _MIN_STEPS_PER_SPLIT = 4
+_SEGMENT_OVERHEAD_STEPS = 3
 
 
 def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int) -> dict:
@@ -103,10 +104,18 @@ def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int) -> dic
     tiles = B * H * -(-L // tile_q)
     steps = -(-L // tile_kv)
     under = tiles < desc["num_units"]
-    kv_splits = 1
+    ctas = tiles
     if under:
-        kv_splits = max(1, min(desc["num_units"] // tiles, steps // _MIN_STEPS_PER_SPLIT))
-    ctas = tiles * kv_splits
+        k = max(1, min(desc["num_units"] // tiles, steps // _MIN_STEPS_PER_SPLIT))
+        cost_uniform = -(-steps // k) + _SEGMENT_OVERHEAD_STEPS
+        total = tiles * steps
+        g = min(total // _MIN_STEPS_PER_SPLIT, desc["num_units"])
+        ctas = tiles * k
+        if g > tiles * k:
+            cost_balanced = -(-total // g) + 2 * _SEGMENT_OVERHEAD_STEPS
+            if cost_balanced < cost_uniform:
+                ctas = g
+    kv_splits = -(-ctas // tiles)
     per_unit = ctas / desc["num_units"]
     cols = n_q * (tile_kv + d)
     return dict(feasible=True, binding=binding, tile_q=tile_q, tile_kv=tile_kv, n_q=n_q, n_s=1,

@@ -177,7 +177,7 @@ def forward(q, k, v, o=None):
     o, B, H, L, d, dev, stream = _prep(q, k, v, o)
     with torch.cuda.device(dev):
         t = plan(_device_desc(dev), B, H, L, d)
-        if t.feasible and t.kv_splits > 1:
+        if t.feasible and t.ctas > t.tiles:
             ensure_workspace(dev, workspace_bytes(t, B, H, L, d))
         _check(lib().attn_forward(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d, stream),
                "attn_forward")
@@ -198,22 +198,25 @@ def forward_static_scratch(q, k, v, o):
     return o
 
 
-def forward_tiles(q, k, v, o=None, *, n_q=0, tile_kv=0, kv_stages=0, kv_splits=0):
-    """Same with tile fields overridden (0 keeps the closed-form value); tile sweep only."""
+def forward_tiles(q, k, v, o=None, *, n_q=0, tile_kv=0, kv_stages=0, kv_splits=0, ctas=0):
+    """Same with tile fields overridden (0 keeps the closed-form value); tile sweep only.
+
+    kv_splits asks for that many CTAs per Q tile; ctas sets the grid size directly (any value from
+    the number of Q tiles up to the number of (Q tile, KV step) units)."""
     import torch
 
     o, B, H, L, d, dev, stream = _prep(q, k, v, o)
     with torch.cuda.device(dev):
-        base = plan(_device_desc(dev), B, H, L, d)
+        desc = _device_desc(dev)
+        base = plan(desc, B, H, L, d)
         ov = AttnTiles()
-        ov.n_q, ov.tile_kv, ov.kv_stages, ov.kv_splits = n_q, tile_kv, kv_stages, kv_splits
+        ov.n_q, ov.tile_kv, ov.kv_stages, ov.kv_splits, ov.ctas = n_q, tile_kv, kv_stages, kv_splits, ctas
         eff_nq = n_q or base.n_q
-        eff_splits = kv_splits or base.kv_splits
-        if eff_splits > 1:
-            w = AttnTiles()
-            w.feasible, w.kv_splits, w.n_q = 1, eff_splits, eff_nq
-            w.ctas = B * H * math.ceil(L / (128 * eff_nq)) * eff_splits
-            ensure_workspace(dev, workspace_bytes(w, B, H, L, d))
+        tiles = B * H * math.ceil(L / (128 * eff_nq))
+        w = AttnTiles()          # upper bound of what the call can need
+        w.feasible, w.n_q, w.tiles = 1, eff_nq, tiles
+        w.ctas = max(ctas, tiles * max(kv_splits, 1), desc.num_units, tiles + 1)
+        ensure_workspace(dev, workspace_bytes(w, B, H, L, d))
         _check(lib().attn_forward_tiles(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d,
                                         ctypes.byref(ov), stream), "attn_forward_tiles")
     return o
@@ -248,7 +251,7 @@ def forward_host(q_host, k_host, v_host, o_host, dev_scratch):
     stream = torch.cuda.current_stream(dev_scratch.device).cuda_stream
     with torch.cuda.device(dev):
         t = plan(_device_desc(dev), B, H, L, d)
-        if t.feasible and t.kv_splits > 1:
+        if t.feasible and t.ctas > t.tiles:
             ensure_workspace(dev, workspace_bytes(t, B, H, L, d))
         _check(lib().attn_forward_host(q_host.data_ptr(), k_host.data_ptr(), v_host.data_ptr(), o_host.data_ptr(),
                                        B, H, L, d, dev_scratch.data_ptr(), dev_scratch.numel(), stream),

@@ -12,6 +12,7 @@
 
 #include "attn.h"
 #include "attn_kernels.cuh"
+#include "attn_plan_internal.h"
 
 namespace {
 
@@ -126,17 +127,19 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   p.L = L;
   p.q_tiles = (L + NQ * attn::kSub - 1) / (NQ * attn::kSub);
   p.n_steps = L / TKV;
-  p.kv_splits = t.kv_splits;
+  p.tiles = BH * p.q_tiles;
   p.stages = t.kv_stages;
   p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
+  p.o = reinterpret_cast<__nv_bfloat16*>(o);
   p.counters = reinterpret_cast<unsigned int*>(ws);                   // head of the workspace
   p.ws = ws ? ws + attn::kCounterBytes / sizeof(float) : nullptr;    // partial results follow
-  if (t.kv_splits > 1 && (size_t)BH * p.q_tiles * NQ > attn::kCounterBytes / sizeof(unsigned int))
-    return ATTN_ERR_BAD_TILES;
+  const int grid = t.ctas;
+  // one CTA per Q tile at least (several whole tiles per CTA are not supported), one KV step per CTA at least
+  if (grid < p.tiles || (long long)grid > (long long)p.tiles * p.n_steps) return ATTN_ERR_BAD_TILES;
+  if (grid > p.tiles && (size_t)p.tiles * NQ > attn::kCounterBytes / sizeof(unsigned int)) return ATTN_ERR_BAD_TILES;
   const int smem = SM::total(t.kv_stages);
   auto kern = attn::attn_fwd_kernel<D, TKV, NQ>;
   ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  const int grid = BH * p.q_tiles * t.kv_splits;
   kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
   ATTN_CUDA_TRY(cudaGetLastError());
   t_launch_count = 1;
@@ -181,13 +184,22 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
     if (t.kv_stages < 2 || t.kv_stages > max_stages) return ATTN_ERR_BAD_TILES;
     t.tile_q = t.n_q * 128;
     t.tiles = B * H * ((L + t.tile_q - 1) / t.tile_q);
-    if (ovr->kv_splits > 0) t.kv_splits = ovr->kv_splits;
-    if (t.kv_splits < 1 || t.kv_splits > L / t.tile_kv) return ATTN_ERR_BAD_TILES;
-    t.ctas = t.tiles * t.kv_splits;
+    // grid: ctas if given, else kv_splits CTAs per Q tile if given, else the planner's occupancy rule
+    // re-applied to the overridden tile shape
+    const int steps = L / t.tile_kv;
+    if (ovr->ctas > 0) {
+      t.ctas = ovr->ctas;
+    } else if (ovr->kv_splits > 0) {
+      t.ctas = t.tiles * ovr->kv_splits;
+    } else {
+      t.ctas = attn_internal::grid_size(st->desc, t.tiles, steps);
+    }
+    t.kv_splits = (t.ctas + t.tiles - 1) / t.tiles;
+    if (t.ctas < t.tiles || (long long)t.ctas > (long long)t.tiles * (L / t.tile_kv)) return ATTN_ERR_BAD_TILES;
     t.smem_bytes = q_bytes + t.kv_stages * stage + 3072;
   }
   float* ws = nullptr;
-  if (t.kv_splits > 1) {
+  if (t.ctas > t.tiles) {
     const size_t need = attn_workspace_bytes(&t, B, H, L, d);
     std::lock_guard<std::mutex> lk(g_mu);
     if (!st->ws || st->ws_bytes < need) return ATTN_ERR_NEED_WORKSPACE;
@@ -341,7 +353,7 @@ extern "C" int attn_forward_static_scratch(const void* q, const void* k, const v
   void* scratch = nullptr;
   if ((rc = static_scratch_address(&scratch)) != ATTN_OK) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (t.kv_splits > 1) {
+  if (t.ctas > t.tiles) {
     if (attn_workspace_bytes(&t, B, H, L, d) > (size_t)ATTN_STATIC_SCRATCH_BYTES) return ATTN_ERR_SCRATCH_LIMIT;
     // the array keeps the previous call's contents: the arrival counters must start at zero
     ATTN_CUDA_TRY(cudaMemsetAsync(scratch, 0, attn::kCounterBytes, stream));
@@ -374,6 +386,14 @@ extern "C" int attn_last_device_status(void* cuda_stream, uint32_t* detail) {
 extern "C" int attn_debug_read_trace(long long* out) {
   ATTN_CUDA_TRY(cudaDeviceSynchronize());
   ATTN_CUDA_TRY(cudaMemcpyFromSymbol(out, attn::g_attn_trace, sizeof(long long) * 5 * 16 * 8));
+  return ATTN_OK;
+}
+#endif
+
+#ifdef ATTN_TRACE
+extern "C" int attn_debug_read_cta_times(unsigned long long* out, int n) {
+  ATTN_CUDA_TRY(cudaDeviceSynchronize());
+  ATTN_CUDA_TRY(cudaMemcpyFromSymbol(out, attn::g_attn_cta_times, sizeof(unsigned long long) * 2 * n));
   return ATTN_OK;
 }
 #endif

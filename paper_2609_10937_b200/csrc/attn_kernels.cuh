@@ -20,6 +20,8 @@
 // in g_attn_dev_status, raises a CTA-wide abort flag and all roles drain.
 #pragma once
 
+#include <cuda_bf16.h>
+
 #include "ptx_sm100.cuh"
 
 namespace attn {
@@ -46,9 +48,25 @@ __device__ long long g_attn_trace[5][16][8];
     if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (step) >= kTraceStep0 && (step) < kTraceStep0 + 16) \
       g_attn_trace[role_slot][(step) - kTraceStep0][ev] = clock64();                            \
   } while (0)
+__device__ unsigned long long g_attn_cta_times[4096][2];
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define ATTN_TRACE_CTA(which)                                                  \
+  do {                                                                         \
+    if (threadIdx.x == 0 && blockIdx.x < 4096) g_attn_cta_times[blockIdx.x][which] = global_timer_ns(); \
+  } while (0)
+#define ATTN_TRACE_MARK(ev)                                                    \
+  do {                                                                         \
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) g_attn_trace[4][ev >> 3][ev & 7] = clock64(); \
+  } while (0)
 #else
 constexpr int kTraceStep0 = 0;
 #define ATTN_TRACE_EVENT(role_slot, step, ev) do {} while (0)
+#define ATTN_TRACE_MARK(ev) do {} while (0)
+#define ATTN_TRACE_CTA(which) do {} while (0)
 #endif
 
 __device__ __noinline__ void report_timeout(uint32_t info) {
@@ -137,13 +155,39 @@ __device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint3
 struct FwdParams {
   int L;                   // sequence length
   int q_tiles;             // Q tiles per head = ceil(L / (NQ*128))
-  int n_steps;             // KV steps per head = L / TKV
-  int kv_splits;           // CTAs per Q tile along the key axis
+  int n_steps;             // KV steps per Q tile = L / TKV
+  int tiles;               // Q tiles in the whole problem = B * H * q_tiles
   int stages;              // ring depth
   float scale_log2;        // log2(e) / sqrt(d)
-  float* ws;               // partial results when kv_splits > 1
+  __nv_bfloat16* o;        // output, written directly by the CTA that merges a shared Q tile
+  float* ws;               // partial results of Q tiles shared by several CTAs
   unsigned int* counters;  // one arrival counter per (Q tile, sub-tile); zero between launches
 };
+
+// Work decomposition.  The problem is a line of tiles * n_steps units (Q tile major, KV step minor);
+// CTA c of G owns units [c*T/G, (c+1)*T/G).  With G == tiles every CTA owns exactly one whole Q tile;
+// with G > tiles the ranges are balanced regardless of tile boundaries, a CTA's range may straddle
+// one boundary (two segments), and Q tiles covered by several CTAs are merged by the last to finish.
+__device__ __forceinline__ long long range_begin(long long c, long long T, long long G) { return (c * T) / G; }
+struct Segment { int tile, j0, j1, n, bh, q_row0, seg; };
+// Next piece of the unit range [u, u_hi) that lies inside one Q tile; advances u and the segment counter.
+__device__ __forceinline__ bool next_segment(long long& u, long long u_hi, int& seg_ctr, int n_steps, int q_tiles,
+                                             int tile_rows, Segment& sg) {
+  if (u >= u_hi) return false;
+  sg.tile = (int)(u / n_steps);
+  sg.j0 = (int)(u % n_steps);
+  const long long left = u_hi - u;
+  sg.j1 = (left < (long long)(n_steps - sg.j0)) ? sg.j0 + (int)left : n_steps;
+  sg.n = sg.j1 - sg.j0;
+  sg.bh = sg.tile / q_tiles;
+  sg.q_row0 = (sg.tile % q_tiles) * tile_rows;
+  sg.seg = seg_ctr++;
+  u += sg.n;
+  return true;
+}
+__device__ __forceinline__ int cta_of_unit(long long u, long long T, long long G) {
+  return (int)(((u + 1) * G - 1) / T);
+}
 
 // Shared-memory footprint helpers (host and device agree through these).
 template <int D, int TKV, int NQ>
@@ -170,6 +214,8 @@ struct FwdMisc {               // lives in the last 3072 bytes of dynamic shared
   uint64_t o_full[2];
   uint64_t alpha_full[2];
   uint64_t epi_sync[2];        // softmax warpgroup rendezvous in the epilogue
+  uint64_t q_empty;            // every product that reads the Q tile of a segment has finished
+  uint64_t o_free[2];          // the epilogue of a segment has read its O accumulator
   uint64_t dbg_bar[2];         // trace builds only: completion of the first half of P V
   uint32_t ticket[2];          // arrival order of this CTA among the splits of its Q sub-tile
   uint32_t tmem_slot;
@@ -303,19 +349,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
-  // Work assignment: split fastest, then Q tile, then head, so that CTAs of one
-  // head are neighbours in launch order and share K/V through L2.
+  // Work assignment (see range_begin): consecutive CTAs work on neighbouring key ranges of the same
+  // head, so K/V are shared through L2.
   const int cta = blockIdx.x;
-  const int split = cta % p.kv_splits;
-  const int tile = cta / p.kv_splits;
-  const int q_tile = tile % p.q_tiles;
-  const int bh = tile / p.q_tiles;
-  const int j0 = (int)(((long long)split * p.n_steps) / p.kv_splits);
-  const int j1 = (int)(((long long)(split + 1) * p.n_steps) / p.kv_splits);
-  const int n = j1 - j0;
-  const int q_row0 = q_tile * NQ * kSub;
+  const long long G = gridDim.x;
+  const long long T = (long long)p.tiles * p.n_steps;
+  const long long u_lo = range_begin(cta, T, G), u_hi = range_begin(cta + 1, T, G);
 
+  ATTN_TRACE_CTA(0);
   if (threadIdx.x == 0) {
+    ATTN_TRACE_MARK(0);
     misc->abort_flag = 0;
     if (smem_base & 1023u) {                 // swizzled tiles need 1024-byte alignment
       report_timeout(wait_info(kRoleLoad, 0, 0xFFFF));
@@ -334,7 +377,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(smem_u32(&misc->alpha_full[i]), kSub);
       mbar_init(smem_u32(&misc->epi_sync[i]), kSub);
       mbar_init(smem_u32(&misc->dbg_bar[i]), 1);
+      mbar_init(smem_u32(&misc->o_free[i]), kSub);
     }
+    mbar_init(smem_u32(&misc->q_empty), 1);
     fence_mbar_init();
     prefetch_tmap(&tm_q);
     prefetch_tmap(&tm_k);
@@ -349,8 +394,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = misc->tmem_slot;
-  const bool run = (*abort_flag == 0) && n > 0;
+  const bool run = (*abort_flag == 0) && u_hi > u_lo;
+  if (threadIdx.x == 0) ATTN_TRACE_MARK(1);
 
+  // Every role walks the same list of segments (see next_segment); `g` counts KV steps over all
+  // segments of this CTA and gives the parity of the per-step barriers.
   if (warp < 4 * NQ) {
     // ===================================================== softmax warpgroup
     setmaxnreg_inc<(NQ == 2) ? 192 : 232>();
@@ -363,84 +411,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t bar_p = smem_u32(&misc->p_full[i]);
     const uint32_t bar_h = smem_u32(&misc->p_half[i]);
     const uint32_t bar_a = smem_u32(&misc->alpha_full[i]);
+    const uint32_t bar_e = smem_u32(&misc->epi_sync[i]);
     const float scale = p.scale_log2;
     const ExpConsts ek = make_exp_consts(scale);
-    float m_run = -INFINITY, delta = 0.f;
-    bool ok = run;
-    for (int jj = 0; ok && jj < n; ++jj) {
-      if (!wait_bar_warp(bar_s, jj & 1, abort_flag, wait_info(kRoleSoftmax, kBarSFull, jj))) { ok = false; break; }
-      tc_fence_after();
-      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 0);
-      uint32_t s[TKV];
-      // load the row in two halves: the maximum of the first half is taken while the second is in flight
-#pragma unroll
-      for (int c = 0; c < NCH / 2; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-#pragma unroll
-      for (int c = 0; c < NCH / 2; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-#pragma unroll
-      for (int c = NCH / 2; c < NCH; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-      const float mx_a = fmaxf(fmaxf(chain_max<0, TKV / 8>(s), chain_max<TKV / 8, TKV / 4>(s)),
-                               fmaxf(chain_max<TKV / 4, 3 * TKV / 8>(s), chain_max<3 * TKV / 8, TKV / 2>(s)));
-#pragma unroll
-      for (int c = NCH / 2; c < NCH; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 1);
-      const float mx_b = fmaxf(fmaxf(chain_max<TKV / 2, 5 * TKV / 8>(s), chain_max<5 * TKV / 8, 3 * TKV / 4>(s)),
-                               fmaxf(chain_max<3 * TKV / 4, 7 * TKV / 8>(s), chain_max<7 * TKV / 8, TKV>(s)));
-      const float mx = fmaxf(mx_a, mx_b);
-      // Lazy rescale.  The reference maximum m_run moves (and O, delta are rescaled by alpha) only
-      //  (a) when the row maximum grew by more than kRescaleThreshold (log2 units), which bounds
-      //      P = exp2(s - m_run) by 2^threshold, or
-      //  (b) when the new maximum is a dominant key: its weight 2^gap is more than 1/16 of the
-      //      running denominator.  Then P of that key is exactly 1 and carries no bf16 rounding
-      //      error; a stale reference would put the rounding error of the heaviest weight on the
-      //      whole row.  For flat score distributions (b) stops firing after the first few tiles.
-      // Otherwise the reference stays stale, which changes nothing in exact arithmetic because
-      // delta and O carry the same factor.  First step: m_run = -inf, gap = +inf, alpha = 0.
-      const float m_cand = fmaxf(m_run, mx * scale);
-      const float gap = m_cand - m_run;
-      const float shrink = ex2_approx(-gap);             // 2^-gap: the rescale factor if the reference moves
-      const bool move = (gap > kRescaleThreshold) || (gap > 0.f && kDominanceFactor > delta * shrink);
-      const float m_new = move ? m_cand : m_run;
-      const float alpha = move ? shrink : 1.0f;
-      misc->alpha[i][jj & 1][row] = alpha;
-      mbar_arrive(bar_a);
-      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 2);
-      const uint64_t neg_m2 = pack_f32x2(-m_new, -m_new);
-      uint64_t sum_a = 0ull, sum_b = 0ull;               // packed (0.f, 0.f)
-      uint32_t pk[16];
-      // first half of the row: the second product may start on it while the rest is computed
-#pragma unroll
-      for (int c = 0; c < NCH / 2; ++c) {
-        exp_chunk<kPoly>(&s[c * 32], ek, neg_m2, sum_a, pk);
-        tmem_st16(s_tmem + c * 16, pk);                  // P aliases the front of the S buffer
-      }
-      uint32_t pk2[16];
-      exp_chunk<kPoly>(&s[(NCH / 2) * 32], ek, neg_m2, sum_b, pk2);
-      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 3);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_p);
-      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 4);
-      tmem_st16(s_tmem + (NCH / 2) * 16, pk2);
-#pragma unroll
-      for (int c = NCH / 2 + 1; c < NCH; ++c) {
-        exp_chunk<kPoly>(&s[c * 32], ek, neg_m2, sum_b, pk);
-        tmem_st16(s_tmem + c * 16, pk);
-      }
-      float sa0, sa1, sb0, sb1;
-      unpack_f32x2(sum_a, sa0, sa1);
-      unpack_f32x2(sum_b, sb0, sb1);
-      const float sum = sa0 + sa1, sum2 = sb0 + sb1;
-      delta = delta * alpha + (sum + sum2);
-      m_run = m_new;
-      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 5);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_h);
-      if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, jj, 6);
-    }
-    // ------------------------------------------------------------- epilogue
-    const uint32_t bar_e = smem_u32(&misc->epi_sync[i]);
+    const size_t per_sub = ws_floats_per_sub(D);
     uint32_t ep_phase = 0;
     auto wg_sync = [&](uint32_t tag) -> bool {          // all 128 threads of this warpgroup, bounded
       mbar_arrive(bar_e);
@@ -448,87 +422,109 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       ep_phase ^= 1u;
       return r;
     };
-    if (ok) ok = wait_bar_warp(smem_u32(&misc->o_full[i]), (n - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, n));
+    bool ok = run;
+    uint32_t g = 0;
     if (ok) {
-      tc_fence_after();
-      const bool direct = (p.kv_splits == 1);
-      bool do_store = direct;
-      float inv = 1.0f / delta;
-      float m_all = 0.f;
-      const size_t per_sub = ws_floats_per_sub(D);
-      const float* tile_ws = p.ws + ((size_t)tile * p.kv_splits * NQ + i) * per_sub;   // split 0 of this sub-tile
-      const size_t split_stride = (size_t)NQ * per_sub;
-      if (!direct) {
-        // un-normalised partial (O, m, delta) of this key range
-        float* ws = p.ws + ((size_t)cta * NQ + i) * per_sub;
+      long long u = u_lo;
+      int seg_ctr = 0;
+      Segment sg;
+      while (ok && next_segment(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, NQ * kSub, sg)) {
+        const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
+        (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
+      float m_run = -INFINITY, delta = 0.f;
+      for (int jj = 0; ok && jj < n; ++jj, ++g) {
+        if (!wait_bar_warp(bar_s, g & 1, abort_flag, wait_info(kRoleSoftmax, kBarSFull, g))) { ok = false; break; }
+        tc_fence_after();
+        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 0);
+        if (warp == 0 && g == 0) ATTN_TRACE_MARK(2);
+        uint32_t s[TKV];
+        // load the row in two halves: the maximum of the first half is taken while the second is in flight
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(o_tmem + c * 32, r);
+        for (int c = 0; c < NCH / 2; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
 #pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            float4 v4 = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]),
-                                    __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
-            reinterpret_cast<float4*>(ws)[(size_t)(c * 8 + g) * kSub + row] = v4;
-          }
+        for (int c = 0; c < NCH / 2; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+#pragma unroll
+        for (int c = NCH / 2; c < NCH; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+        const float mx_a = fmaxf(fmaxf(chain_max<0, TKV / 8>(s), chain_max<TKV / 8, TKV / 4>(s)),
+                                 fmaxf(chain_max<TKV / 4, 3 * TKV / 8>(s), chain_max<3 * TKV / 8, TKV / 2>(s)));
+#pragma unroll
+        for (int c = NCH / 2; c < NCH; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 1);
+        const float mx_b = fmaxf(fmaxf(chain_max<TKV / 2, 5 * TKV / 8>(s), chain_max<5 * TKV / 8, 3 * TKV / 4>(s)),
+                                 fmaxf(chain_max<3 * TKV / 4, 7 * TKV / 8>(s), chain_max<7 * TKV / 8, TKV>(s)));
+        const float mx = fmaxf(mx_a, mx_b);
+        // Lazy rescale.  The reference maximum m_run moves (and O, delta are rescaled by alpha) only
+        //  (a) when the row maximum grew by more than kRescaleThreshold (log2 units), which bounds
+        //      P = exp2(s - m_run) by 2^threshold, or
+        //  (b) when the new maximum is a dominant key: its weight 2^gap is more than 1/16 of the
+        //      running denominator.  Then P of that key is exactly 1 and carries no bf16 rounding
+        //      error; a stale reference would put the rounding error of the heaviest weight on the
+        //      whole row.  For flat score distributions (b) stops firing after the first few tiles.
+        // Otherwise the reference stays stale, which changes nothing in exact arithmetic because
+        // delta and O carry the same factor.  First step: m_run = -inf, gap = +inf, alpha = 0.
+        const float m_cand = fmaxf(m_run, mx * scale);
+        const float gap = m_cand - m_run;
+        const float shrink = ex2_approx(-gap);             // 2^-gap: the rescale factor if the reference moves
+        const bool move = (gap > kRescaleThreshold) || (gap > 0.f && kDominanceFactor > delta * shrink);
+        const float m_new = move ? m_cand : m_run;
+        const float alpha = move ? shrink : 1.0f;
+        misc->alpha[i][g & 1][row] = alpha;
+        mbar_arrive(bar_a);
+        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 2);
+        const uint64_t neg_m2 = pack_f32x2(-m_new, -m_new);
+        uint64_t sum_a = 0ull, sum_b = 0ull;               // packed (0.f, 0.f)
+        uint32_t pk[16];
+        // first half of the row: the second product may start on it while the rest is computed
+#pragma unroll
+        for (int c = 0; c < NCH / 2; ++c) {
+          exp_chunk<kPoly>(&s[c * 32], ek, neg_m2, sum_a, pk);
+          tmem_st16(s_tmem + c * 16, pk);                  // P aliases the front of the S buffer
         }
-        ws[(size_t)kSub * D + row] = m_run;
-        ws[(size_t)kSub * D + kSub + row] = delta;
-        __threadfence();
-        ok = wg_sync(1);
-        if (ok) {
-          if (row == 0) misc->ticket[i] = atomicAdd(&p.counters[tile * NQ + i], 1u);
-          ok = wg_sync(2);
+        uint32_t pk2[16];
+        exp_chunk<kPoly>(&s[(NCH / 2) * 32], ek, neg_m2, sum_b, pk2);
+        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 3);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_p);
+        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 4);
+        tmem_st16(s_tmem + (NCH / 2) * 16, pk2);
+#pragma unroll
+        for (int c = NCH / 2 + 1; c < NCH; ++c) {
+          exp_chunk<kPoly>(&s[c * 32], ek, neg_m2, sum_b, pk);
+          tmem_st16(s_tmem + c * 16, pk);
         }
-        if (ok) {
-          do_store = (*reinterpret_cast<volatile uint32_t*>(&misc->ticket[i]) == (uint32_t)(p.kv_splits - 1));
-          if (do_store) {
-            // Last CTA of this Q sub-tile to finish: merge all splits in ascending order
-            // (the merge operator of the online softmax), independent of arrival order.
-            if (row == 0) p.counters[tile * NQ + i] = 0u;
-            __threadfence();
-            m_all = -INFINITY;
-            for (int sp = 0; sp < p.kv_splits; ++sp)
-              m_all = fmaxf(m_all, __ldcg(tile_ws + sp * split_stride + (size_t)kSub * D + row));
-            float d_all = 0.f;
-            for (int sp = 0; sp < p.kv_splits; ++sp) {
-              const float* b = tile_ws + sp * split_stride + (size_t)kSub * D;
-              d_all += __ldcg(b + kSub + row) * exp2f(__ldcg(b + row) - m_all);
-            }
-            inv = 1.0f / d_all;
-          }
-        }
+        float sa0, sa1, sb0, sb1;
+        unpack_f32x2(sum_a, sa0, sa1);
+        unpack_f32x2(sum_b, sb0, sb1);
+        delta = delta * alpha + ((sa0 + sa1) + (sb0 + sb1));
+        m_run = m_new;
+        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 5);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_h);
+        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 6);
       }
-      if (ok && do_store) {
+      // ----------------------------------------------------- end of segment
+      if (warp == 0) ATTN_TRACE_MARK(3);
+      if (ok) ok = wait_bar_warp(smem_u32(&misc->o_full[i]), (g - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, g));
+      if (!ok) break;
+      tc_fence_after();
+      if (warp == 0) ATTN_TRACE_MARK(4);
+      if (j0 == 0 && j1 == p.n_steps) {
+        // The whole Q tile was processed here: normalise and store through shared memory (TMA).
+        const float inv = 1.0f / delta;
         const uint32_t stage_out = q_smem + i * (kSub * D * 2);   // Q sub-tile is dead: reuse it
 #pragma unroll 1
         for (int c = 0; c < D / 32; ++c) {
+          uint32_t r[32];
           float val[32];
-          if (direct) {
-            uint32_t r[32];
-            tmem_ld32(o_tmem + c * 32, r);
+          tmem_ld32(o_tmem + c * 32, r);
 #pragma unroll
-            for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(r[k]) * inv;
-          } else {
-#pragma unroll
-            for (int k = 0; k < 32; ++k) val[k] = 0.f;
-            for (int sp = 0; sp < p.kv_splits; ++sp) {
-              const float* b = tile_ws + sp * split_stride;
-              const float w = exp2f(__ldcg(b + (size_t)kSub * D + row) - m_all);
-#pragma unroll
-              for (int g = 0; g < 8; ++g) {
-                const float4 v4 = __ldcg(reinterpret_cast<const float4*>(b) + (size_t)(c * 8 + g) * kSub + row);
-                val[g * 4 + 0] += w * v4.x;
-                val[g * 4 + 1] += w * v4.y;
-                val[g * 4 + 2] += w * v4.z;
-                val[g * 4 + 3] += w * v4.w;
-              }
-            }
-#pragma unroll
-            for (int k = 0; k < 32; ++k) val[k] *= inv;
-          }
+          for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(r[k]) * inv;
           stage_row_chunk(stage_out, c, row, val);
         }
+        tc_fence_before();
+        mbar_arrive(smem_u32(&misc->o_free[i]));             // O may be overwritten by the next segment
         fence_proxy_async_smem();
         ok = wg_sync(3);
         if (ok && (warp & 3) == 0 && lane == 0) {
@@ -538,6 +534,103 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tma_store_commit();
           tma_store_wait_read();
         }
+      } else {
+        // Part of a Q tile: un-normalised partial (O, m, delta) of this key range into slot cta + tile.
+        float* ws = p.ws + ((size_t)(cta + tile) * NQ + i) * per_sub;
+        {
+          uint32_t r[D];
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) tmem_ld32_nowait(o_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[c * 32]));
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&r[c * 32]));
+#pragma unroll
+          for (int gq = 0; gq < D / 4; ++gq) {
+            float4 v4 = make_float4(__uint_as_float(r[gq * 4]), __uint_as_float(r[gq * 4 + 1]),
+                                    __uint_as_float(r[gq * 4 + 2]), __uint_as_float(r[gq * 4 + 3]));
+            reinterpret_cast<float4*>(ws)[(size_t)gq * kSub + row] = v4;
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(smem_u32(&misc->o_free[i]));             // O may be overwritten by the next segment
+        ws[(size_t)kSub * D + row] = m_run;
+        ws[(size_t)kSub * D + kSub + row] = delta;
+        __threadfence();
+        if (warp == 0) ATTN_TRACE_MARK(5);
+        ok = wg_sync(1);
+        if (ok) {
+          if (row == 0) misc->ticket[i] = atomicAdd(&p.counters[tile * NQ + i], 1u);
+          ok = wg_sync(2);
+        }
+        if (!ok) break;
+        // CTAs that share this Q tile: those whose ranges meet [tile*n_steps, (tile+1)*n_steps)
+        if (warp == 0) ATTN_TRACE_MARK(6);
+        const int c_first = cta_of_unit((long long)tile * p.n_steps, T, G);
+        const int c_last = cta_of_unit((long long)(tile + 1) * p.n_steps - 1, T, G);
+        if (*reinterpret_cast<volatile uint32_t*>(&misc->ticket[i]) == (uint32_t)(c_last - c_first)) {
+          // Last one to finish: merge all parts in ascending key order (the merge operator of the
+          // online softmax), independent of arrival order, and write the rows of this sub-tile.
+          if (row == 0) p.counters[tile * NQ + i] = 0u;
+          __threadfence();
+          const float* part0 = p.ws + ((size_t)(c_first + tile) * NQ + i) * per_sub;
+          const size_t part_stride = (size_t)NQ * per_sub;
+          const int parts = c_last - c_first + 1;
+          float m_all = -INFINITY;
+#pragma unroll 4
+          for (int sp = 0; sp < parts; ++sp)
+            m_all = fmaxf(m_all, __ldcg(part0 + sp * part_stride + (size_t)kSub * D + row));
+          // whole output row accumulated in registers: per part all loads are independent and in flight together
+          float val[D];
+#pragma unroll
+          for (int k = 0; k < D; ++k) val[k] = 0.f;
+          float d_all = 0.f;
+          for (int sp = 0; sp < parts; ++sp) {
+            const float* b = part0 + sp * part_stride;
+            const float w = exp2f(__ldcg(b + (size_t)kSub * D + row) - m_all);
+            d_all += __ldcg(b + (size_t)kSub * D + kSub + row) * w;
+#pragma unroll
+            for (int gq = 0; gq < D / 4; ++gq) {
+              const float4 v4 = __ldcg(reinterpret_cast<const float4*>(b) + (size_t)gq * kSub + row);
+              val[gq * 4 + 0] += w * v4.x;
+              val[gq * 4 + 1] += w * v4.y;
+              val[gq * 4 + 2] += w * v4.z;
+              val[gq * 4 + 3] += w * v4.w;
+            }
+          }
+          const float inv = 1.0f / d_all;
+#pragma unroll
+          for (int k = 0; k < D; ++k) val[k] *= inv;
+          if (u >= u_hi) {
+            // last segment of this CTA: the Q buffer is dead, store through shared memory (TMA)
+            const uint32_t stage_out = q_smem + i * (kSub * D * 2);
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) stage_row_chunk(stage_out, c, row, *reinterpret_cast<float(*)[32]>(&val[c * 32]));
+            fence_proxy_async_smem();
+            ok = wg_sync(3);
+            if (ok && (warp & 3) == 0 && lane == 0) {
+#pragma unroll
+              for (int c = 0; c < KCH; ++c)
+                tma_store_3d(&tm_o, stage_out + c * (kSub * 128), c * 64, q_row0 + i * kSub, bh);
+              tma_store_commit();
+              tma_store_wait_read();
+            }
+          } else {
+            // another segment follows and its Q tile may already be arriving: store from registers
+            const int grow = q_row0 + i * kSub + row;
+            if (grow < p.L) {
+              uint4* orow = reinterpret_cast<uint4*>(p.o + ((size_t)bh * p.L + grow) * D);
+#pragma unroll
+              for (int u4 = 0; u4 < D / 8; ++u4) {
+                uint4 w4;
+                w4.x = pack_bf16x2(val[u4 * 8 + 0], val[u4 * 8 + 1]);
+                w4.y = pack_bf16x2(val[u4 * 8 + 2], val[u4 * 8 + 3]);
+                w4.z = pack_bf16x2(val[u4 * 8 + 4], val[u4 * 8 + 5]);
+                w4.w = pack_bf16x2(val[u4 * 8 + 6], val[u4 * 8 + 7]);
+                orow[u4] = w4;
+              }
+            }
+          }
+        }
+      }
       }
     }
   } else if (warp >= 8 && warp < 12) {
@@ -546,40 +639,48 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     bool ok = run;
-    for (int jj = 0; ok && jj < n; ++jj) {
+    uint32_t g = 0;
+    if (ok) {
+      long long u = u_lo;
+      int seg_ctr = 0;
+      Segment sg;
+      while (ok && next_segment(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, NQ * kSub, sg)) {
+        const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
+        (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
+      for (int jj = 0; ok && jj < n; ++jj, ++g) {
 #pragma unroll
-      for (int i = 0; i < NQ; ++i) {
-        if (!wait_bar_warp(smem_u32(&misc->alpha_full[i]), jj & 1, abort_flag, wait_info(kRoleCorrection, kBarAlpha, jj))) {
-          ok = false;
-          break;
-        }
-        const float a = misc->alpha[i][jj & 1][row];
-        if (warp == 8) ATTN_TRACE_EVENT(2, jj, i * 4 + 0);
-        if (jj > 0) {
-          const bool need = __any_sync(0xffffffffu, a != 1.0f);
-          if (warp == 8 && need) ATTN_TRACE_EVENT(2, jj, i * 4 + 1);
-          if (need) {
-            if (!wait_bar_warp(smem_u32(&misc->o_full[i]), (jj - 1) & 1, abort_flag,
-                               wait_info(kRoleCorrection, kBarOFull, jj))) {
-              ok = false;
-              break;
-            }
-            tc_fence_after();
-            const uint32_t o_tmem = lane_base + O_COL0 + i * D;
-#pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-              uint32_t r[32];
-              tmem_ld32(o_tmem + c * 32, r);
-#pragma unroll
-              for (int k = 0; k < 32; ++k) r[k] = __float_as_uint(__uint_as_float(r[k]) * a);
-              tmem_st32(o_tmem + c * 32, r);
-            }
-            tmem_wait_st();
+        for (int i = 0; i < NQ; ++i) {
+          if (!wait_bar_warp(smem_u32(&misc->alpha_full[i]), g & 1, abort_flag, wait_info(kRoleCorrection, kBarAlpha, g))) {
+            ok = false;
+            break;
           }
-          tc_fence_before();
+          const float a = misc->alpha[i][g & 1][row];
+          if (jj > 0) {                                   // the first step of a segment starts O afresh
+            const bool need = __any_sync(0xffffffffu, a != 1.0f);
+            if (need) {
+              if (!wait_bar_warp(smem_u32(&misc->o_full[i]), (g - 1) & 1, abort_flag,
+                                 wait_info(kRoleCorrection, kBarOFull, g))) {
+                ok = false;
+                break;
+              }
+              tc_fence_after();
+              const uint32_t o_tmem = lane_base + O_COL0 + i * D;
+#pragma unroll
+              for (int c = 0; c < D / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(o_tmem + c * 32, r);
+#pragma unroll
+                for (int k = 0; k < 32; ++k) r[k] = __float_as_uint(__uint_as_float(r[k]) * a);
+                tmem_st32(o_tmem + c * 32, r);
+              }
+              tmem_wait_st();
+            }
+            tc_fence_before();
+          }
+          mbar_arrive(smem_u32(&misc->p_full[i]));
         }
-        mbar_arrive(smem_u32(&misc->p_full[i]));
-        if (warp == 8) ATTN_TRACE_EVENT(2, jj, i * 4 + 2);
+      }
+      if (!ok) break;
       }
     }
   } else if (warp == 12) {
@@ -590,26 +691,33 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // warpgroups half a step apart, so that one computes exponentials while the tensor pipe works
     // for the other.  (setmaxnreg is warpgroup-aligned: warps 12-15 request the same count.)
     setmaxnreg_dec<64>();
-    if (run) {
-      bool ok = wait_bar_warp(smem_u32(&misc->q_full), 0, abort_flag, wait_info(kRoleMma, kBarQ, 0));
-      int stage = 0;
-      uint32_t phase = 0;
-      auto advance = [&]() { if (++stage == p.stages) { stage = 0; phase ^= 1u; } };
-      if (ok) ok = wait_bar_warp(smem_u32(&misc->kv_full[stage]), phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 0));
-      if (ok) {
-        tc_fence_after();
-        if (elect_one()) {
+    bool ok = run;
+    uint32_t g = 0;
+    int stage = 0;
+    uint32_t phase = 0;
+    auto advance = [&]() { if (++stage == p.stages) { stage = 0; phase ^= 1u; } };
+    if (ok) {
+      long long u = u_lo;
+      int seg_ctr = 0;
+      Segment sg;
+      while (ok && next_segment(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, NQ * kSub, sg)) {
+        const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
+        (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
+      ok = wait_bar_warp(smem_u32(&misc->q_full), seg & 1, abort_flag, wait_info(kRoleMma, kBarQ, seg));
+      if (ok) ok = wait_bar_warp(smem_u32(&misc->kv_full[stage]), phase, abort_flag, wait_info(kRoleMma, kBarKvFull, g));
+      if (!ok) break;
+      tc_fence_after();
+      if (elect_one()) {
 #pragma unroll
-          for (int i = 0; i < NQ; ++i) {
-            issue_qk<D, TKV>(tmem_base + i * S_COLS, q_smem + i * (kSub * D * 2), ring_smem + stage * SM::kStageBytes);
-            umma_commit(smem_u32(&misc->s_full[i]));
-          }
-          umma_commit(smem_u32(&misc->kv_empty[stage]));
+        for (int i = 0; i < NQ; ++i) {
+          issue_qk<D, TKV>(tmem_base + i * S_COLS, q_smem + i * (kSub * D * 2), ring_smem + stage * SM::kStageBytes);
+          umma_commit(smem_u32(&misc->s_full[i]));
         }
-        __syncwarp();
-        advance();
+        umma_commit(smem_u32(&misc->kv_empty[stage]));
       }
-      for (int jj = 0; ok && jj < n; ++jj) {
+      __syncwarp();
+      advance();
+      for (int jj = 0; ok && jj < n; ++jj, ++g) {
         const int v_stage = stage;
         const uint32_t v_phase = phase;
         advance();
@@ -619,14 +727,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (more) advance();
         const uint32_t v_smem = ring_smem + v_stage * SM::kStageBytes;
         const uint32_t k_smem = ring_smem + k_stage * SM::kStageBytes;
-        if (!wait_bar_warp(smem_u32(&misc->kv_full[v_stage]), v_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 2 * jj + 1))) { ok = false; break; }
+        if (!wait_bar_warp(smem_u32(&misc->kv_full[v_stage]), v_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, g))) { ok = false; break; }
 #pragma unroll
         for (int i = 0; i < NQ; ++i) {
           const uint32_t s_acc = tmem_base + i * S_COLS;
           const uint32_t o_acc = tmem_base + O_COL0 + i * D;
-          if (!wait_bar_warp(smem_u32(&misc->p_full[i]), jj & 1, abort_flag, wait_info(kRoleMma, kBarPFull, jj))) { ok = false; break; }
+          if (!wait_bar_warp(smem_u32(&misc->p_full[i]), g & 1, abort_flag, wait_info(kRoleMma, kBarPFull, g))) { ok = false; break; }
+          if (jj == 0 && seg > 0) {
+            // the previous segment's epilogue must have read O before the first product overwrites it
+            if (!wait_bar_warp(smem_u32(&misc->o_free[i]), (seg - 1) & 1, abort_flag, wait_info(kRoleMma, kBarOFull, 0x8000 | seg))) { ok = false; break; }
+          }
           tc_fence_after();
-          ATTN_TRACE_EVENT(3, jj, i * 4 + 0);
+          ATTN_TRACE_EVENT(3, (int)g, i * 4 + 0);
           if (elect_one()) {
             issue_pv<D, TKV>(o_acc, s_acc, v_smem, jj > 0, TKV * 128, 1024, 0, TKV / 32);
 #ifdef ATTN_TRACE
@@ -634,12 +746,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #endif
           }
           __syncwarp();
-          ATTN_TRACE_EVENT(3, jj, i * 4 + 1);
-          if (!wait_bar_warp(smem_u32(&misc->p_half[i]), jj & 1, abort_flag, wait_info(kRoleMma, kBarPFull, 0x8000 | jj))) { ok = false; break; }
+          ATTN_TRACE_EVENT(3, (int)g, i * 4 + 1);
+          if (!wait_bar_warp(smem_u32(&misc->p_half[i]), g & 1, abort_flag, wait_info(kRoleMma, kBarPFull, 0x8000 | g))) { ok = false; break; }
           tc_fence_after();
-          ATTN_TRACE_EVENT(3, jj, i * 4 + 2);
+          ATTN_TRACE_EVENT(3, (int)g, i * 4 + 2);
           if (more && i == 0) {
-            if (!wait_bar_warp(smem_u32(&misc->kv_full[k_stage]), k_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, 2 * jj + 2))) { ok = false; break; }
+            if (!wait_bar_warp(smem_u32(&misc->kv_full[k_stage]), k_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, g))) { ok = false; break; }
             tc_fence_after();
           }
           if (elect_one()) {
@@ -650,80 +762,85 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               issue_qk<D, TKV>(s_acc, q_smem + i * (kSub * D * 2), k_smem);
               umma_commit(smem_u32(&misc->s_full[i]));
               if (i == NQ - 1) umma_commit(smem_u32(&misc->kv_empty[k_stage]));
+            } else if (i == NQ - 1) {
+              umma_commit(smem_u32(&misc->q_empty));       // every product that reads this Q tile is issued
             }
           }
           __syncwarp();
-          ATTN_TRACE_EVENT(3, jj, i * 4 + 3);
+          ATTN_TRACE_EVENT(3, (int)g, i * 4 + 3);
         }
+      }
+      if (!ok) break;
       }
     }
   } else if (warp == 13) {
     // ========================================================== TMA producer
     setmaxnreg_dec<64>();
     if (run && elect_one()) {
-      mbar_arrive_expect_tx(smem_u32(&misc->q_full), SM::kQBytes);
-#pragma unroll
-      for (int i = 0; i < NQ; ++i)
-#pragma unroll
-        for (int c = 0; c < KCH; ++c)
-          tma_load_3d(q_smem + i * (kSub * D * 2) + c * (kSub * 128), &tm_q, c * 64, q_row0 + i * kSub, bh,
-                      smem_u32(&misc->q_full));
       int stage = 0;
       uint32_t phase = 0;
       int issued = 0;
       bool ok = true;
-      for (int t = 0; t < 2 * n; ++t) {
-        if (!wait_bar(smem_u32(&misc->kv_empty[stage]), phase ^ 1u, abort_flag, wait_info(kRoleLoad, kBarKvEmpty, t))) { ok = false; break; }
-        const uint32_t bar = smem_u32(&misc->kv_full[stage]);
-        mbar_arrive_expect_tx(bar, SM::kStageBytes);
-        const CUtensorMap* tm = (t & 1) ? &tm_v : &tm_k;
-        const int kv_row = (j0 + (t >> 1)) * TKV;
-        const uint32_t dst = ring_smem + stage * SM::kStageBytes;
+      int q_loads = 0;
+      {
+      long long u = u_lo;
+      int seg_ctr = 0;
+      Segment sg;
+      while (ok && next_segment(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, NQ * kSub, sg)) {
+        const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
+        (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
+        if (seg > 0 &&
+            !wait_bar(smem_u32(&misc->q_empty), (seg - 1) & 1, abort_flag, wait_info(kRoleLoad, kBarQ, seg))) { ok = false; break; }
+        mbar_arrive_expect_tx(smem_u32(&misc->q_full), SM::kQBytes);
 #pragma unroll
-        for (int c = 0; c < KCH; ++c) tma_load_3d(dst + c * (TKV * 128), tm, c * 64, kv_row, bh, bar);
-        ++issued;
-        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
-      }
+        for (int i = 0; i < NQ; ++i)
+#pragma unroll
+          for (int c = 0; c < KCH; ++c)
+            tma_load_3d(q_smem + i * (kSub * D * 2) + c * (kSub * 128), &tm_q, c * 64, q_row0 + i * kSub, bh,
+                        smem_u32(&misc->q_full));
+        ++q_loads;
+        for (int t = 0; t < 2 * n; ++t) {
+          if (!wait_bar(smem_u32(&misc->kv_empty[stage]), phase ^ 1u, abort_flag, wait_info(kRoleLoad, kBarKvEmpty, t))) { ok = false; break; }
+          const uint32_t bar = smem_u32(&misc->kv_full[stage]);
+          mbar_arrive_expect_tx(bar, SM::kStageBytes);
+          const CUtensorMap* tm = (t & 1) ? &tm_v : &tm_k;
+          const int kv_row = (j0 + (t >> 1)) * TKV;
+          const uint32_t dst = ring_smem + stage * SM::kStageBytes;
+#pragma unroll
+          for (int c = 0; c < KCH; ++c) tma_load_3d(dst + c * (TKV * 128), tm, c * 64, kv_row, bh, bar);
+          ++issued;
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        }
+    }
       if (!ok) {
         // Drain: every copy this thread started must land before the CTA may exit.
         const int first = issued > p.stages ? issued - p.stages : 0;
         for (int t = first; t < issued; ++t) {
-          const int s = t % p.stages;
+          const int sidx = t % p.stages;
           const uint32_t ph = (uint32_t)(t / p.stages) & 1u;
           const long long t0 = clock64();
-          while (!mbar_try_wait(smem_u32(&misc->kv_full[s]), ph) && clock64() - t0 < kWaitLimitCycles) {}
+          while (!mbar_try_wait(smem_u32(&misc->kv_full[sidx]), ph) && clock64() - t0 < kWaitLimitCycles) {}
         }
-        const long long t0 = clock64();
-        while (!mbar_try_wait(smem_u32(&misc->q_full), 0) && clock64() - t0 < kWaitLimitCycles) {}
+        if (q_loads > 0) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(smem_u32(&misc->q_full), (uint32_t)(q_loads - 1) & 1u) && clock64() - t0 < kWaitLimitCycles) {}
+        }
       }
     }
   } else {
     setmaxnreg_dec<64>();
-#ifdef ATTN_TRACE
-    // completion times of the matrix products, observed by an otherwise idle warp
-    if (warp == 15 && lane == 0 && run && blockIdx.x == 0) {
-      for (int jj = 0; jj < n && jj < kTraceStep0 + 16; ++jj) {
-        for (int i = 0; i < NQ; ++i) {
-          if (!wait_bar(smem_u32(&misc->dbg_bar[i]), jj & 1, abort_flag, 0)) break;
-          ATTN_TRACE_EVENT(4, jj, i);          // overwrites the loader's K/V issue slots
-          if (!wait_bar(smem_u32(&misc->o_full[i]), jj & 1, abort_flag, 0)) break;
-          ATTN_TRACE_EVENT(4, jj, 2 + i * 2);
-          if (jj + 1 < n) {
-            if (!wait_bar(smem_u32(&misc->s_full[i]), (jj + 1) & 1, abort_flag, 0)) break;
-            ATTN_TRACE_EVENT(4, jj, 3 + i * 2);
-          }
-        }
-      }
-    }
-#endif
   }
-
+  if (warp == 0) ATTN_TRACE_MARK(7);
   tc_fence_before();
   __syncthreads();
   if (warp == 15) {
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
   }
+  if (threadIdx.x == 0) ATTN_TRACE_MARK(8);
+  ATTN_TRACE_CTA(1);
 }
 
 // ---------------------------------------------------------------------------

@@ -17,6 +17,7 @@
 #include <cstring>
 
 #include "attn.h"
+#include "attn_plan_internal.h"
 
 namespace {
 
@@ -29,6 +30,7 @@ constexpr int kMaxStages = 8;
 constexpr int kMinStages = 4;         // K_j, V_j and one of each in flight
 constexpr int kMinTileKv = 32;
 constexpr int kMinStepsPerSplit = 4;
+constexpr int kSegmentOverheadSteps = 3;  // Q load + first product + partial write/merge, in units of one KV step
 
 inline int floor_to(int x, int m) { return (x / m) * m; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -51,6 +53,29 @@ inline int pow2_ceil(int x) {
 inline int register_machine_regs(int t_q, int t_kv, int d, int simd) {
   return ceil_div(t_q * (2 * d + t_kv + 8), simd) + 16;
 }
+
+}  // namespace
+
+// Occupancy step of the derivation (shared with the tile-override path of the launcher).
+int attn_internal::grid_size(const attn_hw_desc& h, int tiles, int steps) {
+  if (tiles >= h.num_units) return tiles;
+  int k = h.num_units / tiles;
+  const int k_max = steps / kMinStepsPerSplit;
+  if (k > k_max) k = k_max;
+  if (k < 1) k = 1;
+  const int cost_uniform = ceil_div(steps, k) + kSegmentOverheadSteps;
+  const long long total = (long long)tiles * steps;
+  long long g = total / kMinStepsPerSplit;
+  if (g > h.num_units) g = h.num_units;
+  int ctas = tiles * k;
+  if (g > (long long)tiles * k) {
+    const int cost_balanced = (int)((total + g - 1) / g) + 2 * kSegmentOverheadSteps;
+    if (cost_balanced < cost_uniform) ctas = (int)g;
+  }
+  return ctas;
+}
+
+namespace {
 
 void plan_register_machine(const attn_hw_desc& h, int B, int H, int L, int d, attn_tiles* t) {
   // Local memory holds K_t and V_t together.
@@ -118,18 +143,19 @@ void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, attn_t
     if (tile_kv < kMinTileKv) { t->binding_constraint = ATTN_BIND_SMEM; return; }
   }
 
-  // 3. Occupancy: blocks against compute units; split the key axis when short.
+  // 3. Occupancy: blocks against compute units.  With fewer Q tiles than units the key axis is shared
+  //    out in one of two ways, whichever has the shorter critical path (counted in KV steps, a segment
+  //    start/finish costing kSegmentOverheadSteps):
+  //      uniform   k = floor(units / tiles) CTAs per Q tile, each one contiguous piece of its tile;
+  //      balanced  min(units, tiles*steps/kMinStepsPerSplit) CTAs with equal ranges of the
+  //                tiles*steps line, which may straddle one tile boundary (two pieces).
+  //    Q tiles shared by several CTAs are merged with the merge operator of the online softmax.
   const int tile_q = n_q * sub;
   const int tiles = B * H * ceil_div(L, tile_q);
   const int steps = ceil_div(L, tile_kv);
   const int under = tiles < h.num_units;
-  int kv_splits = 1;
-  if (under) {
-    int by_units = h.num_units / tiles;
-    int by_steps = steps / kMinStepsPerSplit;
-    kv_splits = by_units < by_steps ? by_units : by_steps;
-    if (kv_splits < 1) kv_splits = 1;
-  }
+  const int ctas = attn_internal::grid_size(h, tiles, steps);
+  const int kv_splits = ceil_div(ctas, tiles);
 
   t->feasible = 1;
   t->binding_constraint = binding;
@@ -145,7 +171,7 @@ void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, attn_t
   t->regs_softmax = regs_soft;
   t->threads = 128 * (n_q + 2);
   t->tiles = tiles;
-  t->ctas = tiles * kv_splits;
+  t->ctas = ctas;
   t->ctas_per_unit = (float)t->ctas / (float)h.num_units;
   const int waves = ceil_div(t->ctas, h.num_units);
   t->wave_efficiency = (float)((double)t->ctas / ((double)waves * h.num_units));
@@ -194,9 +220,9 @@ extern "C" int attn_plan(const attn_hw_desc* desc, int B, int H, int L, int d, a
 
 extern "C" size_t attn_workspace_bytes(const attn_tiles* t, int B, int H, int L, int d) {
   (void)B; (void)H; (void)L;
-  if (!t || !t->feasible || t->kv_splits <= 1 || t->n_q <= 0) return 0;
-  // 64 KB of arrival counters, then per CTA and sub-tile: 128 x d fp32 un-normalised
-  // output + 128 (m, delta) pairs.
+  if (!t || !t->feasible || t->ctas <= t->tiles || t->n_q <= 0) return 0;
+  // 64 KB of arrival counters, then one slot per (CTA, Q tile) piece -- at most ctas + tiles of
+  // them -- and sub-tile: 128 x d fp32 un-normalised output + 128 (m, delta) pairs.
   const size_t per_sub = (size_t)128 * (size_t)d * 4 + (size_t)128 * 2 * 4;
-  return (size_t)65536 + (size_t)t->ctas * (size_t)t->n_q * per_sub;
+  return (size_t)65536 + ((size_t)t->ctas + (size_t)t->tiles) * (size_t)t->n_q * per_sub;
 }

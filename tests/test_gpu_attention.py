@@ -132,6 +132,20 @@ def test_tile_variants_match_oracle(env, d, n_q, tile_kv, kv_stages, kv_splits):
     _run_and_compare(env, _case("variant", 1, 2, 1408, d, sigma_qk=math.sqrt(3.0)), run)
 
 
+@pytest.mark.parametrize("ctas", [12, 13, 17, 29, 64, 131])
+@pytest.mark.parametrize("d,n_q,tile_kv", [(128, 2, 128), (64, 2, 128), (128, 1, 64)])
+def test_balanced_key_ranges_any_grid_size(env, d, n_q, tile_kv, ctas):
+    """Grid sizes that cut the (Q tile, KV step) line at arbitrary places: ranges that straddle a tile
+    boundary (two segments per CTA), tiles shared by two to many CTAs, tiles owned by a single CTA."""
+    _, _, binding = env
+    case = _case("ranges", 1, 2, 1408, d, sigma_qk=math.sqrt(3.0))
+    tiles = 2 * math.ceil(1408 / (128 * n_q))
+    if ctas < tiles:
+        pytest.skip("fewer CTAs than Q tiles is not a supported launch")
+    run = lambda a, b, c: binding.forward_tiles(a, b, c, n_q=n_q, tile_kv=tile_kv, ctas=ctas)
+    _run_and_compare(env, case, run)
+
+
 def test_two_kernels_agree_and_runs_are_bitwise_reproducible(env):
     torch, _, binding = env
     case = _case("agree", 1, 4, 2048, 128)

@@ -119,8 +119,8 @@ def test_plan_argument_errors(binding):
 def test_workspace_bytes(binding):
     desc = binding.hw_desc_b200()
     t = binding.plan(desc, 1, 1, 16384, 128)
-    assert t.kv_splits == 2
-    assert binding.workspace_bytes(t, 1, 1, 16384, 128) == 65536 + t.ctas * 2 * (128 * 128 + 256) * 4
+    assert (t.tiles, t.ctas) == (64, 148)
+    assert binding.workspace_bytes(t, 1, 1, 16384, 128) == 65536 + (t.ctas + t.tiles) * 2 * (128 * 128 + 256) * 4
     t1 = binding.plan(desc, 4, 32, 4096, 128)
     assert binding.workspace_bytes(t1, 4, 32, 4096, 128) == 0
 
