@@ -1,0 +1,85 @@
+"""Small tile sweep around the closed-form default (measurement aid, not part of the hot path).
+
+    python -m paper_2609_10937_b200.sweep [--workload cfg3] [--iters 20]
+
+Times every compiled tile variant (n_q in {1, 2}, tile_kv in {64, 128}, ring depth default and
+default-1, grid sizes around the planner's choice) with CUDA events, an L2 flush between launches,
+and prints one JSON object: the default's time, the best point and default/best.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+import sys
+
+
+def main(argv=None):
+    import numpy as np
+    import torch
+
+    from . import binding, synth
+
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="cfg3")
+    ap.add_argument("--iters", type=int, default=20)
+    args = ap.parse_args(argv)
+    case = synth.CONFIGS[args.workload]
+    q, k, v = (torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).cuda() for x in synth.make_qkv(case, 0))
+    o = torch.empty_like(q)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    desc = binding.hw_desc_query(torch.cuda.current_device())
+    plan = binding.plan(desc, case.B, case.H, case.L, case.d)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(args.iters):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts)
+
+    default_ms = timed(lambda: binding.forward(q, k, v, o))
+    points = []
+    for n_q in (2, 1):
+        for tile_kv in (128, 64):
+            tiles = case.B * case.H * -(-case.L // (128 * n_q))
+            steps = case.L // tile_kv
+            grids = sorted({tiles, min(tiles * max(1, desc.num_units // tiles), tiles * steps),
+                            min(max(desc.num_units, tiles), tiles * steps)})
+            for stages_delta in (0, 1):
+                for ctas in grids:
+                    base = binding.plan(desc, case.B, case.H, case.L, case.d)
+                    q_bytes, stage = n_q * 128 * case.d * 2, tile_kv * case.d * 2
+                    max_stages = min(8, (desc.local_mem_bytes - q_bytes - 3072) // stage)
+                    stages = max_stages - stages_delta
+                    if stages < 2:
+                        continue
+                    kw = dict(n_q=n_q, tile_kv=tile_kv, kv_stages=stages, ctas=ctas)
+                    try:
+                        ms = timed(lambda: binding.forward_tiles(q, k, v, o, **kw))
+                    except binding.AttnError:
+                        continue
+                    points.append(dict(kw, ms=ms, tflops=case.flops / ms / 1e9))
+    best = min(points, key=lambda p: p["ms"])
+    out = {
+        "workload": args.workload,
+        "default": {"tile_q": plan.tile_q, "tile_kv": plan.tile_kv, "kv_stages": plan.kv_stages, "ctas": plan.ctas,
+                    "ms": default_ms, "tflops": case.flops / default_ms / 1e9},
+        "best": best,
+        "default_over_best_time": default_ms / best["ms"],
+        "points": sorted(points, key=lambda p: p["ms"]),
+    }
+    print(json.dumps(out))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
