@@ -19,7 +19,9 @@
  *     call returns.  attn_forward* are asynchronous on `cuda_stream`
  *     (a cudaStream_t passed as void*; NULL = the default stream) and never
  *     synchronise.
- *   - Supported shapes: d in {64, 128}, L a multiple of 128, B, H >= 1.
+ *   - Supported shapes: d in {64, 128}; any L >= 1 (a ragged last key tile is
+ *     masked with -inf, never zero-padded; the paper's boundary note in Section
+ *     "Online Softmax"), B, H >= 1.
  *   - Results are bitwise reproducible run to run (fixed merge order, no
  *     atomics on the output).
  */
@@ -36,7 +38,7 @@ extern "C" {
 typedef enum attn_status {
   ATTN_OK = 0,
   ATTN_ERR_INVALID_ARG = -1,       /* null pointer, non-positive size, bad struct_bytes   */
-  ATTN_ERR_UNSUPPORTED_SHAPE = -2, /* d not in {64,128} or L not a multiple of 128        */
+  ATTN_ERR_UNSUPPORTED_SHAPE = -2, /* d not in {64,128}, or B*H*L beyond the index range  */
   ATTN_ERR_MISALIGNED = -3,        /* a device pointer is not 16-byte aligned             */
   ATTN_ERR_ALIASING = -4,          /* o overlaps q, k or v                                */
   ATTN_ERR_INFEASIBLE_PLAN = -5,   /* no tile choice fits; see binding_constraint         */

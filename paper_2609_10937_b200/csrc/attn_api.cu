@@ -102,8 +102,8 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
 
 int check_args(const void* q, const void* k, const void* v, const void* o, int B, int H, int L, int d) {
   if (!q || !k || !v || !o || B <= 0 || H <= 0 || L <= 0 || d <= 0) return ATTN_ERR_INVALID_ARG;
-  if ((d != 64 && d != 128) || (L % 128) != 0) return ATTN_ERR_UNSUPPORTED_SHAPE;
-  if ((long long)B * H * (L / 128) > 0x3FFFFFFFLL) return ATTN_ERR_UNSUPPORTED_SHAPE;  // grid index range
+  if (d != 64 && d != 128) return ATTN_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)B * H * ((L + 127) / 128) > 0x3FFFFFFFLL) return ATTN_ERR_UNSUPPORTED_SHAPE;  // grid index range
   if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15u) return ATTN_ERR_MISALIGNED;
   const size_t bytes = (size_t)B * H * L * d * 2;
   if (overlaps(o, bytes, q, bytes) || overlaps(o, bytes, k, bytes) || overlaps(o, bytes, v, bytes))
@@ -126,7 +126,7 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   attn::FwdParams p;
   p.L = L;
   p.q_tiles = (L + NQ * attn::kSub - 1) / (NQ * attn::kSub);
-  p.n_steps = L / TKV;
+  p.n_steps = (L + TKV - 1) / TKV;
   p.tiles = BH * p.q_tiles;
   p.stages = t.kv_stages;
   p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
@@ -186,7 +186,7 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
     t.tiles = B * H * ((L + t.tile_q - 1) / t.tile_q);
     // grid: ctas if given, else kv_splits CTAs per Q tile if given, else the planner's occupancy rule
     // re-applied to the overridden tile shape
-    const int steps = L / t.tile_kv;
+    const int steps = (L + t.tile_kv - 1) / t.tile_kv;
     if (ovr->ctas > 0) {
       t.ctas = ovr->ctas;
     } else if (ovr->kv_splits > 0) {
@@ -195,7 +195,7 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
       t.ctas = attn_internal::grid_size(st->desc, t.tiles, steps);
     }
     t.kv_splits = (t.ctas + t.tiles - 1) / t.tiles;
-    if (t.ctas < t.tiles || (long long)t.ctas > (long long)t.tiles * (L / t.tile_kv)) return ATTN_ERR_BAD_TILES;
+    if (t.ctas < t.tiles || (long long)t.ctas > (long long)t.tiles * steps) return ATTN_ERR_BAD_TILES;
     t.smem_bytes = q_bytes + t.kv_stages * stage + 3072;
   }
   float* ws = nullptr;
@@ -223,7 +223,7 @@ int launch_simple(const void* q, const void* k, const void* v, void* o, int B, i
   const char* dbg = std::getenv("ATTN_SIMPLE_DEBUG_FLAGS");
   const int flags = dbg ? std::atoi(dbg) : 0;
   const float scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
-  dim3 grid(L / attn::kSub, BH);
+  dim3 grid((L + attn::kSub - 1) / attn::kSub, BH);
   kern<<<grid, 128, smem, stream>>>(tq, tk, tv, reinterpret_cast<__nv_bfloat16*>(o), L, scale_log2, scores_out, flags);
   ATTN_CUDA_TRY(cudaGetLastError());
   t_launch_count = 1;
@@ -406,7 +406,7 @@ extern "C" const char* attn_status_string(int status) {
   switch (status) {
     case ATTN_OK: return "ok";
     case ATTN_ERR_INVALID_ARG: return "invalid argument";
-    case ATTN_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (need d in {64,128} and L a multiple of 128)";
+    case ATTN_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (need d in {64,128})";
     case ATTN_ERR_MISALIGNED: return "device pointer not 16-byte aligned";
     case ATTN_ERR_ALIASING: return "output overlaps an input";
     case ATTN_ERR_INFEASIBLE_PLAN: return "no feasible tile plan";

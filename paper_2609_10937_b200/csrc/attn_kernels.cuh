@@ -169,6 +169,8 @@ struct FwdParams {
 // with G > tiles the ranges are balanced regardless of tile boundaries, a CTA's range may straddle
 // one boundary (two segments), and Q tiles covered by several CTAs are merged by the last to finish.
 __device__ __forceinline__ long long range_begin(long long c, long long T, long long G) { return (c * T) / G; }
+template <bool V>
+struct RaggedTag { static constexpr bool value = V; };
 struct Segment { int tile, j0, j1, n, bh, q_row0, seg; };
 // Next piece of the unit range [u, u_hi) that lies inside one Q tile; advances u and the segment counter.
 __device__ __forceinline__ bool next_segment(long long& u, long long u_hi, int& seg_ctr, int n_steps, int q_tiles,
@@ -415,6 +417,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const float scale = p.scale_log2;
     const ExpConsts ek = make_exp_consts(scale);
     const size_t per_sub = ws_floats_per_sub(D);
+    const int kv_tail = p.L % TKV;                     // valid keys in a ragged last KV tile (0: none ragged)
     uint32_t ep_phase = 0;
     auto wg_sync = [&](uint32_t tag) -> bool {          // all 128 threads of this warpgroup, bounded
       mbar_arrive(bar_e);
@@ -432,8 +435,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
       float m_run = -INFINITY, delta = 0.f;
-      for (int jj = 0; ok && jj < n; ++jj, ++g) {
-        if (!wait_bar_warp(bar_s, g & 1, abort_flag, wait_info(kRoleSoftmax, kBarSFull, g))) { ok = false; break; }
+      // One KV step of this sub-tile.  The ragged variant (last KV tile of a sequence whose length is
+      // not a multiple of the tile) is compiled separately so that the common step pays nothing for it.
+      auto softmax_step = [&](auto ragged_tag) -> bool {
+        constexpr bool kRagged = decltype(ragged_tag)::value;
+        if (!wait_bar_warp(bar_s, g & 1, abort_flag, wait_info(kRoleSoftmax, kBarSFull, g))) return false;
         tc_fence_after();
         if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 0);
         if (warp == 0 && g == 0) ATTN_TRACE_MARK(2);
@@ -445,11 +451,23 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int c = 0; c < NCH / 2; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
 #pragma unroll
         for (int c = NCH / 2; c < NCH; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+        // Ragged last KV tile: keys past the end of the sequence were zero-filled by TMA, which would give
+        // them score 0 and weight exp(0 - m) > 0; their scores are set to -inf instead (never zero padding).
+        if constexpr (kRagged) {
+#pragma unroll
+          for (int k = 0; k < TKV / 2; ++k)
+            if (k >= kv_tail) s[k] = 0xFF800000u;
+        }
         const float mx_a = fmaxf(fmaxf(chain_max<0, TKV / 8>(s), chain_max<TKV / 8, TKV / 4>(s)),
                                  fmaxf(chain_max<TKV / 4, 3 * TKV / 8>(s), chain_max<3 * TKV / 8, TKV / 2>(s)));
 #pragma unroll
         for (int c = NCH / 2; c < NCH; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
         if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 1);
+        if constexpr (kRagged) {
+#pragma unroll
+          for (int k = TKV / 2; k < TKV; ++k)
+            if (k >= kv_tail) s[k] = 0xFF800000u;
+        }
         const float mx_b = fmaxf(fmaxf(chain_max<TKV / 2, 5 * TKV / 8>(s), chain_max<5 * TKV / 8, 3 * TKV / 4>(s)),
                                  fmaxf(chain_max<3 * TKV / 4, 7 * TKV / 8>(s), chain_max<7 * TKV / 8, TKV>(s)));
         const float mx = fmaxf(mx_a, mx_b);
@@ -503,6 +521,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tc_fence_before();
         mbar_arrive(bar_h);
         if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 6);
+              return true;
+      };
+      for (int jj = 0; ok && jj < n; ++jj, ++g) {
+        const bool ragged = (kv_tail != 0) && (j0 + jj == p.n_steps - 1);
+        ok = ragged ? softmax_step(RaggedTag<true>{}) : softmax_step(RaggedTag<false>{});
       }
       // ----------------------------------------------------- end of segment
       if (warp == 0) ATTN_TRACE_MARK(3);
@@ -874,7 +897,8 @@ attn_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int row = threadIdx.x;
   const int q_row0 = blockIdx.x * kSub;
   const int bh = blockIdx.y;
-  const int n = L / TKV;
+  const int n = (L + TKV - 1) / TKV;
+  const int kv_tail = L % TKV;
   const uint32_t bar_load = smem_u32(&misc->load_bar), bar_mma = smem_u32(&misc->mma_bar);
   const uint32_t bar_sync = smem_u32(&misc->sync_bar);
 
@@ -926,6 +950,11 @@ attn_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     for (int c = 0; c < TKV / 32; ++c) tmem_ld32(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
     if (scores_out != nullptr && j == 0 && blockIdx.x == 0 && blockIdx.y == 0) {
       for (int k = 0; k < TKV; ++k) scores_out[(size_t)row * TKV + k] = __uint_as_float(s[k]);
+    }
+    if (kv_tail != 0 && j == n - 1) {              // keys past the end of the sequence: -inf, never zero padding
+#pragma unroll
+      for (int k = 0; k < TKV; ++k)
+        if (k >= kv_tail) s[k] = 0xFF800000u;
     }
     float mx = __uint_as_float(s[0]);
 #pragma unroll

@@ -132,6 +132,40 @@ def test_tile_variants_match_oracle(env, d, n_q, tile_kv, kv_stages, kv_splits):
     _run_and_compare(env, _case("variant", 1, 2, 1408, d, sigma_qk=math.sqrt(3.0)), run)
 
 
+@pytest.mark.parametrize("L", [1, 2, 17, 64, 100, 127, 129, 200, 255, 257, 333, 1000, 1111, 2049])
+@pytest.mark.parametrize("d", [64, 128])
+def test_ragged_sequence_lengths(env, d, L):
+    """Any L >= 1: the last key tile is ragged (its out-of-range scores are -inf, never zero-padded,
+    as the paper's boundary note requires) and the last Q tile is clipped."""
+    _, _, binding = env
+    case = _case("ragged", 1, 3, L, d, sigma_qk=1.5)
+    _run_and_compare(env, case, binding.forward)
+    _run_and_compare(env, case, lambda a, b, c: binding.forward_simple(a, b, c, tile_kv=64))
+
+
+@pytest.mark.parametrize("kw", [dict(tile_kv=64), dict(n_q=1), dict(kv_splits=3), dict(ctas=23), dict(n_q=1, tile_kv=64, ctas=41)])
+def test_ragged_length_with_tile_variants_and_key_splits(env, kw):
+    _, _, binding = env
+    case = _case("ragged_variants", 2, 2, 1100, 128, sigma_qk=math.sqrt(3.0))
+    _run_and_compare(env, case, lambda a, b, c: binding.forward_tiles(a, b, c, **kw))
+
+
+def test_zero_padding_would_show(env):
+    """A kernel that treated the zero-filled keys of a ragged tile as real keys would pull every output
+    toward zero-weighted garbage: with all true scores very negative the padded keys would dominate."""
+    torch, orc, binding = env
+    L, d = 130, 64
+    rng = np.random.default_rng(11)
+    q = np.full((1, 1, L, d), 4.0, np.float32)
+    k = np.full((1, 1, L, d), -4.0, np.float32)          # every true score is -16*64/8 = -128
+    v = rng.standard_normal((1, 1, L, d), dtype=np.float32) + 3.0
+    qb, kb, vb = (synth.f32_to_bf16_bits(x) for x in (q, k, v))
+    out = to_host_f64(binding.forward(to_cuda_bf16(qb), to_cuda_bf16(kb), to_cuda_bf16(vb))).reshape(1, L, d)
+    ref = orc.attention_rows(qb, kb, vb, 1, 1, L, d, np.arange(L, dtype=np.int32))
+    assert_close(out, ref, "zero padding")
+    assert np.abs(ref).mean() > 2.0        # the correct answer is the mean of V (~3), not ~0
+
+
 @pytest.mark.parametrize("ctas", [12, 13, 17, 29, 64, 131])
 @pytest.mark.parametrize("d,n_q,tile_kv", [(128, 2, 128), (64, 2, 128), (128, 1, 64)])
 def test_balanced_key_ranges_any_grid_size(env, d, n_q, tile_kv, ctas):

@@ -132,7 +132,7 @@ def test_forward_argument_errors_come_before_any_cuda_call(binding):
     assert L.attn_forward(None, p(b), p(c), p(o), 1, 1, 128, 64, None) == binding.ERR_INVALID_ARG
     assert L.attn_forward(p(a), p(b), p(c), p(o), 0, 1, 128, 64, None) == binding.ERR_INVALID_ARG
     assert L.attn_forward(p(a), p(b), p(c), p(o), 1, 1, 128, 96, None) == binding.ERR_UNSUPPORTED_SHAPE
-    assert L.attn_forward(p(a), p(b), p(c), p(o), 1, 1, 100, 64, None) == binding.ERR_UNSUPPORTED_SHAPE
+    assert L.attn_forward(p(a), p(b), p(c), p(o), 1, 1, 100, 80, None) == binding.ERR_UNSUPPORTED_SHAPE
     assert L.attn_forward(p(a + 8), p(b), p(c), p(o), 1, 1, 128, 64, None) == binding.ERR_MISALIGNED
     assert L.attn_forward(p(a), p(b), p(c), p(a + 1024), 1, 1, 128, 64, None) == binding.ERR_ALIASING
     assert L.attn_forward_simple(p(a), p(b), p(c), p(b), 1, 1, 128, 64, 128, None, None) == binding.ERR_ALIASING

@@ -63,6 +63,6 @@ def test_static_scratch_entry_point_checks_arguments_first():
     p = ctypes.c_void_p
     assert lib.attn_forward_static_scratch(None, p(0x1000), p(0x2000), p(0x3000), 1, 1, 128, 64, None) == \
         binding.ERR_INVALID_ARG
-    assert lib.attn_forward_static_scratch(p(0x100000), p(0x200000), p(0x300000), p(0x400000), 1, 1, 100, 64, None) == \
+    assert lib.attn_forward_static_scratch(p(0x100000), p(0x200000), p(0x300000), p(0x400000), 1, 1, 100, 48, None) == \
         binding.ERR_UNSUPPORTED_SHAPE
     assert "scratch" in binding.status_string(binding.ERR_SCRATCH_LIMIT)
