@@ -28,6 +28,13 @@
  * The paper prints no numeric attention outputs, so parity with the paper's
  * own outputs is unpinned.
  *
+ * Causal variant (attn_oracle_rows_causal): the same definition with the scores of
+ * keys after the query's own position set to -inf before the softmax (the
+ * paper's boundary rule -- masked elements are -inf, never zero -- applied to a
+ * triangular mask), i.e. row i attends to keys 0..i only.  Pinned by: row i
+ * equals the non-causal result over the first i+1 keys; row 0 equals V[0];
+ * changing K/V rows after position i leaves row i unchanged.
+ *
  * Layout: q, k, v are contiguous [B][H][L][d], d fastest.
  * rows[]: n_rows row indices in [0, L), the same list for every head.
  * out:    [B*H][n_rows][d] fp64.
@@ -56,9 +63,9 @@ int attn_oracle_threads(void) {
 #endif
 }
 
-int attn_oracle_rows(const uint16_t *q, const uint16_t *k, const uint16_t *v,
-                     int B, int H, int L, int d, const int32_t *rows,
-                     int n_rows, double *out, double *psum) {
+static int oracle_rows_impl(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                            int B, int H, int L, int d, const int32_t *rows,
+                            int n_rows, double *out, double *psum, int causal) {
   if (!q || !k || !v || !rows || !out) return -1;
   if (B <= 0 || H <= 0 || L <= 0 || d <= 0 || n_rows < 0) return -1;
   for (int r = 0; r < n_rows; ++r)
@@ -99,9 +106,11 @@ int attn_oracle_rows(const uint16_t *q, const uint16_t *k, const uint16_t *v,
           const int i = rows[r];
           for (int c = 0; c < d; ++c) qi[c] = bf16_to_f64(qh[(size_t)i * d + c]);
 
+          /* keys this row may attend to: all of them, or 0..i when causal */
+          const int Lk = causal ? i + 1 : L;
           /* scores and their maximum */
           double M = -INFINITY;
-          for (int j = 0; j < L; ++j) {
+          for (int j = 0; j < Lk; ++j) {
             const double *kj = Kd + (size_t)j * d;
             double dot = 0.0;
             for (int c = 0; c < d; ++c) dot += qi[c] * kj[c];
@@ -110,13 +119,13 @@ int attn_oracle_rows(const uint16_t *q, const uint16_t *k, const uint16_t *v,
           }
           /* weights and normaliser */
           double delta = 0.0;
-          for (int j = 0; j < L; ++j) {
+          for (int j = 0; j < Lk; ++j) {
             s[j] = exp(s[j] - M);
             delta += s[j];
           }
           /* weighted sum of value rows */
           for (int c = 0; c < d; ++c) acc[c] = 0.0;
-          for (int j = 0; j < L; ++j) {
+          for (int j = 0; j < Lk; ++j) {
             const double pj = s[j];
             const double *vj = Vd + (size_t)j * d;
             for (int c = 0; c < d; ++c) acc[c] += pj * vj[c];
@@ -125,7 +134,7 @@ int attn_oracle_rows(const uint16_t *q, const uint16_t *k, const uint16_t *v,
           for (int c = 0; c < d; ++c) o[c] = acc[c] / delta;
           if (psum) {
             double t = 0.0;
-            for (int j = 0; j < L; ++j) t += s[j] / delta;
+            for (int j = 0; j < Lk; ++j) t += s[j] / delta;
             psum[(size_t)bh * n_rows + r] = t;
           }
         }
@@ -139,4 +148,16 @@ int attn_oracle_rows(const uint16_t *q, const uint16_t *k, const uint16_t *v,
     if (status) return status;
   }
   return 0;
+}
+
+int attn_oracle_rows(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                     int B, int H, int L, int d, const int32_t *rows,
+                     int n_rows, double *out, double *psum) {
+  return oracle_rows_impl(q, k, v, B, H, L, d, rows, n_rows, out, psum, 0);
+}
+
+int attn_oracle_rows_causal(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                            int B, int H, int L, int d, const int32_t *rows,
+                            int n_rows, double *out, double *psum) {
+  return oracle_rows_impl(q, k, v, B, H, L, d, rows, n_rows, out, psum, 1);
 }

@@ -54,6 +54,8 @@ def _load():
         lib.attn_oracle_rows.restype = ctypes.c_int
         lib.attn_oracle_rows.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int] * 4 + [
             ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
+        lib.attn_oracle_rows_causal.restype = ctypes.c_int
+        lib.attn_oracle_rows_causal.argtypes = lib.attn_oracle_rows.argtypes
         lib.attn_oracle_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -70,8 +72,10 @@ def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
-def attention_rows(q_bits, k_bits, v_bits, B, H, L, d, rows, want_psum=False):
+def attention_rows(q_bits, k_bits, v_bits, B, H, L, d, rows, want_psum=False, causal=False):
     """Definition of attention for the given rows of every head (C, fp64).
+
+    causal=True: row i attends to keys 0..i only (later keys have score -inf).
 
     q_bits, k_bits, v_bits: uint16 bf16 bit patterns, contiguous [B][H][L][d].
     rows: 1-D int array of row indices (same for every head).
@@ -87,7 +91,8 @@ def attention_rows(q_bits, k_bits, v_bits, B, H, L, d, rows, want_psum=False):
     rows = np.ascontiguousarray(rows, dtype=np.int32)
     out = np.empty((B * H, rows.size, d), dtype=np.float64)
     psum = np.empty((B * H, rows.size), dtype=np.float64) if want_psum else None
-    rc = lib.attn_oracle_rows(
+    fn = lib.attn_oracle_rows_causal if causal else lib.attn_oracle_rows
+    rc = fn(
         q_bits.ctypes.data, k_bits.ctypes.data, v_bits.ctypes.data, B, H, L, d,
         rows.ctypes.data, int(rows.size), out.ctypes.data,
         psum.ctypes.data if want_psum else None)
@@ -96,14 +101,18 @@ def attention_rows(q_bits, k_bits, v_bits, B, H, L, d, rows, want_psum=False):
     return (out, psum) if want_psum else out
 
 
-def attention_definition(q: np.ndarray, k: np.ndarray, v: np.ndarray) -> np.ndarray:
-    """softmax(Q K^T / sqrt(d)) V for one head, fp64, via scipy + numpy."""
+def attention_definition(q: np.ndarray, k: np.ndarray, v: np.ndarray, causal: bool = False) -> np.ndarray:
+    """softmax(Q K^T / sqrt(d)) V for one head, fp64, via scipy + numpy.
+
+    causal=True masks the scores of keys after the query's position with -inf."""
     from scipy.special import softmax
 
     q = np.asarray(q, dtype=np.float64)
     k = np.asarray(k, dtype=np.float64)
     v = np.asarray(v, dtype=np.float64)
     s = (q @ k.T) * (1.0 / np.sqrt(np.float64(q.shape[1])))
+    if causal:
+        s = np.where(np.tril(np.ones(s.shape, dtype=bool)), s, -np.inf)
     return softmax(s, axis=1) @ v
 
 

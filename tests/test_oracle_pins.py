@@ -222,3 +222,45 @@ def test_sample_rows_properties():
             assert counts.min() >= 2
             for r in (0, 127, 128, L - 128, L - 1):
                 assert r in rows
+
+
+# ----------------------------------------------------------------------------- causal variant
+def test_causal_row_equals_noncausal_attention_over_its_prefix():
+    """Brute force through the already pinned non-causal oracle: row i of the causal result is the
+    last row of plain attention over the first i+1 keys and values."""
+    B, H, L, d = 1, 2, 70, 16
+    q, k, v = (_rand_bits((B, H, L, d), 1.5, 21, t) for t in range(3))
+    got = orc.attention_rows(q, k, v, B, H, L, d, _rows(L), causal=True)
+    for i in (0, 1, 2, 31, 32, 63, 64, 69):
+        ref = orc.attention_rows(q[:, :, : i + 1].copy(), k[:, :, : i + 1].copy(), v[:, :, : i + 1].copy(),
+                                 B, H, i + 1, d, np.array([i], dtype=np.int32))
+        np.testing.assert_allclose(got[:, i], ref[:, 0], rtol=1e-13, atol=1e-15)
+    # row 0 sees one key only: the output is V[0] exactly
+    assert np.array_equal(got[:, 0], _f64(v).reshape(B * H, L, d)[:, 0])
+
+
+def test_causal_rows_ignore_later_keys_and_values():
+    B, H, L, d = 1, 1, 50, 8
+    q, k, v = (_rand_bits((B, H, L, d), 1.0, 22, t) for t in range(3))
+    base = orc.attention_rows(q, k, v, B, H, L, d, _rows(L), causal=True)[0]
+    k2, v2 = k.copy(), v.copy()
+    k2[:, :, 30:] = _rand_bits((B, H, 20, d), 3.0, 23, 1)
+    v2[:, :, 30:] = _rand_bits((B, H, 20, d), 3.0, 23, 2)
+    out = orc.attention_rows(q, k2, v2, B, H, L, d, _rows(L), causal=True)[0]
+    assert np.array_equal(out[:30], base[:30])            # rows before the change are untouched
+    assert np.abs(out[30:] - base[30:]).max() > 1e-3      # rows that can see it do change
+    # and the causal result differs from the non-causal one (a mask that does nothing would be caught)
+    full = orc.attention_rows(q, k, v, B, H, L, d, _rows(L))[0]
+    assert np.abs(full[:-1] - base[:-1]).max() > 1e-3
+    np.testing.assert_allclose(full[-1], base[-1], rtol=1e-13)   # the last row sees every key either way
+
+
+def test_causal_c_oracle_matches_library_definition():
+    B, H, L, d = 2, 2, 200, 64
+    q, k, v = (_rand_bits((B, H, L, d), math.sqrt(3.0), 24, t) for t in range(3))
+    out, psum = orc.attention_rows(q, k, v, B, H, L, d, _rows(L), want_psum=True, causal=True)
+    np.testing.assert_allclose(psum, 1.0, rtol=0, atol=1e-13)
+    qf, kf, vf = (_f64(x).reshape(B * H, L, d) for x in (q, k, v))
+    for bh in range(B * H):
+        np.testing.assert_allclose(out[bh], orc.attention_definition(qf[bh], kf[bh], vf[bh], causal=True),
+                                   rtol=1e-12, atol=1e-14)
