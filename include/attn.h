@@ -107,7 +107,7 @@ typedef struct attn_tiles {
   int32_t feasible;       /* 1 if a tile choice fits                                    */
   int32_t binding_constraint; /* attn_binding                                           */
   int32_t under_occupied; /* 1 if tiles < num_units (occupancy check of the derivation) */
-  int32_t reserved;
+  int32_t causal;         /* 1 if planned for causal attention (row i sees keys 0..i)   */
 } attn_tiles;
 
 /* Built-in descriptor of one B200 (148 SMs, 227 KB SMEM opt-in, 64 K registers,
@@ -128,9 +128,17 @@ int attn_hw_desc_query(int device, attn_hw_desc *out);
  */
 int attn_plan(const attn_hw_desc *desc, int B, int H, int L, int d, attn_tiles *out);
 
-/* Bytes of workspace attn_forward* needs for this plan: 0 unless ctas > tiles
- * (64 KB of arrival counters, then ctas + tiles slots of partial outputs and row
- * statistics for the merge operator, Section "Online Softmax"). */
+/* Same derivation for causal attention (causal != 0): Q tile q needs only the key
+ * steps up to its own last row, so the work per tile is unequal and the occupancy
+ * step always deals the (Q tile, KV step) units out in equal ranges, one per unit.
+ * (The paper treats non-causal attention only; this applies its -inf masking rule,
+ * Section "Online Softmax", to a triangular mask.) */
+int attn_plan_ex(const attn_hw_desc *desc, int B, int H, int L, int d, int causal, attn_tiles *out);
+
+/* Bytes of workspace attn_forward* needs for this plan: 0 if every CTA owns exactly
+ * one whole Q tile (ctas == tiles, not causal); otherwise 64 KB of arrival counters,
+ * then two slots per CTA of partial outputs and row statistics for the merge
+ * operator, Section "Online Softmax". */
 size_t attn_workspace_bytes(const attn_tiles *tiles, int B, int H, int L, int d);
 
 /* Registers a caller-owned device buffer as the workspace of `device` (pass
@@ -150,11 +158,23 @@ int attn_set_workspace(int device, void *dev_ptr, size_t bytes);
 int attn_forward(const void *q, const void *k, const void *v, void *o,
                  int B, int H, int L, int d, void *cuda_stream);
 
+/*
+ * Causal fused attention forward: as attn_forward, but row i attends to keys 0..i
+ * only -- the scores of later keys are -inf before the softmax (the paper's rule
+ * that masked elements are -inf, never zero, Section "Online Softmax", applied to
+ * a triangular mask; the paper itself evaluates non-causal attention only).
+ * Key steps wholly after a Q tile's last row are skipped, not computed and masked.
+ * Always needs a registered workspace (attn_workspace_bytes of attn_plan_ex(...,1,...)).
+ */
+int attn_forward_causal(const void *q, const void *k, const void *v, void *o,
+                        int B, int H, int L, int d, void *cuda_stream);
+
 /* Same, with tile fields overridden (tile sweep only).  Honoured fields (0 keeps
  * the closed-form value): n_q (1|2), tile_kv (64|128), kv_stages (2..plan maximum),
- * kv_splits (that many CTAs per Q tile) or ctas (the grid size itself, from the
- * number of Q tiles up to tiles * KV steps).  ATTN_ERR_BAD_TILES if the combination
- * was not compiled or does not fit. */
+ * kv_splits (that many CTAs per Q tile) or ctas (the grid size itself, from 1 up
+ * to the number of (Q tile, KV step) units), causal (non-zero selects causal
+ * attention).  ATTN_ERR_BAD_TILES if the combination was not compiled or does not
+ * fit. */
 int attn_forward_tiles(const void *q, const void *k, const void *v, void *o,
                        int B, int H, int L, int d, const attn_tiles *override_tiles,
                        void *cuda_stream);
@@ -197,7 +217,7 @@ int attn_forward_host(const void *q_host, const void *k_host, const void *v_host
  * attn_forward needs a caller-supplied workspace whenever the plan splits the
  * key axis; such callers have nowhere to get one from.  Here the partial
  * results and arrival counters live in an array that is part of the library
- * image itself: ATTN_STATIC_SCRATCH_BYTES (about 37.5 MiB) of device memory,
+ * image itself: ATTN_STATIC_SCRATCH_BYTES (about 37.6 MiB) of device memory,
  * held by every GPU that loads the library until the process exits.
  *
  * q, k, v, o, shapes, stream and results are exactly those of attn_forward (same
@@ -215,7 +235,7 @@ int attn_forward_host(const void *q_host, const void *k_host, const void *v_host
  *     ATTN_STATIC_SCRATCH_BYTES (never the case for the built-in B200 descriptor
  *     with d <= 128); other errors as attn_forward.
  */
-#define ATTN_STATIC_SCRATCH_BYTES 39335936
+#define ATTN_STATIC_SCRATCH_BYTES 39469056
 int attn_forward_static_scratch(const void *q, const void *k, const void *v, void *o,
                                 int B, int H, int L, int d, void *cuda_stream);
 

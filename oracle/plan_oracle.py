@@ -66,7 +66,12 @@ _MIN_STEPS_PER_SPLIT = 4
 _SEGMENT_OVERHEAD_STEPS = 3
 
 
-def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int) -> dict:
+def causal_head_units(q_tiles: int, steps: int, ratio: int) -> int:
+    """KV steps summed over the Q tiles of one head when tile q needs min(steps, (q+1)*ratio) of them."""
+    return sum(min(steps, (q + 1) * ratio) for q in range(q_tiles))
+
+
+def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal: bool = False) -> dict:
     sub = desc["atom_m"]
     out = dict(feasible=False, binding=BIND_SHAPE)
     if d % desc["atom_k"] or d % desc["atom_n"] or d > desc["atom_n_max"] or min(B, H, L, d) <= 0:
@@ -105,7 +110,10 @@ def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int) -> dic
     steps = -(-L // tile_kv)
     under = tiles < desc["num_units"]
     ctas = tiles
-    if under:
+    if causal:
+        total = B * H * causal_head_units(-(-L // tile_q), steps, tile_q // tile_kv)
+        ctas = max(1, min(total // _MIN_STEPS_PER_SPLIT, desc["num_units"]))
+    elif under:
         k = max(1, min(desc["num_units"] // tiles, steps // _MIN_STEPS_PER_SPLIT))
         cost_uniform = -(-steps // k) + _SEGMENT_OVERHEAD_STEPS
         total = tiles * steps

@@ -21,8 +21,8 @@ ERR_DEVICE_TIMEOUT, ERR_BAD_TILES, ERR_SCRATCH_LIMIT = -9, -10, -11
 BIND_NAMES = ("none", "smem", "tmem", "reg", "atom", "shape")
 
 EXPORTED_SYMBOLS = (
-    "attn_hw_desc_b200", "attn_hw_desc_query", "attn_plan", "attn_workspace_bytes", "attn_set_workspace",
-    "attn_forward", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_static_scratch",
+    "attn_hw_desc_b200", "attn_hw_desc_query", "attn_plan", "attn_plan_ex", "attn_workspace_bytes",
+    "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_static_scratch",
     "attn_last_device_status",
     "attn_last_launch_count", "attn_status_string", "attn_last_cuda_error",
 )
@@ -40,7 +40,7 @@ class AttnTiles(ctypes.Structure):
         "tile_q", "tile_kv", "n_q", "n_s", "kv_stages", "kv_splits", "smem_bytes", "tmem_columns", "regs_softmax",
         "threads", "tiles", "ctas",
     )] + [("ctas_per_unit", ctypes.c_float), ("wave_efficiency", ctypes.c_float)] + [
-        (n, ctypes.c_int32) for n in ("feasible", "binding_constraint", "under_occupied", "reserved")]
+        (n, ctypes.c_int32) for n in ("feasible", "binding_constraint", "under_occupied", "causal")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.attn_hw_desc_b200.argtypes = [ctypes.POINTER(AttnHwDesc)]
         L.attn_hw_desc_query.argtypes = [i32, ctypes.POINTER(AttnHwDesc)]
         L.attn_plan.argtypes = [ctypes.POINTER(AttnHwDesc), i32, i32, i32, i32, ctypes.POINTER(AttnTiles)]
+        L.attn_plan_ex.argtypes = [ctypes.POINTER(AttnHwDesc), i32, i32, i32, i32, i32, ctypes.POINTER(AttnTiles)]
+        L.attn_forward_causal.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
         L.attn_workspace_bytes.argtypes = [ctypes.POINTER(AttnTiles), i32, i32, i32, i32]
         L.attn_workspace_bytes.restype = ctypes.c_size_t
         L.attn_set_workspace.argtypes = [i32, vp, ctypes.c_size_t]
@@ -116,9 +118,12 @@ def hw_desc_query(device: int = 0) -> AttnHwDesc:
     return d
 
 
-def plan(desc: AttnHwDesc, B: int, H: int, L: int, d: int) -> AttnTiles:
+def plan(desc: AttnHwDesc, B: int, H: int, L: int, d: int, causal: bool = False) -> AttnTiles:
     t = AttnTiles()
-    _check(lib().attn_plan(ctypes.byref(desc), B, H, L, d, ctypes.byref(t)), "attn_plan")
+    if causal:
+        _check(lib().attn_plan_ex(ctypes.byref(desc), B, H, L, d, 1, ctypes.byref(t)), "attn_plan_ex")
+    else:
+        _check(lib().attn_plan(ctypes.byref(desc), B, H, L, d, ctypes.byref(t)), "attn_plan")
     return t
 
 
@@ -170,17 +175,20 @@ def _prep(q, k, v, o):
     return o, B, H, L, d, dev, stream
 
 
-def forward(q, k, v, o=None):
-    """O = softmax(Q K^T / sqrt(d)) V with the closed-form default tiles (asynchronous)."""
+def forward(q, k, v, o=None, causal=False):
+    """O = softmax(Q K^T / sqrt(d)) V with the closed-form default tiles (asynchronous).
+
+    causal=True: row i attends to keys 0..i only."""
     import torch
 
     o, B, H, L, d, dev, stream = _prep(q, k, v, o)
     with torch.cuda.device(dev):
-        t = plan(_device_desc(dev), B, H, L, d)
-        if t.feasible and t.ctas > t.tiles:
+        t = plan(_device_desc(dev), B, H, L, d, causal)
+        if t.feasible:
             ensure_workspace(dev, workspace_bytes(t, B, H, L, d))
-        _check(lib().attn_forward(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d, stream),
-               "attn_forward")
+        fn = lib().attn_forward_causal if causal else lib().attn_forward
+        _check(fn(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d, stream),
+               "attn_forward_causal" if causal else "attn_forward")
     return o
 
 
@@ -198,11 +206,11 @@ def forward_static_scratch(q, k, v, o):
     return o
 
 
-def forward_tiles(q, k, v, o=None, *, n_q=0, tile_kv=0, kv_stages=0, kv_splits=0, ctas=0):
+def forward_tiles(q, k, v, o=None, *, n_q=0, tile_kv=0, kv_stages=0, kv_splits=0, ctas=0, causal=False):
     """Same with tile fields overridden (0 keeps the closed-form value); tile sweep only.
 
-    kv_splits asks for that many CTAs per Q tile; ctas sets the grid size directly (any value from
-    the number of Q tiles up to the number of (Q tile, KV step) units)."""
+    kv_splits asks for that many CTAs per Q tile; ctas sets the grid size directly (any value from 1
+    up to the number of (Q tile, KV step) units); causal selects causal attention."""
     import torch
 
     o, B, H, L, d, dev, stream = _prep(q, k, v, o)
@@ -211,11 +219,12 @@ def forward_tiles(q, k, v, o=None, *, n_q=0, tile_kv=0, kv_stages=0, kv_splits=0
         base = plan(desc, B, H, L, d)
         ov = AttnTiles()
         ov.n_q, ov.tile_kv, ov.kv_stages, ov.kv_splits, ov.ctas = n_q, tile_kv, kv_stages, kv_splits, ctas
+        ov.causal = 1 if causal else 0
         eff_nq = n_q or base.n_q
         tiles = B * H * math.ceil(L / (128 * eff_nq))
         w = AttnTiles()          # upper bound of what the call can need
-        w.feasible, w.n_q, w.tiles = 1, eff_nq, tiles
-        w.ctas = max(ctas, tiles * max(kv_splits, 1), desc.num_units, tiles + 1)
+        w.feasible, w.n_q, w.tiles, w.causal = 1, eff_nq, tiles, 1
+        w.ctas = max(ctas, tiles * max(kv_splits, 1), desc.num_units, tiles)
         ensure_workspace(dev, workspace_bytes(w, B, H, L, d))
         _check(lib().attn_forward_tiles(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d,
                                         ctypes.byref(ov), stream), "attn_forward_tiles")
@@ -251,7 +260,7 @@ def forward_host(q_host, k_host, v_host, o_host, dev_scratch):
     stream = torch.cuda.current_stream(dev_scratch.device).cuda_stream
     with torch.cuda.device(dev):
         t = plan(_device_desc(dev), B, H, L, d)
-        if t.feasible and t.ctas > t.tiles:
+        if t.feasible:
             ensure_workspace(dev, workspace_bytes(t, B, H, L, d))
         _check(lib().attn_forward_host(q_host.data_ptr(), k_host.data_ptr(), v_host.data_ptr(), o_host.data_ptr(),
                                        B, H, L, d, dev_scratch.data_ptr(), dev_scratch.numel(), stream),

@@ -129,18 +129,28 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   p.n_steps = (L + TKV - 1) / TKV;
   p.tiles = BH * p.q_tiles;
   p.stages = t.kv_stages;
+  p.causal = t.causal ? 1 : 0;
+  p.ratio = NQ * attn::kSub / TKV;
+  p.head_units = attn::tile_prefix(p.n_steps, p.ratio, p.causal, p.q_tiles);
   p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
   p.o = reinterpret_cast<__nv_bfloat16*>(o);
   p.counters = reinterpret_cast<unsigned int*>(ws);                   // head of the workspace
   p.ws = ws ? ws + attn::kCounterBytes / sizeof(float) : nullptr;    // partial results follow
   const int grid = t.ctas;
-  // one CTA per Q tile at least (several whole tiles per CTA are not supported), one KV step per CTA at least
-  if (grid < p.tiles || (long long)grid > (long long)p.tiles * p.n_steps) return ATTN_ERR_BAD_TILES;
-  if (grid > p.tiles && (size_t)p.tiles * NQ > attn::kCounterBytes / sizeof(unsigned int)) return ATTN_ERR_BAD_TILES;
+  const long long total_units = p.head_units * BH;
+  // at least one KV step per CTA; two arrival counters per CTA must fit the counter block
+  if (grid < 1 || (long long)grid > total_units) return ATTN_ERR_BAD_TILES;
+  if ((size_t)grid * NQ > attn::kCounterBytes / sizeof(unsigned int)) return ATTN_ERR_BAD_TILES;
   const int smem = SM::total(t.kv_stages);
-  auto kern = attn::attn_fwd_kernel<D, TKV, NQ>;
-  ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
+  if (p.causal) {
+    auto kern = attn::attn_fwd_kernel<D, TKV, NQ, true>;
+    ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
+  } else {
+    auto kern = attn::attn_fwd_kernel<D, TKV, NQ, false>;
+    ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
+  }
   ATTN_CUDA_TRY(cudaGetLastError());
   t_launch_count = 1;
   return ATTN_OK;
@@ -162,15 +172,19 @@ int dispatch_fwd(const void* q, const void* k, const void* v, void* o, int B, in
   return ATTN_ERR_BAD_TILES;
 }
 
-int forward_impl(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
+// A plan needs the workspace unless every CTA owns exactly one whole Q tile.
+bool plan_needs_workspace(const attn_tiles& t) { return t.causal != 0 || t.ctas != t.tiles; }
+
+int forward_impl(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d, int causal,
                  const attn_tiles* ovr, void* cuda_stream) {
   t_launch_count = 0;
   int rc = check_args(q, k, v, o, B, H, L, d);
   if (rc != ATTN_OK) return rc;
   DeviceState* st = nullptr;
   if ((rc = device_state(&st)) != ATTN_OK) return rc;
+  if (ovr && ovr->causal) causal = 1;
   attn_tiles t;
-  if ((rc = attn_plan(&st->desc, B, H, L, d, &t)) != ATTN_OK) return rc;
+  if ((rc = attn_plan_ex(&st->desc, B, H, L, d, causal, &t)) != ATTN_OK) return rc;
   if (!t.feasible) return ATTN_ERR_INFEASIBLE_PLAN;
   if (ovr) {
     if (ovr->n_q > 0) t.n_q = ovr->n_q;
@@ -192,14 +206,14 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
     } else if (ovr->kv_splits > 0) {
       t.ctas = t.tiles * ovr->kv_splits;
     } else {
-      t.ctas = attn_internal::grid_size(st->desc, t.tiles, steps);
+      t.ctas = attn_internal::grid_size(st->desc, B * H, (L + t.tile_q - 1) / t.tile_q, steps, t.tile_q / t.tile_kv, causal);
     }
     t.kv_splits = (t.ctas + t.tiles - 1) / t.tiles;
-    if (t.ctas < t.tiles || (long long)t.ctas > (long long)t.tiles * steps) return ATTN_ERR_BAD_TILES;
+    if (t.ctas < 1) return ATTN_ERR_BAD_TILES;
     t.smem_bytes = q_bytes + t.kv_stages * stage + 3072;
   }
   float* ws = nullptr;
-  if (t.ctas > t.tiles) {
+  if (plan_needs_workspace(t)) {
     const size_t need = attn_workspace_bytes(&t, B, H, L, d);
     std::lock_guard<std::mutex> lk(g_mu);
     if (!st->ws || st->ws_bytes < need) return ATTN_ERR_NEED_WORKSPACE;
@@ -267,12 +281,17 @@ extern "C" int attn_set_workspace(int device, void* dev_ptr, size_t bytes) {
 
 extern "C" int attn_forward(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
                             void* cuda_stream) {
-  return forward_impl(q, k, v, o, B, H, L, d, nullptr, cuda_stream);
+  return forward_impl(q, k, v, o, B, H, L, d, 0, nullptr, cuda_stream);
+}
+
+extern "C" int attn_forward_causal(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
+                                   void* cuda_stream) {
+  return forward_impl(q, k, v, o, B, H, L, d, 1, nullptr, cuda_stream);
 }
 
 extern "C" int attn_forward_tiles(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
                                   const attn_tiles* override_tiles, void* cuda_stream) {
-  return forward_impl(q, k, v, o, B, H, L, d, override_tiles, cuda_stream);
+  return forward_impl(q, k, v, o, B, H, L, d, 0, override_tiles, cuda_stream);
 }
 
 extern "C" int attn_forward_simple(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
@@ -305,7 +324,7 @@ extern "C" int attn_forward_host(const void* q_host, const void* k_host, const v
   ATTN_CUDA_TRY(cudaMemcpyAsync(dq, q_host, bytes, cudaMemcpyHostToDevice, s));
   ATTN_CUDA_TRY(cudaMemcpyAsync(dk, k_host, bytes, cudaMemcpyHostToDevice, s));
   ATTN_CUDA_TRY(cudaMemcpyAsync(dv, v_host, bytes, cudaMemcpyHostToDevice, s));
-  rc = forward_impl(dq, dk, dv, dout, B, H, L, d, nullptr, cuda_stream);
+  rc = forward_impl(dq, dk, dv, dout, B, H, L, d, 0, nullptr, cuda_stream);
   if (rc != ATTN_OK) return rc;
   ATTN_CUDA_TRY(cudaMemcpyAsync(o_host, dout, bytes, cudaMemcpyDeviceToHost, s));
   return ATTN_OK;
@@ -353,7 +372,7 @@ extern "C" int attn_forward_static_scratch(const void* q, const void* k, const v
   void* scratch = nullptr;
   if ((rc = static_scratch_address(&scratch)) != ATTN_OK) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (t.ctas > t.tiles) {
+  if (plan_needs_workspace(t)) {
     if (attn_workspace_bytes(&t, B, H, L, d) > (size_t)ATTN_STATIC_SCRATCH_BYTES) return ATTN_ERR_SCRATCH_LIMIT;
     // the array keeps the previous call's contents: the arrival counters must start at zero
     ATTN_CUDA_TRY(cudaMemsetAsync(scratch, 0, attn::kCounterBytes, stream));

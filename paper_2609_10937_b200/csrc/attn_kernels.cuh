@@ -155,40 +155,79 @@ __device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint3
 struct FwdParams {
   int L;                   // sequence length
   int q_tiles;             // Q tiles per head = ceil(L / (NQ*128))
-  int n_steps;             // KV steps per Q tile = L / TKV
+  int n_steps;             // KV steps of the whole key axis = ceil(L / TKV)
   int tiles;               // Q tiles in the whole problem = B * H * q_tiles
   int stages;              // ring depth
+  int causal;              // 1: row i attends to keys 0..i only
+  int ratio;               // Q-tile rows / TKV (1, 2 or 4)
+  long long head_units;    // work units of one head (see tile_prefix)
   float scale_log2;        // log2(e) / sqrt(d)
-  __nv_bfloat16* o;        // output, written directly by the CTA that merges a shared Q tile
+  __nv_bfloat16* o;        // output, written directly when a result cannot go through the Q buffer
   float* ws;               // partial results of Q tiles shared by several CTAs
-  unsigned int* counters;  // one arrival counter per (Q tile, sub-tile); zero between launches
+  unsigned int* counters;  // arrival counters of shared Q tiles; zero between launches
 };
 
-// Work decomposition.  The problem is a line of tiles * n_steps units (Q tile major, KV step minor);
-// CTA c of G owns units [c*T/G, (c+1)*T/G).  With G == tiles every CTA owns exactly one whole Q tile;
-// with G > tiles the ranges are balanced regardless of tile boundaries, a CTA's range may straddle
-// one boundary (two segments), and Q tiles covered by several CTAs are merged by the last to finish.
+// Work decomposition.  A work unit is one KV step of one Q tile.  Q tile q of a head needs
+// tile_steps(q) steps: all n_steps of them, or -- causal -- only those whose keys are not after the
+// tile's last row, min(n_steps, (q+1)*ratio).  The units of the whole problem form one line (head
+// major, Q tile, KV step); CTA c of G owns units [c*T/G, (c+1)*T/G) and walks them as segments, one per
+// Q tile it touches.  A Q tile covered by several CTAs is merged by the last of them to finish.
+__host__ __device__ __forceinline__ int tile_steps(int n_steps, int ratio, int causal, int q) {
+  if (!causal) return n_steps;
+  const long long s = (long long)(q + 1) * ratio;
+  return s < n_steps ? (int)s : n_steps;
+}
+// Units of Q tiles 0..q-1 of one head (closed form: a triangular number until the step count saturates).
+__host__ __device__ __forceinline__ long long tile_prefix(int n_steps, int ratio, int causal, int q) {
+  if (!causal) return (long long)q * n_steps;
+  long long qc = n_steps / ratio;
+  if (qc > q) qc = q;
+  return (long long)ratio * qc * (qc + 1) / 2 + (long long)(q - qc) * n_steps;
+}
 __device__ __forceinline__ long long range_begin(long long c, long long T, long long G) { return (c * T) / G; }
+__device__ __forceinline__ int cta_of_unit(long long u, long long T, long long G) {
+  return (int)(((u + 1) * G - 1) / T);
+}
 template <bool V>
-struct RaggedTag { static constexpr bool value = V; };
-struct Segment { int tile, j0, j1, n, bh, q_row0, seg; };
+struct MaskTag { static constexpr bool value = V; };
+struct Segment { int tile, q, j0, j1, n, bh, q_row0, seg, steps_t; bool full; long long unit0; };
+// Q tile (head, index) that owns unit u, and the unit at which that tile starts.
 // Next piece of the unit range [u, u_hi) that lies inside one Q tile; advances u and the segment counter.
+// (Scalar arguments and straight-line code on purpose: the non-causal instantiation must stay as lean as
+// it was before causal support existed -- measured, helper structs here cost several per cent.)
+template <bool CAUSAL>
 __device__ __forceinline__ bool next_segment(long long& u, long long u_hi, int& seg_ctr, int n_steps, int q_tiles,
-                                             int tile_rows, Segment& sg) {
+                                             int ratio, long long head_units, int tile_rows, Segment& sg) {
   if (u >= u_hi) return false;
-  sg.tile = (int)(u / n_steps);
-  sg.j0 = (int)(u % n_steps);
+  if constexpr (!CAUSAL) {
+    sg.tile = (int)(u / n_steps);
+    sg.j0 = (int)(u % n_steps);
+    sg.bh = sg.tile / q_tiles;
+    sg.q = sg.tile % q_tiles;
+    sg.steps_t = n_steps;
+    sg.unit0 = (long long)sg.tile * n_steps;
+  } else {
+    sg.bh = (int)(u / head_units);
+    const long long r = u - (long long)sg.bh * head_units;
+    int lo = 0, hi = q_tiles - 1;                     // largest q with tile_prefix(q) <= r
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (tile_prefix(n_steps, ratio, 1, mid) <= r) lo = mid; else hi = mid - 1;
+    }
+    sg.q = lo;
+    sg.tile = sg.bh * q_tiles + lo;
+    sg.unit0 = (long long)sg.bh * head_units + tile_prefix(n_steps, ratio, 1, lo);
+    sg.steps_t = tile_steps(n_steps, ratio, 1, lo);
+    sg.j0 = (int)(u - sg.unit0);
+  }
   const long long left = u_hi - u;
-  sg.j1 = (left < (long long)(n_steps - sg.j0)) ? sg.j0 + (int)left : n_steps;
+  sg.j1 = (left < (long long)(sg.steps_t - sg.j0)) ? sg.j0 + (int)left : sg.steps_t;
   sg.n = sg.j1 - sg.j0;
-  sg.bh = sg.tile / q_tiles;
-  sg.q_row0 = (sg.tile % q_tiles) * tile_rows;
+  sg.full = (sg.j0 == 0 && sg.j1 == sg.steps_t);
+  sg.q_row0 = sg.q * tile_rows;
   sg.seg = seg_ctr++;
   u += sg.n;
   return true;
-}
-__device__ __forceinline__ int cta_of_unit(long long u, long long T, long long G) {
-  return (int)(((u + 1) * G - 1) / T);
 }
 
 // Shared-memory footprint helpers (host and device agree through these).
@@ -244,14 +283,12 @@ __device__ __forceinline__ float chain_max(const uint32_t* s) {
 }
 // Constants of the exponential evaluation, packed once per thread.
 struct ExpConsts {
-  uint64_t scale2, magic2, neg_magic2, minus_one2, c3, c2, c1, c0;
+  uint64_t scale2, magic2, c3, c2, c1, c0;
 };
 __device__ __forceinline__ ExpConsts make_exp_consts(float scale) {
   ExpConsts k;
   k.scale2 = pack_f32x2(scale, scale);
   k.magic2 = pack_f32x2(12582912.0f, 12582912.0f);          // 1.5 * 2^23: adding it rounds to an integer
-  k.neg_magic2 = pack_f32x2(-12582912.0f, -12582912.0f);
-  k.minus_one2 = pack_f32x2(-1.0f, -1.0f);
   // minimax cubic for 2^f on [-0.5, 0.5], relative error 7.6e-5 (bf16 rounding of P is 2e-3)
   k.c3 = pack_f32x2(0.055168043822050095f, 0.055168043822050095f);
   k.c2 = pack_f32x2(0.24260213971138f, 0.24260213971138f);
@@ -268,8 +305,8 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, const ExpConsts& k, 
   x1 = fmaxf(x1, -126.0f);
   const uint64_t xc = pack_f32x2(x0, x1);
   const uint64_t r2 = add_f32x2(xc, k.magic2);
-  const uint64_t n2 = add_f32x2(r2, k.neg_magic2);
-  const uint64_t f2 = fma_f32x2(n2, k.minus_one2, xc);
+  const uint64_t n2 = sub_f32x2(r2, k.magic2);
+  const uint64_t f2 = sub_f32x2(xc, n2);
   uint64_t p2 = fma_f32x2(f2, k.c3, k.c2);
   p2 = fma_f32x2(p2, f2, k.c1);
   p2 = fma_f32x2(p2, f2, k.c0);
@@ -323,7 +360,7 @@ __device__ __forceinline__ void stage_row_chunk(uint32_t stage_out, int c, int r
   }
 }
 
-template <int D, int TKV, int NQ>
+template <int D, int TKV, int NQ, bool CAUSAL>
 __global__ void __launch_bounds__(512, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -355,7 +392,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // head, so K/V are shared through L2.
   const int cta = blockIdx.x;
   const long long G = gridDim.x;
-  const long long T = (long long)p.tiles * p.n_steps;
+  const long long T = p.head_units * (p.tiles / p.q_tiles);
   const long long u_lo = range_begin(cta, T, G), u_hi = range_begin(cta + 1, T, G);
 
   ATTN_TRACE_CTA(0);
@@ -431,14 +468,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       long long u = u_lo;
       int seg_ctr = 0;
       Segment sg;
-      while (ok && next_segment(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, NQ * kSub, sg)) {
+      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg)) {
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
       float m_run = -INFINITY, delta = 0.f;
-      // One KV step of this sub-tile.  The ragged variant (last KV tile of a sequence whose length is
-      // not a multiple of the tile) is compiled separately so that the common step pays nothing for it.
-      auto softmax_step = [&](auto ragged_tag) -> bool {
-        constexpr bool kRagged = decltype(ragged_tag)::value;
+      // One KV step of this sub-tile.  The masked variant (a ragged last KV tile, or a causal step that
+      // reaches past the sub-tile's first row) is compiled separately so that the common step pays
+      // nothing for it; `lim` is the last key column of this step the thread's row may attend to.
+      auto softmax_step = [&](auto mask_tag, int lim) __attribute__((always_inline)) -> bool {
+        constexpr bool kMasked = decltype(mask_tag)::value;
         if (!wait_bar_warp(bar_s, g & 1, abort_flag, wait_info(kRoleSoftmax, kBarSFull, g))) return false;
         tc_fence_after();
         if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 0);
@@ -451,22 +489,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int c = 0; c < NCH / 2; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
 #pragma unroll
         for (int c = NCH / 2; c < NCH; ++c) tmem_ld32_nowait(s_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-        // Ragged last KV tile: keys past the end of the sequence were zero-filled by TMA, which would give
-        // them score 0 and weight exp(0 - m) > 0; their scores are set to -inf instead (never zero padding).
-        if constexpr (kRagged) {
+        // Masked keys -- past the end of the sequence (zero-filled by TMA, which would give them score 0
+        // and weight exp(0 - m) > 0) or after the query's position (causal) -- get score -inf, never zero.
+        if constexpr (kMasked) {
 #pragma unroll
           for (int k = 0; k < TKV / 2; ++k)
-            if (k >= kv_tail) s[k] = 0xFF800000u;
+            if (k > lim) s[k] = 0xFF800000u;
         }
         const float mx_a = fmaxf(fmaxf(chain_max<0, TKV / 8>(s), chain_max<TKV / 8, TKV / 4>(s)),
                                  fmaxf(chain_max<TKV / 4, 3 * TKV / 8>(s), chain_max<3 * TKV / 8, TKV / 2>(s)));
 #pragma unroll
         for (int c = NCH / 2; c < NCH; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
         if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 1);
-        if constexpr (kRagged) {
+        if constexpr (kMasked) {
 #pragma unroll
           for (int k = TKV / 2; k < TKV; ++k)
-            if (k >= kv_tail) s[k] = 0xFF800000u;
+            if (k > lim) s[k] = 0xFF800000u;
         }
         const float mx_b = fmaxf(fmaxf(chain_max<TKV / 2, 5 * TKV / 8>(s), chain_max<5 * TKV / 8, 3 * TKV / 4>(s)),
                                  fmaxf(chain_max<3 * TKV / 4, 7 * TKV / 8>(s), chain_max<7 * TKV / 8, TKV>(s)));
@@ -480,7 +518,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         //      whole row.  For flat score distributions (b) stops firing after the first few tiles.
         // Otherwise the reference stays stale, which changes nothing in exact arithmetic because
         // delta and O carry the same factor.  First step: m_run = -inf, gap = +inf, alpha = 0.
-        const float m_cand = fmaxf(m_run, mx * scale);
+        // (masked steps can leave a row with no admissible key yet: keep the reference finite)
+        const float m_cand = kMasked ? fmaxf(fmaxf(m_run, mx * scale), -1e30f) : fmaxf(m_run, mx * scale);
         const float gap = m_cand - m_run;
         const float shrink = ex2_approx(-gap);             // 2^-gap: the rescale factor if the reference moves
         const bool move = (gap > kRescaleThreshold) || (gap > 0.f && kDominanceFactor > delta * shrink);
@@ -524,8 +563,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               return true;
       };
       for (int jj = 0; ok && jj < n; ++jj, ++g) {
-        const bool ragged = (kv_tail != 0) && (j0 + jj == p.n_steps - 1);
-        ok = ragged ? softmax_step(RaggedTag<true>{}) : softmax_step(RaggedTag<false>{});
+        const int j = j0 + jj;
+        const bool ragged = (kv_tail != 0) && (j == p.n_steps - 1);
+        const bool diagonal = CAUSAL && ((j + 1) * TKV - 1 > q_row0 + i * kSub);   // warp-uniform
+        if (ragged || diagonal) {
+          int lim = ragged ? kv_tail - 1 : TKV - 1;
+          if (CAUSAL) {
+            const int cl = q_row0 + i * kSub + row - j * TKV;     // may be negative: nothing admissible
+            if (cl < lim) lim = cl;
+          }
+          ok = softmax_step(MaskTag<true>{}, lim);
+        } else {
+          ok = softmax_step(MaskTag<false>{}, TKV - 1);
+        }
       }
       // ----------------------------------------------------- end of segment
       if (warp == 0) ATTN_TRACE_MARK(3);
@@ -533,10 +583,44 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (!ok) break;
       tc_fence_after();
       if (warp == 0) ATTN_TRACE_MARK(4);
-      if (j0 == 0 && j1 == p.n_steps) {
-        // The whole Q tile was processed here: normalise and store through shared memory (TMA).
+      const bool last_seg = (u >= u_hi);                     // u was advanced past this segment already
+      const int grow = q_row0 + i * kSub + row;              // this thread's row in the sequence
+      // Normalised values of one output row chunk -> memory.  On the CTA's last segment the Q buffer is
+      // dead and the rows go through shared memory and a TMA store; otherwise the next segment's Q tile
+      // may already be arriving there and the rows are stored from registers.
+      auto put_chunk = [&](int c, const float (&val)[32]) {
+        if (last_seg) {
+          stage_row_chunk(q_smem + i * (kSub * D * 2), c, row, val);
+        } else if (grow < p.L) {
+          uint4* orow = reinterpret_cast<uint4*>(p.o + ((size_t)bh * p.L + grow) * D) + c * 4;
+#pragma unroll
+          for (int u4 = 0; u4 < 4; ++u4) {
+            uint4 w4;
+            w4.x = pack_bf16x2(val[u4 * 8 + 0], val[u4 * 8 + 1]);
+            w4.y = pack_bf16x2(val[u4 * 8 + 2], val[u4 * 8 + 3]);
+            w4.z = pack_bf16x2(val[u4 * 8 + 4], val[u4 * 8 + 5]);
+            w4.w = pack_bf16x2(val[u4 * 8 + 6], val[u4 * 8 + 7]);
+            orow[u4] = w4;
+          }
+        }
+      };
+      auto finish_rows = [&]() -> bool {                     // after put_chunk on the last segment
+        if (!last_seg) return true;
+        const uint32_t stage_out = q_smem + i * (kSub * D * 2);
+        fence_proxy_async_smem();
+        const bool r = wg_sync(3);
+        if (r && (warp & 3) == 0 && lane == 0) {
+#pragma unroll
+          for (int c = 0; c < KCH; ++c)
+            tma_store_3d(&tm_o, stage_out + c * (kSub * 128), c * 64, q_row0 + i * kSub, bh);
+          tma_store_commit();
+          tma_store_wait_read();
+        }
+        return r;
+      };
+      if (sg.full) {
+        // The whole Q tile was processed here: normalise and store.
         const float inv = 1.0f / delta;
-        const uint32_t stage_out = q_smem + i * (kSub * D * 2);   // Q sub-tile is dead: reuse it
 #pragma unroll 1
         for (int c = 0; c < D / 32; ++c) {
           uint32_t r[32];
@@ -544,22 +628,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tmem_ld32(o_tmem + c * 32, r);
 #pragma unroll
           for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(r[k]) * inv;
-          stage_row_chunk(stage_out, c, row, val);
+          put_chunk(c, val);
         }
         tc_fence_before();
         mbar_arrive(smem_u32(&misc->o_free[i]));             // O may be overwritten by the next segment
-        fence_proxy_async_smem();
-        ok = wg_sync(3);
-        if (ok && (warp & 3) == 0 && lane == 0) {
-#pragma unroll
-          for (int c = 0; c < KCH; ++c)
-            tma_store_3d(&tm_o, stage_out + c * (kSub * 128), c * 64, q_row0 + i * kSub, bh);
-          tma_store_commit();
-          tma_store_wait_read();
-        }
+        ok = finish_rows();
       } else {
-        // Part of a Q tile: un-normalised partial (O, m, delta) of this key range into slot cta + tile.
-        float* ws = p.ws + ((size_t)(cta + tile) * NQ + i) * per_sub;
+        // Part of a Q tile: un-normalised partial (O, m, delta) of this key range.  A CTA has at most two
+        // such pieces, its first and its last segment: slots 2*cta and 2*cta + 1.
+        float* ws = p.ws + ((size_t)(2 * cta + (seg == 0 ? 0 : 1)) * NQ + i) * per_sub;
         {
           uint32_t r[D];
 #pragma unroll
@@ -579,35 +656,39 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         ws[(size_t)kSub * D + kSub + row] = delta;
         __threadfence();
         if (warp == 0) ATTN_TRACE_MARK(5);
+        // CTAs that share this Q tile: those whose ranges meet the tile's units; the first of them owns
+        // the tile's arrival counter.
+        const int c_first = cta_of_unit(sg.unit0, T, G);
+        const int c_last = cta_of_unit(sg.unit0 + sg.steps_t - 1, T, G);
         ok = wg_sync(1);
         if (ok) {
-          if (row == 0) misc->ticket[i] = atomicAdd(&p.counters[tile * NQ + i], 1u);
+          if (row == 0) misc->ticket[i] = atomicAdd(&p.counters[c_first * NQ + i], 1u);
           ok = wg_sync(2);
         }
         if (!ok) break;
-        // CTAs that share this Q tile: those whose ranges meet [tile*n_steps, (tile+1)*n_steps)
         if (warp == 0) ATTN_TRACE_MARK(6);
-        const int c_first = cta_of_unit((long long)tile * p.n_steps, T, G);
-        const int c_last = cta_of_unit((long long)(tile + 1) * p.n_steps - 1, T, G);
         if (*reinterpret_cast<volatile uint32_t*>(&misc->ticket[i]) == (uint32_t)(c_last - c_first)) {
           // Last one to finish: merge all parts in ascending key order (the merge operator of the
           // online softmax), independent of arrival order, and write the rows of this sub-tile.
-          if (row == 0) p.counters[tile * NQ + i] = 0u;
+          if (row == 0) p.counters[c_first * NQ + i] = 0u;
           __threadfence();
-          const float* part0 = p.ws + ((size_t)(c_first + tile) * NQ + i) * per_sub;
-          const size_t part_stride = (size_t)NQ * per_sub;
           const int parts = c_last - c_first + 1;
+          // part sp comes from CTA c_first + sp: its first piece if its range starts inside this tile
+          auto part_ptr = [&](int sp) -> const float* {
+            const int c = c_first + sp;
+            const int slot = (range_begin(c, T, G) >= sg.unit0) ? 0 : 1;
+            return p.ws + ((size_t)(2 * c + slot) * NQ + i) * per_sub;
+          };
           float m_all = -INFINITY;
 #pragma unroll 4
-          for (int sp = 0; sp < parts; ++sp)
-            m_all = fmaxf(m_all, __ldcg(part0 + sp * part_stride + (size_t)kSub * D + row));
+          for (int sp = 0; sp < parts; ++sp) m_all = fmaxf(m_all, __ldcg(part_ptr(sp) + (size_t)kSub * D + row));
           // whole output row accumulated in registers: per part all loads are independent and in flight together
           float val[D];
 #pragma unroll
           for (int k = 0; k < D; ++k) val[k] = 0.f;
           float d_all = 0.f;
           for (int sp = 0; sp < parts; ++sp) {
-            const float* b = part0 + sp * part_stride;
+            const float* b = part_ptr(sp);
             const float w = exp2f(__ldcg(b + (size_t)kSub * D + row) - m_all);
             d_all += __ldcg(b + (size_t)kSub * D + kSub + row) * w;
 #pragma unroll
@@ -622,36 +703,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const float inv = 1.0f / d_all;
 #pragma unroll
           for (int k = 0; k < D; ++k) val[k] *= inv;
-          if (u >= u_hi) {
-            // last segment of this CTA: the Q buffer is dead, store through shared memory (TMA)
-            const uint32_t stage_out = q_smem + i * (kSub * D * 2);
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) stage_row_chunk(stage_out, c, row, *reinterpret_cast<float(*)[32]>(&val[c * 32]));
-            fence_proxy_async_smem();
-            ok = wg_sync(3);
-            if (ok && (warp & 3) == 0 && lane == 0) {
-#pragma unroll
-              for (int c = 0; c < KCH; ++c)
-                tma_store_3d(&tm_o, stage_out + c * (kSub * 128), c * 64, q_row0 + i * kSub, bh);
-              tma_store_commit();
-              tma_store_wait_read();
-            }
-          } else {
-            // another segment follows and its Q tile may already be arriving: store from registers
-            const int grow = q_row0 + i * kSub + row;
-            if (grow < p.L) {
-              uint4* orow = reinterpret_cast<uint4*>(p.o + ((size_t)bh * p.L + grow) * D);
-#pragma unroll
-              for (int u4 = 0; u4 < D / 8; ++u4) {
-                uint4 w4;
-                w4.x = pack_bf16x2(val[u4 * 8 + 0], val[u4 * 8 + 1]);
-                w4.y = pack_bf16x2(val[u4 * 8 + 2], val[u4 * 8 + 3]);
-                w4.z = pack_bf16x2(val[u4 * 8 + 4], val[u4 * 8 + 5]);
-                w4.w = pack_bf16x2(val[u4 * 8 + 6], val[u4 * 8 + 7]);
-                orow[u4] = w4;
-              }
-            }
-          }
+          for (int c = 0; c < D / 32; ++c) put_chunk(c, *reinterpret_cast<float(*)[32]>(&val[c * 32]));
+          ok = finish_rows();
         }
       }
       }
@@ -667,7 +721,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       long long u = u_lo;
       int seg_ctr = 0;
       Segment sg;
-      while (ok && next_segment(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, NQ * kSub, sg)) {
+      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg)) {
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
       for (int jj = 0; ok && jj < n; ++jj, ++g) {
@@ -723,7 +777,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       long long u = u_lo;
       int seg_ctr = 0;
       Segment sg;
-      while (ok && next_segment(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, NQ * kSub, sg)) {
+      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg)) {
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
       ok = wait_bar_warp(smem_u32(&misc->q_full), seg & 1, abort_flag, wait_info(kRoleMma, kBarQ, seg));
@@ -809,7 +863,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       long long u = u_lo;
       int seg_ctr = 0;
       Segment sg;
-      while (ok && next_segment(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, NQ * kSub, sg)) {
+      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg)) {
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
         if (seg > 0 &&

@@ -56,15 +56,32 @@ inline int register_machine_regs(int t_q, int t_kv, int d, int simd) {
 
 }  // namespace
 
+// Work units of one head: every Q tile takes all `steps` KV steps, or -- causal -- only the steps whose
+// keys are not after the tile's last row, min(steps, (q+1)*ratio): a triangular number until that saturates.
+long long attn_internal::head_units(int q_tiles, int steps, int ratio, int causal) {
+  if (!causal) return (long long)q_tiles * steps;
+  long long qc = steps / ratio;
+  if (qc > q_tiles) qc = q_tiles;
+  return (long long)ratio * qc * (qc + 1) / 2 + (long long)(q_tiles - qc) * steps;
+}
+
 // Occupancy step of the derivation (shared with the tile-override path of the launcher).
-int attn_internal::grid_size(const attn_hw_desc& h, int tiles, int steps) {
+int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int steps, int ratio, int causal) {
+  const long long tiles_ll = (long long)heads * q_tiles;
+  const long long total = (long long)heads * head_units(q_tiles, steps, ratio, causal);
+  if (causal) {
+    long long g = total / kMinStepsPerSplit;
+    if (g > h.num_units) g = h.num_units;
+    if (g < 1) g = 1;
+    return (int)g;
+  }
+  const int tiles = (int)tiles_ll;
   if (tiles >= h.num_units) return tiles;
   int k = h.num_units / tiles;
   const int k_max = steps / kMinStepsPerSplit;
   if (k > k_max) k = k_max;
   if (k < 1) k = 1;
   const int cost_uniform = ceil_div(steps, k) + kSegmentOverheadSteps;
-  const long long total = (long long)tiles * steps;
   long long g = total / kMinStepsPerSplit;
   if (g > h.num_units) g = h.num_units;
   int ctas = tiles * k;
@@ -105,7 +122,7 @@ void plan_register_machine(const attn_hw_desc& h, int B, int H, int L, int d, at
   t->under_occupied = t->tiles < h.num_units;
 }
 
-void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, attn_tiles* t) {
+void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, int causal, attn_tiles* t) {
   const int sub = h.atom_m;  // one tensor-memory lane per Q row
   t->binding_constraint = ATTN_BIND_SHAPE;
   if (d % h.atom_k || d % h.atom_n || d > h.atom_n_max) return;
@@ -154,7 +171,7 @@ void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, attn_t
   const int tiles = B * H * ceil_div(L, tile_q);
   const int steps = ceil_div(L, tile_kv);
   const int under = tiles < h.num_units;
-  const int ctas = attn_internal::grid_size(h, tiles, steps);
+  const int ctas = attn_internal::grid_size(h, B * H, ceil_div(L, tile_q), steps, tile_q / tile_kv, causal);
   const int kv_splits = ceil_div(ctas, tiles);
 
   t->feasible = 1;
@@ -176,6 +193,7 @@ void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, attn_t
   const int waves = ceil_div(t->ctas, h.num_units);
   t->wave_efficiency = (float)((double)t->ctas / ((double)waves * h.num_units));
   t->under_occupied = under;
+  t->causal = causal ? 1 : 0;
 }
 
 }  // namespace
@@ -203,6 +221,10 @@ extern "C" int attn_hw_desc_b200(attn_hw_desc* out) {
 }
 
 extern "C" int attn_plan(const attn_hw_desc* desc, int B, int H, int L, int d, attn_tiles* out) {
+  return attn_plan_ex(desc, B, H, L, d, 0, out);
+}
+
+extern "C" int attn_plan_ex(const attn_hw_desc* desc, int B, int H, int L, int d, int causal, attn_tiles* out) {
   if (!desc || !out) return ATTN_ERR_INVALID_ARG;
   if (desc->struct_bytes != (int32_t)sizeof(attn_hw_desc)) return ATTN_ERR_INVALID_ARG;
   std::memset(out, 0, sizeof(*out));
@@ -212,7 +234,7 @@ extern "C" int attn_plan(const attn_hw_desc* desc, int B, int H, int L, int d, a
       desc->atom_k <= 0 || desc->elem_bytes <= 0 || desc->simd_width <= 0 || desc->max_regs_per_thread <= 16)
     return ATTN_ERR_INVALID_ARG;
   if (desc->acc_mem_columns > 0)
-    plan_tmem_machine(*desc, B, H, L, d, out);
+    plan_tmem_machine(*desc, B, H, L, d, causal, out);
   else
     plan_register_machine(*desc, B, H, L, d, out);
   return ATTN_OK;
@@ -220,9 +242,9 @@ extern "C" int attn_plan(const attn_hw_desc* desc, int B, int H, int L, int d, a
 
 extern "C" size_t attn_workspace_bytes(const attn_tiles* t, int B, int H, int L, int d) {
   (void)B; (void)H; (void)L;
-  if (!t || !t->feasible || t->ctas <= t->tiles || t->n_q <= 0) return 0;
-  // 64 KB of arrival counters, then one slot per (CTA, Q tile) piece -- at most ctas + tiles of
-  // them -- and sub-tile: 128 x d fp32 un-normalised output + 128 (m, delta) pairs.
+  if (!t || !t->feasible || t->n_q <= 0 || (t->ctas == t->tiles && !t->causal)) return 0;
+  // 64 KB of arrival counters, then two slots per CTA (its first and its last piece of a Q tile) and
+  // sub-tile: 128 x d fp32 un-normalised output + 128 (m, delta) pairs.
   const size_t per_sub = (size_t)128 * (size_t)d * 4 + (size_t)128 * 2 * 4;
-  return (size_t)65536 + ((size_t)t->ctas + (size_t)t->tiles) * (size_t)t->n_q * per_sub;
+  return (size_t)65536 + (size_t)2 * (size_t)t->ctas * (size_t)t->n_q * per_sub;
 }

@@ -33,7 +33,7 @@ def _case(name, B, H, L, d, sigma_qk=1.0, cfg_id=50):
     return synth.AttnCase(name, B, H, L, d, sigma_qk=sigma_qk, cfg_id=cfg_id)
 
 
-def _run_and_compare(env, case, runner, rows=None, what=""):
+def _run_and_compare(env, case, runner, rows=None, what="", causal=False):
     torch, orc, binding = env
     q, k, v = synth.make_qkv(case, seed=0)
     tq, tk, tv = (to_cuda_bf16(x) for x in (q, k, v))
@@ -43,7 +43,7 @@ def _run_and_compare(env, case, runner, rows=None, what=""):
     assert code == 0, f"{what}: device status {code} detail {detail}"
     got = to_host_f64(out).reshape(case.B * case.H, case.L, case.d)
     rows = np.arange(case.L, dtype=np.int32) if rows is None else rows
-    ref = orc.attention_rows(q, k, v, case.B, case.H, case.L, case.d, rows)
+    ref = orc.attention_rows(q, k, v, case.B, case.H, case.L, case.d, rows, causal=causal)
     stats = assert_close(got[:, rows], ref, what or case.name)
     # whole-output properties that hold at any size: finite, inside the per-column hull of V
     vf = to_host_f64(tv).reshape(case.B * case.H, case.L, case.d)
@@ -166,18 +166,66 @@ def test_zero_padding_would_show(env):
     assert np.abs(ref).mean() > 2.0        # the correct answer is the mean of V (~3), not ~0
 
 
-@pytest.mark.parametrize("ctas", [12, 13, 17, 29, 64, 131])
+@pytest.mark.parametrize("ctas", [1, 3, 5, 12, 13, 17, 29, 64, 131])
 @pytest.mark.parametrize("d,n_q,tile_kv", [(128, 2, 128), (64, 2, 128), (128, 1, 64)])
 def test_balanced_key_ranges_any_grid_size(env, d, n_q, tile_kv, ctas):
-    """Grid sizes that cut the (Q tile, KV step) line at arbitrary places: ranges that straddle a tile
-    boundary (two segments per CTA), tiles shared by two to many CTAs, tiles owned by a single CTA."""
+    """Grid sizes that cut the (Q tile, KV step) line at arbitrary places: ranges that straddle tile
+    boundaries (several segments per CTA, whole tiles in the middle), tiles shared by two to many CTAs,
+    tiles owned by a single CTA, one CTA doing everything."""
     _, _, binding = env
     case = _case("ranges", 1, 2, 1408, d, sigma_qk=math.sqrt(3.0))
-    tiles = 2 * math.ceil(1408 / (128 * n_q))
-    if ctas < tiles:
-        pytest.skip("fewer CTAs than Q tiles is not a supported launch")
     run = lambda a, b, c: binding.forward_tiles(a, b, c, n_q=n_q, tile_kv=tile_kv, ctas=ctas)
     _run_and_compare(env, case, run)
+
+
+# --------------------------------------------------------------------------- causal
+@pytest.mark.parametrize("L", [1, 3, 64, 128, 129, 200, 256, 257, 640, 1000, 1408, 2049])
+@pytest.mark.parametrize("d", [64, 128])
+def test_causal_matches_oracle(env, d, L):
+    """Row i attends to keys 0..i: diagonal tiles masked with -inf, key steps after a Q tile skipped."""
+    _, _, binding = env
+    case = _case("causal", 1, 3, L, d, sigma_qk=1.5)
+    _run_and_compare(env, case, lambda a, b, c: binding.forward(a, b, c, causal=True), causal=True)
+
+
+@pytest.mark.parametrize("kw", [dict(ctas=1), dict(ctas=2), dict(ctas=7), dict(ctas=37), dict(ctas=101),
+                                dict(tile_kv=64), dict(n_q=1), dict(n_q=1, tile_kv=64, ctas=53), dict(kv_stages=2)])
+def test_causal_tile_variants_and_grid_sizes(env, kw):
+    _, _, binding = env
+    case = _case("causal_variants", 2, 2, 1100, 128, sigma_qk=math.sqrt(3.0))
+    _run_and_compare(env, case, lambda a, b, c: binding.forward_tiles(a, b, c, causal=True, **kw), causal=True)
+
+
+def test_causal_structured_and_reproducible(env):
+    torch, orc, binding = env
+    L, d = 512, 128
+    rng = np.random.default_rng(5)
+    rnd = lambda: synth.f32_to_bf16_bits(rng.standard_normal((1, 1, L, d), dtype=np.float32))
+    qb, kb, vb = rnd(), rnd(), rnd()
+    q, k, v = (to_cuda_bf16(x) for x in (qb, kb, vb))
+    a = binding.forward(q, k, v, causal=True)
+    b = binding.forward(q, k, v, causal=True)
+    torch.cuda.synchronize()
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    out = to_host_f64(a).reshape(L, d)
+    # row 0 sees only key 0: the output is V[0] exactly (one weight, equal to 1)
+    assert np.array_equal(out[0], orc.bf16_bits_to_f64(vb).reshape(L, d)[0])
+    # changing keys/values after position 300 must not change rows 0..300
+    kb2, vb2 = kb.copy(), vb.copy()
+    kb2[:, :, 301:] = rnd()[:, :, 301:]
+    vb2[:, :, 301:] = rnd()[:, :, 301:]
+    c = to_host_f64(binding.forward(q, to_cuda_bf16(kb2), to_cuda_bf16(vb2), causal=True)).reshape(L, d)
+    assert np.array_equal(c[:301], out[:301]) and np.abs(c[301:] - out[301:]).max() > 1e-3
+
+
+def test_causal_full_size_sampled_rows(env):
+    _, _, binding = env
+    case = synth.CONFIGS["cfg3"]
+    _run_and_compare(env, case, lambda a, b, c: binding.forward(a, b, c, causal=True),
+                     rows=synth.sample_rows(case.L), causal=True)
+    case = synth.CONFIGS["cfg5a"]
+    _run_and_compare(env, case, lambda a, b, c: binding.forward(a, b, c, causal=True),
+                     rows=synth.sample_rows(case.L), causal=True)
 
 
 def test_two_kernels_agree_and_runs_are_bitwise_reproducible(env):

@@ -41,6 +41,7 @@ def test_struct_sizes_match_the_header(binding):
     d = binding.hw_desc_b200()
     assert d.struct_bytes == ctypes.sizeof(binding.AttnHwDesc) == 80
     assert ctypes.sizeof(binding.AttnTiles) == 72
+    assert binding.AttnTiles.causal.offset == 68
 
 
 def _desc_dict(d):
@@ -64,6 +65,10 @@ def test_b200_plan_equals_oracle_restatement(binding):
         assert bool(got.under_occupied) == ref["under_occupied"]
         assert got.wave_efficiency == pytest.approx(ref["wave_efficiency"], rel=1e-6)
         assert got.ctas_per_unit == pytest.approx(ref["ctas_per_unit"], rel=1e-6)
+        gc = binding.plan(desc, B, H, L, d, causal=True)
+        rc = po.derive_tiles_tmem_machine(dd, B, H, L, d, causal=True)
+        assert (gc.feasible, gc.causal, gc.tile_q, gc.tile_kv, gc.kv_stages, gc.ctas) == (
+            1, 1, rc["tile_q"], rc["tile_kv"], rc["kv_stages"], rc["ctas"]), (B, H, L, d)
 
 
 def test_other_descriptors_rerun_the_same_derivation(binding):
@@ -120,7 +125,7 @@ def test_workspace_bytes(binding):
     desc = binding.hw_desc_b200()
     t = binding.plan(desc, 1, 1, 16384, 128)
     assert (t.tiles, t.ctas) == (64, 148)
-    assert binding.workspace_bytes(t, 1, 1, 16384, 128) == 65536 + (t.ctas + t.tiles) * 2 * (128 * 128 + 256) * 4
+    assert binding.workspace_bytes(t, 1, 1, 16384, 128) == 65536 + 2 * t.ctas * 2 * (128 * 128 + 256) * 4
     t1 = binding.plan(desc, 4, 32, 4096, 128)
     assert binding.workspace_bytes(t1, 4, 32, 4096, 128) == 0
 

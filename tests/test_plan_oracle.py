@@ -75,6 +75,8 @@ def test_tmem_machine_capacity_invariants(B, H, L, d):
     assert regs_total <= 65536 and t["regs_softmax"] <= 248
     assert t["tile_kv"] + t["tile_kv"] // 4 + 32 <= t["regs_softmax"]
     assert t["tiles"] <= t["ctas"] <= t["tiles"] * t["kv_splits"]
+    tc = po.derive_tiles_tmem_machine(B200, B, H, L, d, causal=True)
+    assert tc["feasible"] and 1 <= tc["ctas"] <= 148 and tc["tile_kv"] == t["tile_kv"] and tc["tile_q"] == t["tile_q"]
     assert 0 < t["wave_efficiency"] <= 1.0
     if t["ctas"] > t["tiles"]:
         assert t["under_occupied"] and t["ctas"] <= 148

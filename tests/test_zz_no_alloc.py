@@ -39,7 +39,7 @@ def test_static_scratch_entry_point_matches_attn_forward_twice_in_a_row():
     for case in cases:
         plan = binding.plan(desc, case.B, case.H, case.L, case.d)
         assert plan.feasible and plan.kv_splits > 1, "test shape no longer exercises the scratch path"
-        assert binding.workspace_bytes(plan, case.B, case.H, case.L, case.d) <= 39335936
+        assert binding.workspace_bytes(plan, case.B, case.H, case.L, case.d) <= 39469056
         q, k, v = (to_cuda_bf16(x) for x in synth.make_qkv(case, seed=5))
         want = binding.forward(q, k, v)                  # existing entry point (caller-owned workspace)
         got = torch.full_like(q, float("nan"))           # every element must be overwritten
