@@ -82,7 +82,7 @@ typedef struct attn_hw_desc {
   int32_t atom_k;              /* K of one instruction (16 | 4)                       */
   int32_t atom_n_max;          /* largest N of one instruction (256 | 16)             */
   int32_t elem_bytes;          /* operand element size (2 = bf16, 4 = fp32)           */
-  int32_t reserved;
+  int32_t cache_bytes;         /* last-level cache shared by all units (L2); 0 if not modelled */
   double hbm_gbps;             /* sustained HBM bandwidth, GB/s                       */
   double peak_tflops;          /* dense tensor peak for the operand type, TFLOP/s     */
   double sm_clock_mhz;         /* maximum SM clock                                    */
@@ -95,13 +95,14 @@ typedef struct attn_tiles {
   int32_t n_q;            /* Q sub-tiles per CTA (ping-pong partners), 1 or 2           */
   int32_t n_s;            /* score buffers per sub-tile (1)                             */
   int32_t kv_stages;      /* depth of the shared-memory K/V ring (one K or V tile each) */
-  int32_t kv_splits;      /* most CTAs sharing one Q tile along the key axis = ceil(ctas / tiles) */
+  int32_t kv_splits;      /* ceil(ctas / tiles): CTAs sharing one Q tile along the key axis (1 for a persistent
+                             grid of fewer CTAs than tiles; a tile at a range boundary is then still shared by two) */
   int32_t smem_bytes;     /* dynamic shared memory per CTA                              */
   int32_t tmem_columns;   /* tensor-memory columns allocated per CTA                    */
   int32_t regs_softmax;   /* register allowance of a softmax thread                     */
   int32_t threads;        /* threads per CTA                                            */
   int32_t tiles;          /* B * H * ceil(L / tile_q)                                   */
-  int32_t ctas;           /* grid size: tiles, or min(num_units, tiles*steps/4) if under-occupied */
+  int32_t ctas;           /* grid size: tiles, or fewer/more CTAs walking equal ranges of the (tile, step) line */
   float ctas_per_unit;    /* ctas / num_units                                           */
   float wave_efficiency;  /* ctas_per_unit / ceil(ctas_per_unit)                        */
   int32_t feasible;       /* 1 if a tile choice fits                                    */

@@ -58,12 +58,15 @@ def derive_tiles_register_machine(lds_bytes, regs_per_thread, wavefront, num_uni
 _REGS_CORRECTION = 64      # per thread, correction warpgroup
 _REGS_OTHER = 64           # per thread, TMA / MMA-issue warpgroup
 _REGS_ROW_OVERHEAD = 32    # softmax thread: addresses, row statistics, loop state
-_SMEM_RESERVE = 3072       # barriers, rescale factors, tensor-memory slot
+_SMEM_MISC = 3072          # barriers, rescale factors, tensor-memory slot
+_OUT_ROW_BYTES = 128       # output staging: per softmax warpgroup 64 bf16 columns of each of its rows
 _MAX_STAGES = 8
 _MIN_STAGES = 4
 _MIN_TILE_KV = 32
 _MIN_STEPS_PER_SPLIT = 4
 _SEGMENT_OVERHEAD_STEPS = 3
+_CTA_OVERHEAD_STEPS = 2     # start and end of a CTA that handles one whole Q tile
+_TRANSITION_STEPS = 1       # a persistent CTA moving on to its next Q tile
 
 
 def causal_head_units(q_tiles: int, steps: int, ratio: int) -> int:
@@ -95,9 +98,10 @@ def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal
         out["binding"] = binding
         return out
     q_bytes = n_q * sub * d * desc["elem_bytes"]
+    reserve = _SMEM_MISC + n_q * sub * _OUT_ROW_BYTES
     while True:
         stage = tile_kv * d * desc["elem_bytes"]
-        stages = min((desc["local_mem_bytes"] - q_bytes - _SMEM_RESERVE) // stage, _MAX_STAGES)
+        stages = min((desc["local_mem_bytes"] - q_bytes - reserve) // stage, _MAX_STAGES)
         if stages >= _MIN_STAGES:
             break
         tile_kv //= 2
@@ -110,6 +114,7 @@ def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal
     steps = -(-L // tile_kv)
     under = tiles < desc["num_units"]
     ctas = tiles
+    kv_head_bytes = 2 * L * d * desc["elem_bytes"]            # K and V of one head
     if causal:
         total = B * H * causal_head_units(-(-L // tile_q), steps, tile_q // tile_kv)
         ctas = max(1, min(total // _MIN_STEPS_PER_SPLIT, desc["num_units"]))
@@ -123,12 +128,24 @@ def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal
             cost_balanced = -(-total // g) + 2 * _SEGMENT_OVERHEAD_STEPS
             if cost_balanced < cost_uniform:
                 ctas = g
+    else:
+        # enough tiles for every unit: one CTA per tile (whole waves, each CTA its own start and end), or one
+        # persistent CTA per unit on an equal range of the (tile, step) line -- only if the K/V of the heads
+        # then in flight stay inside two thirds of the last-level cache
+        units = desc["num_units"]
+        total = tiles * steps
+        cost_tiles = -(-tiles // units) * (steps + _CTA_OVERHEAD_STEPS)
+        cost_balanced = -(-total // units) + 2 * _SEGMENT_OVERHEAD_STEPS + -(-tiles // units) * _TRANSITION_STEPS
+        in_flight = min(B * H, units)
+        cached = desc.get("cache_bytes", 0) > 0 and 3 * in_flight * kv_head_bytes <= 2 * desc["cache_bytes"]
+        if cached and cost_balanced < cost_tiles:
+            ctas = units
     kv_splits = -(-ctas // tiles)
     per_unit = ctas / desc["num_units"]
     cols = n_q * (tile_kv + d)
     return dict(feasible=True, binding=binding, tile_q=tile_q, tile_kv=tile_kv, n_q=n_q, n_s=1,
                 kv_stages=stages, kv_splits=kv_splits,
-                smem_bytes=q_bytes + stages * stage + _SMEM_RESERVE,
+                smem_bytes=q_bytes + stages * stage + reserve,
                 tmem_columns=max(32, 1 << (cols - 1).bit_length()), regs_softmax=regs_soft,
                 threads=threads, tiles=tiles, ctas=ctas, ctas_per_unit=per_unit,
                 wave_efficiency=per_unit / math.ceil(per_unit), under_occupied=under)

@@ -192,7 +192,8 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
     if (t.n_q != 1 && t.n_q != 2) return ATTN_ERR_BAD_TILES;
     if (t.tile_kv != 64 && t.tile_kv != 128) return ATTN_ERR_BAD_TILES;
     const int q_bytes = t.n_q * 128 * d * 2, stage = t.tile_kv * d * 2;
-    int max_stages = (st->desc.local_mem_bytes - q_bytes - 3072) / stage;
+    const int reserve = 3072 + t.n_q * 128 * 128;   // barriers etc. + output staging (see FwdSmem)
+    int max_stages = (st->desc.local_mem_bytes - q_bytes - reserve) / stage;
     if (max_stages > attn::kMaxStages) max_stages = attn::kMaxStages;
     t.kv_stages = ovr->kv_stages > 0 ? ovr->kv_stages : max_stages;
     if (t.kv_stages < 2 || t.kv_stages > max_stages) return ATTN_ERR_BAD_TILES;
@@ -206,11 +207,12 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
     } else if (ovr->kv_splits > 0) {
       t.ctas = t.tiles * ovr->kv_splits;
     } else {
-      t.ctas = attn_internal::grid_size(st->desc, B * H, (L + t.tile_q - 1) / t.tile_q, steps, t.tile_q / t.tile_kv, causal);
+      t.ctas = attn_internal::grid_size(st->desc, B * H, (L + t.tile_q - 1) / t.tile_q, steps, t.tile_q / t.tile_kv, causal,
+                                        2LL * L * d * st->desc.elem_bytes);
     }
     t.kv_splits = (t.ctas + t.tiles - 1) / t.tiles;
     if (t.ctas < 1) return ATTN_ERR_BAD_TILES;
-    t.smem_bytes = q_bytes + t.kv_stages * stage + 3072;
+    t.smem_bytes = q_bytes + t.kv_stages * stage + reserve;
   }
   float* ws = nullptr;
   if (plan_needs_workspace(t)) {
@@ -256,6 +258,9 @@ extern "C" int attn_hw_desc_query(int device, attn_hw_desc* out) {
   ATTN_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
   ATTN_CUDA_TRY(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
   ATTN_CUDA_TRY(cudaDeviceGetAttribute(&regs, cudaDevAttrMaxRegistersPerMultiprocessor, device));
+  int l2 = 0;
+  ATTN_CUDA_TRY(cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, device));
+  if (l2 > 0) out->cache_bytes = l2;
   ATTN_CUDA_TRY(cudaDeviceGetAttribute(&clock_khz, cudaDevAttrClockRate, device));
   out->num_units = sms;
   out->local_mem_bytes = smem_optin;

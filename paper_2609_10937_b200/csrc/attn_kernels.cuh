@@ -41,7 +41,10 @@ enum BarId : uint32_t { kBarQ = 1, kBarKvFull = 2, kBarKvEmpty = 3, kBarSFull = 
 // Optional timeline instrumentation (debug builds only, -DATTN_TRACE): CTA 0 records clock64()
 // at fixed points of each role for KV steps [kTraceStep0, kTraceStep0 + 16).
 #ifdef ATTN_TRACE
-constexpr int kTraceStep0 = 8;
+#ifndef ATTN_TRACE_STEP0
+#define ATTN_TRACE_STEP0 8
+#endif
+constexpr int kTraceStep0 = ATTN_TRACE_STEP0;
 __device__ long long g_attn_trace[5][16][8];
 #define ATTN_TRACE_EVENT(role_slot, step, ev)                                                   \
   do {                                                                                          \
@@ -235,8 +238,11 @@ template <int D, int TKV, int NQ>
 struct FwdSmem {
   static constexpr int kQBytes = NQ * kSub * D * 2;
   static constexpr int kStageBytes = TKV * D * 2;
+  static constexpr int kOutBytes = NQ * kSub * 128;    // per softmax warpgroup one [128 rows][64 columns] bf16 output chunk
   static constexpr int kMiscBytes = 3072;
-  __host__ __device__ static constexpr int total(int stages) { return kQBytes + stages * kStageBytes + kMiscBytes; }
+  __host__ __device__ static constexpr int total(int stages) {
+    return kQBytes + stages * kStageBytes + kOutBytes + kMiscBytes;
+  }
 };
 
 constexpr int kMaxStages = 8;
@@ -246,7 +252,7 @@ constexpr int kCounterBytes = 65536;   // head of the workspace: 16384 arrival c
 
 struct FwdMisc {               // lives in the last 3072 bytes of dynamic shared memory
   float alpha[2][2][kSub];     // [sub-tile][step parity][row] rescale factor
-  uint64_t q_full;
+  uint64_t q_full[2];          // one per Q sub-tile: the first product starts when sub-tile 0 and K_0 are in
   uint64_t kv_full[kMaxStages];
   uint64_t kv_empty[kMaxStages];
   uint64_t s_full[2];
@@ -382,7 +388,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const uint32_t smem_base = smem_u32(smem_raw);
   const uint32_t q_smem = smem_base;
   const uint32_t ring_smem = smem_base + SM::kQBytes;
-  FwdMisc* misc = reinterpret_cast<FwdMisc*>(smem_raw + SM::kQBytes + p.stages * SM::kStageBytes);
+  const uint32_t out_smem = ring_smem + p.stages * SM::kStageBytes;   // output staging of segments that are not the CTA's last
+  FwdMisc* misc = reinterpret_cast<FwdMisc*>(smem_raw + SM::kQBytes + p.stages * SM::kStageBytes + SM::kOutBytes);
   volatile int* abort_flag = &misc->abort_flag;
 
   const int warp = threadIdx.x >> 5;
@@ -403,7 +410,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       report_timeout(wait_info(kRoleLoad, 0, 0xFFFF));
       misc->abort_flag = 1;
     }
-    mbar_init(smem_u32(&misc->q_full), 1);
+    mbar_init(smem_u32(&misc->q_full[0]), 1);
+    mbar_init(smem_u32(&misc->q_full[1]), 1);
     for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(smem_u32(&misc->kv_full[s]), 1);
       mbar_init(smem_u32(&misc->kv_empty[s]), 1);
@@ -584,25 +592,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tc_fence_after();
       if (warp == 0) ATTN_TRACE_MARK(4);
       const bool last_seg = (u >= u_hi);                     // u was advanced past this segment already
-      const int grow = q_row0 + i * kSub + row;              // this thread's row in the sequence
-      // Normalised values of one output row chunk -> memory.  On the CTA's last segment the Q buffer is
-      // dead and the rows go through shared memory and a TMA store; otherwise the next segment's Q tile
-      // may already be arriving there and the rows are stored from registers.
-      auto put_chunk = [&](int c, const float (&val)[32]) {
+      // Normalised values of one 32-column chunk of this thread's output row -> memory, always through
+      // shared memory and a TMA store (coalesced, and rows past the end of the sequence are clipped by the
+      // tensor map).  On the CTA's last segment the Q buffer is dead and takes the whole sub-tile; before
+      // that the next segment's Q tile may already be arriving there, so the rows go through this
+      // warpgroup's [128][64] staging chunk, one 64-column half of the row at a time.
+      auto put_chunk = [&](int c, const float (&val)[32]) -> bool {
         if (last_seg) {
           stage_row_chunk(q_smem + i * (kSub * D * 2), c, row, val);
-        } else if (grow < p.L) {
-          uint4* orow = reinterpret_cast<uint4*>(p.o + ((size_t)bh * p.L + grow) * D) + c * 4;
-#pragma unroll
-          for (int u4 = 0; u4 < 4; ++u4) {
-            uint4 w4;
-            w4.x = pack_bf16x2(val[u4 * 8 + 0], val[u4 * 8 + 1]);
-            w4.y = pack_bf16x2(val[u4 * 8 + 2], val[u4 * 8 + 3]);
-            w4.z = pack_bf16x2(val[u4 * 8 + 4], val[u4 * 8 + 5]);
-            w4.w = pack_bf16x2(val[u4 * 8 + 6], val[u4 * 8 + 7]);
-            orow[u4] = w4;
-          }
+          return true;
         }
+        const uint32_t stage_out = out_smem + i * (kSub * 128);
+        stage_row_chunk(stage_out, c & 1, row, val);
+        if ((c & 1) == 0) return true;
+        fence_proxy_async_smem();
+        bool r = wg_sync(4);
+        if (r && (warp & 3) == 0 && lane == 0) {
+          tma_store_3d(&tm_o, stage_out, (c >> 1) * 64, q_row0 + i * kSub, bh);
+          tma_store_commit();
+          tma_store_wait_read();
+        }
+        if (r) r = wg_sync(5);                               // the staging chunk may be written again
+        return r;
       };
       auto finish_rows = [&]() -> bool {                     // after put_chunk on the last segment
         if (!last_seg) return true;
@@ -628,11 +639,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tmem_ld32(o_tmem + c * 32, r);
 #pragma unroll
           for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(r[k]) * inv;
-          put_chunk(c, val);
+          if (!put_chunk(c, val)) { ok = false; break; }
         }
         tc_fence_before();
         mbar_arrive(smem_u32(&misc->o_free[i]));             // O may be overwritten by the next segment
-        ok = finish_rows();
+        if (ok) ok = finish_rows();
       } else {
         // Part of a Q tile: un-normalised partial (O, m, delta) of this key range.  A CTA has at most two
         // such pieces, its first and its last segment: slots 2*cta and 2*cta + 1.
@@ -704,8 +715,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
           for (int k = 0; k < D; ++k) val[k] *= inv;
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) put_chunk(c, *reinterpret_cast<float(*)[32]>(&val[c * 32]));
-          ok = finish_rows();
+          for (int c = 0; c < D / 32; ++c)
+            if (ok) ok = put_chunk(c, *reinterpret_cast<float(*)[32]>(&val[c * 32]));
+          if (ok) ok = finish_rows();
         }
       }
       }
@@ -780,17 +792,27 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg)) {
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
-      ok = wait_bar_warp(smem_u32(&misc->q_full), seg & 1, abort_flag, wait_info(kRoleMma, kBarQ, seg));
+      ok = wait_bar_warp(smem_u32(&misc->q_full[0]), seg & 1, abort_flag, wait_info(kRoleMma, kBarQ, seg));
       if (ok) ok = wait_bar_warp(smem_u32(&misc->kv_full[stage]), phase, abort_flag, wait_info(kRoleMma, kBarKvFull, g));
       if (!ok) break;
       tc_fence_after();
       if (elect_one()) {
-#pragma unroll
-        for (int i = 0; i < NQ; ++i) {
-          issue_qk<D, TKV>(tmem_base + i * S_COLS, q_smem + i * (kSub * D * 2), ring_smem + stage * SM::kStageBytes);
-          umma_commit(smem_u32(&misc->s_full[i]));
+        issue_qk<D, TKV>(tmem_base, q_smem, ring_smem + stage * SM::kStageBytes);
+        umma_commit(smem_u32(&misc->s_full[0]));
+      }
+      __syncwarp();
+      if (NQ == 2) {
+        ok = wait_bar_warp(smem_u32(&misc->q_full[1]), seg & 1, abort_flag, wait_info(kRoleMma, kBarQ, 0x8000 | seg));
+        if (!ok) break;
+        tc_fence_after();
+      }
+      if (elect_one()) {
+        if (NQ == 2) {
+          issue_qk<D, TKV>(tmem_base + S_COLS, q_smem + kSub * D * 2, ring_smem + stage * SM::kStageBytes);
+          umma_commit(smem_u32(&misc->s_full[1]));
         }
         umma_commit(smem_u32(&misc->kv_empty[stage]));
+        if (n == 1) umma_commit(smem_u32(&misc->q_empty));   // a one-step segment reads Q only here
       }
       __syncwarp();
       advance();
@@ -838,9 +860,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (more) {
               issue_qk<D, TKV>(s_acc, q_smem + i * (kSub * D * 2), k_smem);
               umma_commit(smem_u32(&misc->s_full[i]));
-              if (i == NQ - 1) umma_commit(smem_u32(&misc->kv_empty[k_stage]));
-            } else if (i == NQ - 1) {
-              umma_commit(smem_u32(&misc->q_empty));       // every product that reads this Q tile is issued
+              if (i == NQ - 1) {
+                umma_commit(smem_u32(&misc->kv_empty[k_stage]));
+                // The last product that reads this segment's Q tile is issued one step before the segment
+                // ends: the next segment's Q tile can be fetched while that last step runs.
+                if (jj + 2 == n) umma_commit(smem_u32(&misc->q_empty));
+              }
             }
           }
           __syncwarp();
@@ -868,13 +893,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
         if (seg > 0 &&
             !wait_bar(smem_u32(&misc->q_empty), (seg - 1) & 1, abort_flag, wait_info(kRoleLoad, kBarQ, seg))) { ok = false; break; }
-        mbar_arrive_expect_tx(smem_u32(&misc->q_full), SM::kQBytes);
-#pragma unroll
-        for (int i = 0; i < NQ; ++i)
+        // Q sub-tile 0, then the first K tile, then Q sub-tile 1: the first product needs only the first two.
+        auto load_q = [&](int i) {
+          mbar_arrive_expect_tx(smem_u32(&misc->q_full[i]), kSub * D * 2);
 #pragma unroll
           for (int c = 0; c < KCH; ++c)
             tma_load_3d(q_smem + i * (kSub * D * 2) + c * (kSub * 128), &tm_q, c * 64, q_row0 + i * kSub, bh,
-                        smem_u32(&misc->q_full));
+                        smem_u32(&misc->q_full[i]));
+        };
+        load_q(0);
         ++q_loads;
         for (int t = 0; t < 2 * n; ++t) {
           if (!wait_bar(smem_u32(&misc->kv_empty[stage]), phase ^ 1u, abort_flag, wait_info(kRoleLoad, kBarKvEmpty, t))) { ok = false; break; }
@@ -887,6 +914,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           for (int c = 0; c < KCH; ++c) tma_load_3d(dst + c * (TKV * 128), tm, c * 64, kv_row, bh, bar);
           ++issued;
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+          if (t == 0 && NQ == 2) load_q(1);
         }
         if (!ok) break;
         }
@@ -901,8 +929,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           while (!mbar_try_wait(smem_u32(&misc->kv_full[sidx]), ph) && clock64() - t0 < kWaitLimitCycles) {}
         }
         if (q_loads > 0) {
-          const long long t0 = clock64();
-          while (!mbar_try_wait(smem_u32(&misc->q_full), (uint32_t)(q_loads - 1) & 1u) && clock64() - t0 < kWaitLimitCycles) {}
+          // (sub-tile 1 of the last Q load may not have been started; its barrier then completes no phase
+          // and the limit below ends the wait -- the CTA is already aborting)
+          for (int i = 0; i < NQ; ++i) {
+            const long long t0 = clock64();
+            while (!mbar_try_wait(smem_u32(&misc->q_full[i]), (uint32_t)(q_loads - 1) & 1u) && clock64() - t0 < kWaitLimitCycles) {}
+          }
         }
       }
     }

@@ -25,12 +25,15 @@ namespace {
 constexpr int kRegsCorrection = 64;   // per thread: O-rescale warpgroup
 constexpr int kRegsOther = 64;        // per thread: TMA and MMA-issue warpgroup
 constexpr int kRegsRowOverhead = 32;  // softmax thread: row statistics, addresses, loop state
-constexpr int kSmemReserve = 3072;    // barriers, rescale factors, tensor-memory slot
+constexpr int kSmemMisc = 3072;       // barriers, rescale factors, tensor-memory slot
+constexpr int kOutRowBytes = 128;     // output staging: per softmax warpgroup one chunk of 64 bf16 columns per row
 constexpr int kMaxStages = 8;
 constexpr int kMinStages = 4;         // K_j, V_j and one of each in flight
 constexpr int kMinTileKv = 32;
 constexpr int kMinStepsPerSplit = 4;
 constexpr int kSegmentOverheadSteps = 3;  // Q load + first product + partial write/merge, in units of one KV step
+constexpr int kCtaOverheadSteps = 2;      // start and end of a CTA that handles one whole Q tile
+constexpr int kTransitionSteps = 1;       // a persistent CTA moving on to its next Q tile
 
 inline int floor_to(int x, int m) { return (x / m) * m; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -66,7 +69,8 @@ long long attn_internal::head_units(int q_tiles, int steps, int ratio, int causa
 }
 
 // Occupancy step of the derivation (shared with the tile-override path of the launcher).
-int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int steps, int ratio, int causal) {
+int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int steps, int ratio, int causal,
+                             long long kv_bytes_per_head) {
   const long long tiles_ll = (long long)heads * q_tiles;
   const long long total = (long long)heads * head_units(q_tiles, steps, ratio, causal);
   if (causal) {
@@ -76,7 +80,20 @@ int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int 
     return (int)g;
   }
   const int tiles = (int)tiles_ll;
-  if (tiles >= h.num_units) return tiles;
+  if (tiles_ll >= h.num_units) {
+    // Enough tiles for every unit.  One CTA per tile runs ceil(tiles/units) waves, the last one partly
+    // empty, and every CTA pays its own start and end.  One persistent CTA per unit with an equal range
+    // of the unit line has neither cost but works on `units` different places at once: it is taken only
+    // when the K and V of the heads then in flight stay in two thirds of the cache.
+    const long long waves = (tiles_ll + h.num_units - 1) / h.num_units;
+    const long long cost_tiles = waves * (steps + kCtaOverheadSteps);
+    const long long g = h.num_units;
+    const long long cost_balanced = (total + g - 1) / g + 2 * kSegmentOverheadSteps + ((tiles_ll + g - 1) / g) * kTransitionSteps;
+    const long long heads_in_flight = heads < g ? heads : g;
+    const bool cached = h.cache_bytes > 0 && 3 * heads_in_flight * kv_bytes_per_head <= 2 * (long long)h.cache_bytes;
+    if (cached && cost_balanced < cost_tiles) return (int)g;
+    return (int)tiles_ll;
+  }
   int k = h.num_units / tiles;
   const int k_max = steps / kMinStepsPerSplit;
   if (k > k_max) k = k_max;
@@ -147,8 +164,10 @@ void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, int ca
   t->binding_constraint = binding;
   if (tile_kv < kMinTileKv) return;
 
-  // 2. Shared memory => depth of the K/V ring (Q tile resident, O staged in its place).
+  // 2. Shared memory => depth of the K/V ring.  Resident beside it: the Q tile, and per softmax warpgroup
+  //    one 64-column chunk of its output rows, through which finished Q tiles leave while the next one loads.
   const int q_bytes = n_q * sub * d * h.elem_bytes;
+  const int kSmemReserve = kSmemMisc + n_q * sub * kOutRowBytes;
   int stage = 0, stages = 0;
   for (;;) {
     stage = tile_kv * d * h.elem_bytes;
@@ -171,7 +190,8 @@ void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, int ca
   const int tiles = B * H * ceil_div(L, tile_q);
   const int steps = ceil_div(L, tile_kv);
   const int under = tiles < h.num_units;
-  const int ctas = attn_internal::grid_size(h, B * H, ceil_div(L, tile_q), steps, tile_q / tile_kv, causal);
+  const int ctas = attn_internal::grid_size(h, B * H, ceil_div(L, tile_q), steps, tile_q / tile_kv, causal,
+                                             2LL * L * d * h.elem_bytes);
   const int kv_splits = ceil_div(ctas, tiles);
 
   t->feasible = 1;
@@ -214,6 +234,7 @@ extern "C" int attn_hw_desc_b200(attn_hw_desc* out) {
   out->atom_k = 16;
   out->atom_n_max = 256;
   out->elem_bytes = 2;
+  out->cache_bytes = 126 << 20;   // L2
   out->hbm_gbps = 7700.0;
   out->peak_tflops = 2250.0;
   out->sm_clock_mhz = 1965.0;

@@ -15,7 +15,7 @@ CDNA = dict(lds_bytes=64 * 1024, regs_per_thread=256, wavefront=64, atom_m=16, a
 
 B200 = dict(num_units=148, local_mem_bytes=232448, regs_per_unit=65536, max_regs_per_thread=255,
             simd_width=32, acc_mem_lanes=128, acc_mem_columns=512, atom_m=128, atom_n=16, atom_k=16,
-            atom_n_max=256, elem_bytes=2)
+            atom_n_max=256, elem_bytes=2, cache_bytes=126 << 20)
 
 
 def test_table2_register_use_and_feasibility():
@@ -69,12 +69,13 @@ def test_tmem_machine_capacity_invariants(B, H, L, d):
     assert t["tile_q"] == 128 * n_q and t["tile_kv"] % 16 == 0 and 32 <= t["tile_kv"] <= 256
     assert n_q * (t["tile_kv"] + d) <= 512 <= 512 and t["tmem_columns"] <= 512       # tensor memory
     assert t["smem_bytes"] <= B200["local_mem_bytes"]                                  # shared memory
-    assert t["smem_bytes"] == n_q * 128 * d * 2 + t["kv_stages"] * t["tile_kv"] * d * 2 + 3072
+    assert t["smem_bytes"] == n_q * 128 * d * 2 + t["kv_stages"] * t["tile_kv"] * d * 2 + 3072 + n_q * 128 * 128
     assert 4 <= t["kv_stages"] <= 8
     regs_total = 128 * n_q * t["regs_softmax"] + 128 * 64 + 128 * 64                   # register file
     assert regs_total <= 65536 and t["regs_softmax"] <= 248
     assert t["tile_kv"] + t["tile_kv"] // 4 + 32 <= t["regs_softmax"]
-    assert t["tiles"] <= t["ctas"] <= t["tiles"] * t["kv_splits"]
+    # one CTA per tile, several per tile (key split), or one persistent CTA per unit
+    assert t["tiles"] <= t["ctas"] <= t["tiles"] * t["kv_splits"] or (t["ctas"] == 148 and t["tiles"] > 148)
     tc = po.derive_tiles_tmem_machine(B200, B, H, L, d, causal=True)
     assert tc["feasible"] and 1 <= tc["ctas"] <= 148 and tc["tile_kv"] == t["tile_kv"] and tc["tile_q"] == t["tile_q"]
     assert 0 < t["wave_efficiency"] <= 1.0
@@ -86,10 +87,21 @@ def test_tmem_machine_capacity_invariants(B, H, L, d):
 
 def test_tmem_machine_expected_defaults_for_the_benchmark_shapes():
     t = po.derive_tiles_tmem_machine(B200, 1, 1, 16384, 128)
-    assert (t["tile_q"], t["tile_kv"], t["kv_stages"], t["kv_splits"], t["ctas"]) == (256, 128, 5, 3, 148)
+    assert (t["tile_q"], t["tile_kv"], t["kv_stages"], t["kv_splits"], t["ctas"]) == (256, 128, 4, 3, 148)   # 65536 Q + 4 x 32768 ring + 32768 output staging + 3072 = 232448
     assert t["under_occupied"] and abs(t["wave_efficiency"] - 1.0) < 1e-12
     t = po.derive_tiles_tmem_machine(B200, 4, 32, 8192, 64)
     assert (t["tile_q"], t["tile_kv"], t["kv_stages"], t["kv_splits"]) == (256, 128, 8, 1)
     assert not t["under_occupied"]
+    # more tiles than SMs: a persistent grid of 148 CTAs when it saves partial waves and CTA starts and the
+    # K/V of the heads in flight fit two thirds of the L2 (4 heads x 8.4 MB), else one CTA per tile
+    t = po.derive_tiles_tmem_machine(B200, 1, 4, 16384, 128)
+    assert (t["tiles"], t["ctas"], t["kv_splits"]) == (256, 148, 1)
+    t = po.derive_tiles_tmem_machine(B200, 4, 32, 4096, 128)                             # 128 heads x 2.1 MB
+    assert (t["tiles"], t["ctas"]) == (2048, 2048)
+    t = po.derive_tiles_tmem_machine(B200, 1, 42, 4096, 128)                             # 42 x 2 MiB = 84 MiB = 2/3 of 126 MiB
+    assert (t["tiles"], t["ctas"]) == (672, 148)
+    t = po.derive_tiles_tmem_machine(B200, 1, 43, 4096, 128)                             # 86 MiB: over
+    assert (t["tiles"], t["ctas"]) == (688, 688)
+    assert po.derive_tiles_tmem_machine(dict(B200, cache_bytes=0), 1, 4, 16384, 128)["ctas"] == 256
     assert not po.derive_tiles_tmem_machine(B200, 1, 1, 1024, 72)["feasible"]          # d not a multiple of 16
     assert not po.derive_tiles_tmem_machine(B200, 1, 1, 1024, 512)["feasible"]         # d beyond the atom's N
