@@ -25,6 +25,7 @@ EXPORTED_SYMBOLS = (
     "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_static_scratch",
     "attn_last_device_status",
     "attn_last_launch_count", "attn_status_string", "attn_last_cuda_error",
+    "gemm_plan", "gemm_forward", "softmax_rows_forward", "attn_forward_unfused",
 )
 
 
@@ -41,6 +42,15 @@ class AttnTiles(ctypes.Structure):
         "threads", "tiles", "ctas",
     )] + [("ctas_per_unit", ctypes.c_float), ("wave_efficiency", ctypes.c_float)] + [
         (n, ctypes.c_int32) for n in ("feasible", "binding_constraint", "under_occupied", "causal")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class GemmTiles(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "tile_m", "tile_n", "tile_k", "n_sub", "stages", "smem_bytes", "tmem_columns", "tiles", "ctas", "feasible",
+    )] + [("wave_efficiency", ctypes.c_float), ("binding_constraint", ctypes.c_int32)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -87,6 +97,10 @@ def lib() -> ctypes.CDLL:
         L.attn_status_string.restype = ctypes.c_char_p
         L.attn_last_cuda_error.argtypes = []
         L.attn_last_cuda_error.restype = ctypes.c_char_p
+        L.gemm_plan.argtypes = [ctypes.POINTER(AttnHwDesc), i32, i32, i32, i32, ctypes.POINTER(GemmTiles)]
+        L.gemm_forward.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
+        L.softmax_rows_forward.argtypes = [vp, vp, ctypes.c_longlong, i32, ctypes.c_float, vp]
+        L.attn_forward_unfused.argtypes = [vp, vp, vp, vp, vp, ctypes.c_size_t, i32, i32, i32, i32, vp]
         for name in EXPORTED_SYMBOLS:
             getattr(L, name)
         _lib = L
@@ -282,3 +296,77 @@ def last_device_status(device=None):
 
 def last_launch_count() -> int:
     return int(lib().attn_last_launch_count())
+
+
+# ----------------------------------------------------------------- unfused path
+def gemm_plan(desc: AttnHwDesc, batch: int, M: int, N: int, K: int) -> GemmTiles:
+    t = GemmTiles()
+    _check(lib().gemm_plan(ctypes.byref(desc), batch, M, N, K, ctypes.byref(t)), "gemm_plan")
+    return t
+
+
+def _mat(x, name):
+    import torch
+
+    if x.dtype != torch.bfloat16 or not x.is_cuda or not x.is_contiguous() or x.dim() not in (2, 3):
+        raise ValueError(f"{name} must be a contiguous CUDA bfloat16 tensor of 2 or 3 dimensions")
+    return x if x.dim() == 3 else x.unsqueeze(0)
+
+
+def gemm(a, b, c=None, *, b_layout="kn"):
+    """C = A B ("kn": b is [.., K, N]) or C = A B^T ("nk": b is [.., N, K]); bf16 in and out, fp32 accumulation."""
+    import torch
+
+    a3, b3 = _mat(a, "a"), _mat(b, "b")
+    batch, M, K = (int(x) for x in a3.shape)
+    if b_layout == "kn":
+        kb, N = int(b3.shape[1]), int(b3.shape[2])
+    elif b_layout == "nk":
+        N, kb = int(b3.shape[1]), int(b3.shape[2])
+    else:
+        raise ValueError("b_layout is 'kn' or 'nk'")
+    if kb != K or int(b3.shape[0]) != batch:
+        raise ValueError("a and b do not agree in batch or K")
+    if c is None:
+        c = torch.empty((batch, M, N) if a.dim() == 3 else (M, N), dtype=torch.bfloat16, device=a.device)
+    elif c.dtype != torch.bfloat16 or not c.is_contiguous() or c.numel() != batch * M * N or c.device != a.device:
+        raise ValueError("c must be a contiguous bfloat16 tensor of batch*M*N elements on a's device")
+    dev = a.device.index if a.device.index is not None else torch.cuda.current_device()
+    with torch.cuda.device(dev):
+        stream = torch.cuda.current_stream(a.device).cuda_stream
+        _check(lib().gemm_forward(a.data_ptr(), b.data_ptr(), c.data_ptr(), batch, M, N, K,
+                                  0 if b_layout == "kn" else 1, stream), "gemm_forward")
+    return c
+
+
+def softmax_rows(s, scale: float, out=None):
+    """Row softmax of scale * s over the last dimension (bf16, CUDA, contiguous); out may be s."""
+    import torch
+
+    if s.dtype != torch.bfloat16 or not s.is_cuda or not s.is_contiguous():
+        raise ValueError("s must be a contiguous CUDA bfloat16 tensor")
+    if out is None:
+        out = torch.empty_like(s)
+    elif out.shape != s.shape or out.dtype != s.dtype or not out.is_contiguous() or out.device != s.device:
+        raise ValueError("out must match s")
+    cols = int(s.shape[-1])
+    rows = s.numel() // cols
+    dev = s.device.index if s.device.index is not None else torch.cuda.current_device()
+    with torch.cuda.device(dev):
+        stream = torch.cuda.current_stream(s.device).cuda_stream
+        _check(lib().softmax_rows_forward(s.data_ptr(), out.data_ptr(), rows, cols, float(scale), stream),
+               "softmax_rows_forward")
+    return out
+
+
+def forward_unfused(q, k, v, scores, o=None):
+    """The three-kernel path (S = Q K^T materialised in `scores`, softmax in place, P V); comparison only."""
+    import torch
+
+    o, B, H, L, d, dev, stream = _prep(q, k, v, o)
+    if scores.dtype != torch.bfloat16 or not scores.is_cuda or not scores.is_contiguous() or scores.device != q.device:
+        raise ValueError("scores must be a contiguous CUDA bfloat16 tensor on q's device")
+    with torch.cuda.device(dev):
+        _check(lib().attn_forward_unfused(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), scores.data_ptr(),
+                                          scores.numel() * 2, B, H, L, d, stream), "attn_forward_unfused")
+    return o

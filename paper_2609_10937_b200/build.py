@@ -11,7 +11,8 @@ ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libattn_b200.so"
 SOURCES = [CSRC / "attn_api.cu", CSRC / "attn_plan.cpp"]
-HEADERS = [CSRC / "attn_kernels.cuh", CSRC / "ptx_sm100.cuh", CSRC / "attn_plan_internal.h", ROOT / "include" / "attn.h"]
+HEADERS = [CSRC / "attn_kernels.cuh", CSRC / "gemm_kernels.cuh", CSRC / "ptx_sm100.cuh", CSRC / "attn_plan_internal.h",
+           ROOT / "include" / "attn.h", ROOT / "include" / "gemm.h"]
 
 
 def needs_build() -> bool:

@@ -13,6 +13,8 @@
 #include "attn.h"
 #include "attn_kernels.cuh"
 #include "attn_plan_internal.h"
+#include "gemm.h"
+#include "gemm_kernels.cuh"
 
 namespace {
 
@@ -442,4 +444,108 @@ extern "C" const char* attn_status_string(int status) {
     case ATTN_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the library's built-in array holds";
     default: return "unknown status";
   }
+}
+
+// ===========================================================================
+// Unfused path: matrix product, row softmax, three-kernel attention
+// ===========================================================================
+namespace {
+
+// 3-D map over a contiguous [batch][rows][cols] bf16 tensor with a (64 columns, box_rows rows, 1) box.
+int make_tmap_mat(CUtensorMap* m, const void* base, int batch, int rows, int cols, int box_rows) {
+  return make_tmap(m, base, batch, rows, cols, box_rows);
+}
+
+int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, int K, int b_layout, cudaStream_t stream) {
+  if (!a || !b || !c || batch <= 0 || M <= 0 || N <= 0 || K <= 0) return ATTN_ERR_INVALID_ARG;
+  if (b_layout != 0 && b_layout != 1) return ATTN_ERR_INVALID_ARG;
+  if ((K & 7) || (N & 7)) return ATTN_ERR_UNSUPPORTED_SHAPE;
+  if (((uintptr_t)a | (uintptr_t)b | (uintptr_t)c) & 15u) return ATTN_ERR_MISALIGNED;
+  const size_t a_bytes = (size_t)batch * M * K * 2, b_bytes = (size_t)batch * N * K * 2, c_bytes = (size_t)batch * M * N * 2;
+  if (overlaps(c, c_bytes, a, a_bytes) || overlaps(c, c_bytes, b, b_bytes)) return ATTN_ERR_ALIASING;
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);
+  if (rc != ATTN_OK) return rc;
+  gemm_tiles t;
+  if ((rc = gemm_plan(&st->desc, batch, M, N, K, &t)) != ATTN_OK) return rc;
+  // the kernel is compiled for exactly the tile shape the derivation gives on this architecture
+  if (!t.feasible || t.tile_m != gemm::kTileM || t.tile_n != gemm::kTileN || t.tile_k != gemm::kTileK ||
+      t.stages > gemm::kMaxStages)
+    return ATTN_ERR_INFEASIBLE_PLAN;
+  CUtensorMap ta, tb, tc;
+  if ((rc = make_tmap_mat(&ta, a, batch, M, K, attn::kSub)) != ATTN_OK) return rc;
+  if (b_layout == 0) rc = make_tmap_mat(&tb, b, batch, K, N, gemm::kTileK);    // [K][N]: box 64 columns x 64 k-rows
+  else rc = make_tmap_mat(&tb, b, batch, N, K, gemm::kTileN);                  // [N][K]: box 64 k-columns x 256 rows
+  if (rc != ATTN_OK) return rc;
+  if ((rc = make_tmap_mat(&tc, c, batch, M, N, attn::kSub)) != ATTN_OK) return rc;
+  gemm::GemmParams p;
+  p.M = M; p.N = N; p.K = K; p.batch = batch;
+  p.m_tiles = (M + gemm::kTileM - 1) / gemm::kTileM;
+  p.n_tiles = (N + gemm::kTileN - 1) / gemm::kTileN;
+  p.k_steps = (K + gemm::kTileK - 1) / gemm::kTileK;
+  p.stages = t.stages;
+  const int smem = gemm::smem_total(t.stages);
+  if (b_layout == 0) {
+    ATTN_CUDA_TRY(cudaFuncSetAttribute(gemm::gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    gemm::gemm_kernel<true><<<t.ctas, gemm::kThreads, smem, stream>>>(ta, tb, tc, p);
+  } else {
+    ATTN_CUDA_TRY(cudaFuncSetAttribute(gemm::gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    gemm::gemm_kernel<false><<<t.ctas, gemm::kThreads, smem, stream>>>(ta, tb, tc, p);
+  }
+  ATTN_CUDA_TRY(cudaGetLastError());
+  ++t_launch_count;
+  return ATTN_OK;
+}
+
+int softmax_launch(const void* s, void* pout, long long rows, int cols, float scale, cudaStream_t stream) {
+  if (!s || !pout || rows <= 0 || cols <= 0) return ATTN_ERR_INVALID_ARG;
+  if ((cols & 7) || cols > 32768 || rows > 0x7FFFFFFFLL) return ATTN_ERR_UNSUPPORTED_SHAPE;
+  if (((uintptr_t)s | (uintptr_t)pout) & 15u) return ATTN_ERR_MISALIGNED;
+  const float scale_log2 = scale * 1.4426950408889634f;
+  const int nvec = cols / 8;
+  const int vpt = (nvec + gemm::kSoftmaxThreads - 1) / gemm::kSoftmaxThreads;
+  const __nv_bfloat16* sp = static_cast<const __nv_bfloat16*>(s);
+  __nv_bfloat16* pp = static_cast<__nv_bfloat16*>(pout);
+  const dim3 grid((unsigned)rows);
+  if (vpt <= 1) gemm::softmax_rows_kernel<1><<<grid, gemm::kSoftmaxThreads, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (vpt <= 2) gemm::softmax_rows_kernel<2><<<grid, gemm::kSoftmaxThreads, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (vpt <= 4) gemm::softmax_rows_kernel<4><<<grid, gemm::kSoftmaxThreads, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (vpt <= 8) gemm::softmax_rows_kernel<8><<<grid, gemm::kSoftmaxThreads, 0, stream>>>(sp, pp, cols, scale_log2);
+  else gemm::softmax_rows_kernel<16><<<grid, gemm::kSoftmaxThreads, 0, stream>>>(sp, pp, cols, scale_log2);
+  ATTN_CUDA_TRY(cudaGetLastError());
+  ++t_launch_count;
+  return ATTN_OK;
+}
+
+}  // namespace
+
+extern "C" int gemm_forward(const void* a, const void* b, void* c, int batch, int M, int N, int K, int b_layout,
+                            void* cuda_stream) {
+  t_launch_count = 0;
+  return gemm_launch(a, b, c, batch, M, N, K, b_layout, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int softmax_rows_forward(const void* s, void* p, long long rows, int cols, float scale, void* cuda_stream) {
+  t_launch_count = 0;
+  return softmax_launch(s, p, rows, cols, scale, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int attn_forward_unfused(const void* q, const void* k, const void* v, void* o, void* scores, size_t scores_bytes,
+                                    int B, int H, int L, int d, void* cuda_stream) {
+  t_launch_count = 0;
+  if (!q || !k || !v || !o || !scores || B <= 0 || H <= 0 || L <= 0 || d <= 0) return ATTN_ERR_INVALID_ARG;
+  if ((L & 7) || (d & 7) || L > 32768) return ATTN_ERR_UNSUPPORTED_SHAPE;
+  const size_t need = (size_t)B * H * L * L * 2;
+  if (scores_bytes < need) return ATTN_ERR_INVALID_ARG;
+  const size_t bytes = (size_t)B * H * L * d * 2;
+  if (overlaps(o, bytes, q, bytes) || overlaps(o, bytes, k, bytes) || overlaps(o, bytes, v, bytes)) return ATTN_ERR_ALIASING;
+  if (overlaps(scores, need, q, bytes) || overlaps(scores, need, k, bytes) || overlaps(scores, need, v, bytes) ||
+      overlaps(scores, need, o, bytes))
+    return ATTN_ERR_ALIASING;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int rc;
+  if ((rc = gemm_launch(q, k, scores, B * H, L, L, d, 1, stream)) != ATTN_OK) return rc;           // S = Q K^T
+  if ((rc = softmax_launch(scores, scores, (long long)B * H * L, L, 1.0f / std::sqrt((float)d), stream)) != ATTN_OK)
+    return rc;                                                                                      // P = softmax(S / sqrt(d))
+  return gemm_launch(scores, v, o, B * H, L, d, L, 0, stream);                                      // O = P V
 }

@@ -18,6 +18,7 @@
 
 #include "attn.h"
 #include "attn_plan_internal.h"
+#include "gemm.h"
 
 namespace {
 
@@ -268,4 +269,43 @@ extern "C" size_t attn_workspace_bytes(const attn_tiles* t, int B, int H, int L,
   // sub-tile: 128 x d fp32 un-normalised output + 128 (m, delta) pairs.
   const size_t per_sub = (size_t)128 * (size_t)d * 4 + (size_t)128 * 2 * 4;
   return (size_t)65536 + (size_t)2 * (size_t)t->ctas * (size_t)t->n_q * per_sub;
+}
+
+// Matrix product: the same derivation for the GEMM kernel's tile structure (Eq. 2: the local memory
+// bounds the block tile through the ring depth; Eq. 3: the accumulator storage -- here tensor memory --
+// bounds the rows one CTA can accumulate).
+extern "C" int gemm_plan(const attn_hw_desc* desc, int batch, int M, int N, int K, gemm_tiles* out) {
+  if (!desc || !out) return ATTN_ERR_INVALID_ARG;
+  if (desc->struct_bytes != (int32_t)sizeof(attn_hw_desc)) return ATTN_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  if (batch <= 0 || M <= 0 || N <= 0 || K <= 0) return ATTN_ERR_INVALID_ARG;
+  const attn_hw_desc& h = *desc;
+  out->binding_constraint = ATTN_BIND_TMEM;
+  if (h.acc_mem_columns <= 0 || h.atom_n_max <= 0 || h.elem_bytes <= 0) return ATTN_OK;   // not a tensor-memory machine
+  const int tile_n = h.atom_n_max;
+  int n_sub = h.acc_mem_columns / tile_n;      // fp32 accumulator columns: one per output column and sub-tile
+  if (n_sub > 2) n_sub = 2;
+  if (n_sub < 1) return ATTN_OK;
+  const int tile_m = n_sub * h.atom_m;
+  const int tile_k = 128 / h.elem_bytes;       // one swizzle row
+  const int stage = (tile_m + tile_n) * tile_k * h.elem_bytes;
+  const int staging = n_sub * h.atom_m * 128;  // per sub-tile one 64-column chunk of the output rows
+  int stages = (h.local_mem_bytes - staging - 1024) / stage;
+  if (stages > 8) stages = 8;
+  if (stages < 2) { out->binding_constraint = ATTN_BIND_SMEM; return ATTN_OK; }
+  const long long tiles = (long long)batch * ceil_div(M, tile_m) * ceil_div(N, tile_n);
+  if (tiles > 0x3FFFFFFFLL) return ATTN_OK;
+  out->tile_m = tile_m;
+  out->tile_n = tile_n;
+  out->tile_k = tile_k;
+  out->n_sub = n_sub;
+  out->stages = stages;
+  out->smem_bytes = stages * stage + staging + 1024;
+  out->tmem_columns = pow2_ceil(n_sub * tile_n);
+  out->tiles = (int)tiles;
+  out->ctas = tiles < h.num_units ? (int)tiles : h.num_units;
+  const long long waves = (tiles + out->ctas - 1) / out->ctas;
+  out->wave_efficiency = (float)((double)tiles / ((double)waves * out->ctas));
+  out->feasible = 1;
+  return ATTN_OK;
 }

@@ -1,0 +1,298 @@
+// sm_100a kernels of the unfused path: a dense bf16 matrix product C = A B (the paper's Section
+// "GEMM") on tcgen05 tensor cores, and a row softmax (Section "Online Softmax": per-thread running
+// (m, d) statistics merged with the associative operator of that section).
+//
+//   gemm_kernel   persistent, warp-specialised: one TMA producer warp -> shared-memory ring of
+//                 (A tile, B tile) stages -> one MMA-issuing thread (tcgen05.mma, two 128-row
+//                 sub-tiles x 256 columns accumulated in tensor memory) -> eight epilogue warps
+//                 (tensor memory -> bf16 -> shared-memory staging -> TMA store).
+//   softmax_rows_kernel  one CTA per row, the row held in registers: one read, one write.
+//
+// Every device-side wait is bounded (see attn_kernels.cuh).
+#pragma once
+
+#include "attn_kernels.cuh"
+
+namespace gemm {
+
+using namespace sm100;
+using attn::kSub;
+
+constexpr int kTileM = 2 * kSub;   // two 128-row sub-tiles share every B tile
+constexpr int kTileN = 256;        // largest N of one matrix instruction
+constexpr int kTileK = 64;         // one 128-byte swizzle row of bf16
+constexpr int kStageA = kTileM * kTileK * 2;
+constexpr int kStageB = kTileN * kTileK * 2;
+constexpr int kStageBytes = kStageA + kStageB;
+constexpr int kOutBytes = 2 * kSub * 128;    // per sub-tile one [128 rows][64 columns] bf16 staging chunk
+constexpr int kMiscBytes = 1024;
+constexpr int kMaxStages = 8;
+constexpr int kThreads = 320;      // producer warp, MMA warp, eight epilogue warps
+__host__ __device__ constexpr int smem_total(int stages) { return stages * kStageBytes + kOutBytes + kMiscBytes; }
+
+enum Role : uint32_t { kRoleGemmLoad = 6, kRoleGemmMma = 7, kRoleGemmEpi = 8 };
+
+struct GemmParams {
+  int M, N, K;
+  int batch;
+  int m_tiles, n_tiles;   // ceil(M / 256), ceil(N / 256)
+  int k_steps;            // ceil(K / 64)
+  int stages;
+};
+
+struct GemmMisc {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t acc_full;      // all products of a tile have finished
+  uint64_t acc_empty;     // the epilogue has read the accumulators of a tile
+  uint64_t epi_sync[2];   // rendezvous of the four epilogue warps of a sub-tile
+  uint32_t tmem_slot;
+  int abort_flag;
+};
+static_assert(sizeof(GemmMisc) <= kMiscBytes, "misc region too large");
+
+// B_KN: B is stored [K][N] row-major (C = A B; the MN-major operand form, as V in P V);
+// otherwise B is stored [N][K] row-major (C = A B^T; K-major, as K in Q K^T).
+template <bool B_KN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+            const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = smem_u32(smem_raw);
+  const uint32_t out_smem = smem_base + p.stages * kStageBytes;
+  GemmMisc* misc = reinterpret_cast<GemmMisc*>(smem_raw + p.stages * kStageBytes + kOutBytes);
+  volatile int* abort_flag = &misc->abort_flag;
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    misc->abort_flag = 0;
+    if (smem_base & 1023u) {
+      attn::report_timeout(attn::wait_info(kRoleGemmLoad, 0, 0xFFFF));
+      misc->abort_flag = 1;
+    }
+    for (int s = 0; s < kMaxStages; ++s) {
+      mbar_init(smem_u32(&misc->full[s]), 1);
+      mbar_init(smem_u32(&misc->empty[s]), 1);
+    }
+    mbar_init(smem_u32(&misc->acc_full), 1);
+    mbar_init(smem_u32(&misc->acc_empty), 2 * kSub);
+    mbar_init(smem_u32(&misc->epi_sync[0]), kSub);
+    mbar_init(smem_u32(&misc->epi_sync[1]), kSub);
+    fence_mbar_init();
+    prefetch_tmap(&tm_a);
+    prefetch_tmap(&tm_b);
+    prefetch_tmap(&tm_c);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&misc->tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = misc->tmem_slot;
+  const long long tiles = (long long)p.batch * p.m_tiles * p.n_tiles;
+  const bool run = (*abort_flag == 0);
+
+  if (warp == 0) {
+    // ========================================================== TMA producer
+    if (run && elect_one()) {
+      int stage = 0, issued = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (long long t = blockIdx.x; ok && t < tiles; t += gridDim.x) {
+        const int nt = (int)(t % p.n_tiles), mt = (int)((t / p.n_tiles) % p.m_tiles), b = (int)(t / ((long long)p.n_tiles * p.m_tiles));
+        for (int ks = 0; ks < p.k_steps; ++ks) {
+          if (!attn::wait_bar(smem_u32(&misc->empty[stage]), phase ^ 1u, abort_flag, attn::wait_info(kRoleGemmLoad, 1, ks))) { ok = false; break; }
+          const uint32_t bar = smem_u32(&misc->full[stage]);
+          const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kStageA;
+          mbar_arrive_expect_tx(bar, kStageBytes);
+          tma_load_3d(a_dst, &tm_a, ks * kTileK, mt * kTileM, b, bar);
+          tma_load_3d(a_dst + kSub * 128, &tm_a, ks * kTileK, mt * kTileM + kSub, b, bar);
+          if (B_KN) {
+#pragma unroll
+            for (int c = 0; c < kTileN / 64; ++c)
+              tma_load_3d(b_dst + c * (kTileK * 128), &tm_b, nt * kTileN + c * 64, ks * kTileK, b, bar);
+          } else {
+            tma_load_3d(b_dst, &tm_b, ks * kTileK, nt * kTileN, b, bar);
+          }
+          ++issued;
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // Drain: every copy this thread started must land before the CTA may exit.
+        const int first = issued > p.stages ? issued - p.stages : 0;
+        for (int t = first; t < issued; ++t) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(smem_u32(&misc->full[t % p.stages]), (uint32_t)(t / p.stages) & 1u) &&
+                 clock64() - t0 < attn::kWaitLimitCycles) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ============================================================ MMA issuer
+    bool ok = run;
+    int stage = 0;
+    uint32_t phase = 0, tile_ctr = 0;
+    constexpr uint32_t idesc = make_idesc_bf16(kSub, kTileN, B_KN);
+    constexpr uint32_t hi_k = attn::desc_hi_sw128(1024);
+    for (long long t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++tile_ctr) {
+      if (tile_ctr > 0) {
+        ok = attn::wait_bar_warp(smem_u32(&misc->acc_empty), (tile_ctr - 1) & 1, abort_flag, attn::wait_info(kRoleGemmMma, 2, tile_ctr));
+        if (!ok) break;
+        tc_fence_after();
+      }
+      for (int ks = 0; ok && ks < p.k_steps; ++ks) {
+        if (!attn::wait_bar_warp(smem_u32(&misc->full[stage]), phase, abort_flag, attn::wait_info(kRoleGemmMma, 1, ks))) { ok = false; break; }
+        tc_fence_after();
+        if (elect_one()) {
+          const uint32_t a_smem = smem_base + stage * kStageBytes, b_smem = a_smem + kStageA;
+          const uint32_t b_lo = B_KN ? attn::desc_lo(b_smem, kTileK * 128) : attn::desc_lo(b_smem, 16);
+#pragma unroll
+          for (int sub = 0; sub < 2; ++sub) {
+            const uint32_t a_lo = attn::desc_lo(a_smem + sub * (kSub * 128), 16);
+#pragma unroll
+            for (int k16 = 0; k16 < kTileK / 16; ++k16) {
+              const uint64_t a = attn::desc_from_words(a_lo + ((k16 * 32) >> 4), hi_k);
+              // K-major B: 16 columns further along the swizzle row; MN-major B: 16 key rows = 2048 bytes further
+              const uint64_t b = attn::desc_from_words(b_lo + ((B_KN ? k16 * 2048 : k16 * 32) >> 4), hi_k);
+              umma_ss(tmem_base + sub * kTileN, a, b, idesc, (ks > 0 || k16 > 0) ? 1u : 0u);
+            }
+          }
+          umma_commit(smem_u32(&misc->empty[stage]));
+          if (ks == p.k_steps - 1) umma_commit(smem_u32(&misc->acc_full));
+        }
+        __syncwarp();
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else {
+    // ============================================================== epilogue
+    const int sub = (warp - 2) >> 2;
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t acc = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + sub * kTileN;
+    const uint32_t bar_e = smem_u32(&misc->epi_sync[sub]);
+    const uint32_t stage_out = out_smem + sub * (kSub * 128);
+    const bool leader = ((warp - 2) & 3) == 0 && lane == 0;
+    uint32_t ep_phase = 0, tile_ctr = 0;
+    bool ok = run;
+    auto group_sync = [&](uint32_t tag) -> bool {
+      mbar_arrive(bar_e);
+      const bool r = attn::wait_bar_warp(bar_e, ep_phase, abort_flag, attn::wait_info(kRoleGemmEpi, 3, tag));
+      ep_phase ^= 1u;
+      return r;
+    };
+    for (long long t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++tile_ctr) {
+      const int nt = (int)(t % p.n_tiles), mt = (int)((t / p.n_tiles) % p.m_tiles), b = (int)(t / ((long long)p.n_tiles * p.m_tiles));
+      ok = attn::wait_bar_warp(smem_u32(&misc->acc_full), tile_ctr & 1, abort_flag, attn::wait_info(kRoleGemmEpi, 2, tile_ctr));
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll 1
+      for (int c = 0; c < kTileN / 32; ++c) {
+        uint32_t r[32];
+        float val[32];
+        tmem_ld32(acc + c * 32, r);
+#pragma unroll
+        for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(r[k]);
+        if (c == kTileN / 32 - 1) {
+          tc_fence_before();
+          mbar_arrive(smem_u32(&misc->acc_empty));       // the next tile may overwrite the accumulators
+        }
+        attn::stage_row_chunk(stage_out, c & 1, row, val);
+        if ((c & 1) == 0) continue;
+        fence_proxy_async_smem();
+        if (!(ok = group_sync(c))) break;
+        if (leader) {
+          tma_store_3d(&tm_c, stage_out, nt * kTileN + (c >> 1) * 64, mt * kTileM + sub * kSub, b);
+          tma_store_commit();
+          tma_store_wait_read();
+        }
+        if (!(ok = group_sync(0x100 | c))) break;          // the staging chunk may be written again
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Row softmax of scale * S, bf16 in and out (in place allowed).  One CTA per row; thread t holds VPT
+// vectors of 8 consecutive columns (vector v covers columns (v * 256 + t) * 8 ...).  Each thread keeps
+// the running statistics (m, d) of its columns; partials are merged with
+//   (m1, d1) (+) (m2, d2) = (max(m1, m2), d1 2^(m1 - m) + d2 2^(m2 - m))
+// first across the warp by shuffles, then across warps through shared memory.
+// ---------------------------------------------------------------------------
+constexpr int kSoftmaxThreads = 256;
+
+__device__ __forceinline__ void merge_md(float& m, float& d, float m2, float d2) {
+  const float mn = fmaxf(m, m2);
+  // a side with no element yet has m = -inf and d = 0: its term is 0, not NaN
+  const float t1 = (m == -INFINITY) ? 0.f : d * exp2f(m - mn);
+  const float t2 = (m2 == -INFINITY) ? 0.f : d2 * exp2f(m2 - mn);
+  m = mn;
+  d = t1 + t2;
+}
+
+template <int VPT>
+__global__ void __launch_bounds__(kSoftmaxThreads)
+softmax_rows_kernel(const __nv_bfloat16* s, __nv_bfloat16* pout, int cols, float scale_log2) {
+  __shared__ float sm_m[kSoftmaxThreads / 32], sm_d[kSoftmaxThreads / 32];
+  const size_t row = blockIdx.x;
+  const uint4* src = reinterpret_cast<const uint4*>(s + row * (size_t)cols);
+  uint4* dst = reinterpret_cast<uint4*>(pout + row * (size_t)cols);
+  const int nvec = cols / 8;
+  float x[VPT][8];
+  float m = -INFINITY;
+#pragma unroll
+  for (int v = 0; v < VPT; ++v) {
+    const int idx = v * kSoftmaxThreads + threadIdx.x;
+    if (idx < nvec) {
+      const uint4 w = src[idx];
+      const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        x[v][2 * e] = __uint_as_float(u[e] << 16) * scale_log2;
+        x[v][2 * e + 1] = __uint_as_float(u[e] & 0xFFFF0000u) * scale_log2;
+        m = fmaxf(m, fmaxf(x[v][2 * e], x[v][2 * e + 1]));
+      }
+    }
+  }
+  float d = 0.f;
+#pragma unroll
+  for (int v = 0; v < VPT; ++v)
+    if (v * kSoftmaxThreads + threadIdx.x < nvec) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) d += exp2f(x[v][e] - m);
+    }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, off), d2 = __shfl_xor_sync(0xffffffffu, d, off);
+    merge_md(m, d, m2, d2);
+  }
+  if ((threadIdx.x & 31) == 0) { sm_m[threadIdx.x >> 5] = m; sm_d[threadIdx.x >> 5] = d; }
+  __syncthreads();
+  float mr = sm_m[0], dr = sm_d[0];
+#pragma unroll
+  for (int w = 1; w < kSoftmaxThreads / 32; ++w) merge_md(mr, dr, sm_m[w], sm_d[w]);
+  const float inv = 1.0f / dr;
+#pragma unroll
+  for (int v = 0; v < VPT; ++v) {
+    const int idx = v * kSoftmaxThreads + threadIdx.x;
+    if (idx < nvec) {
+      uint4 w;
+      w.x = pack_bf16x2(exp2f(x[v][0] - mr) * inv, exp2f(x[v][1] - mr) * inv);
+      w.y = pack_bf16x2(exp2f(x[v][2] - mr) * inv, exp2f(x[v][3] - mr) * inv);
+      w.z = pack_bf16x2(exp2f(x[v][4] - mr) * inv, exp2f(x[v][5] - mr) * inv);
+      w.w = pack_bf16x2(exp2f(x[v][6] - mr) * inv, exp2f(x[v][7] - mr) * inv);
+      dst[idx] = w;
+    }
+  }
+}
+
+}  // namespace gemm

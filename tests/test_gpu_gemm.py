@@ -1,0 +1,122 @@
+"""GPU parity of the unfused path (matrix product, row softmax, three-kernel attention) against the fp64 oracle."""
+import math
+
+import numpy as np
+import pytest
+
+from paper_2609_10937_b200 import synth
+from tests.gpu_util import to_cuda_bf16, to_host_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+
+    from oracle import gemm_oracle as go
+    from paper_2609_10937_b200 import binding, build
+
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    build.build()
+    binding.lib()
+    return torch, go, binding
+
+
+def _rand_bits(rng, shape, sigma=1.0):
+    return synth.f32_to_bf16_bits((rng.standard_normal(shape) * sigma).astype(np.float32))
+
+
+def _check_product(env, batch, M, N, K, layout, seed, rows_per_batch=None):
+    torch, go, binding = env
+    rng = np.random.default_rng([seed, M, N, K])
+    a = _rand_bits(rng, (batch, M, K))
+    b = _rand_bits(rng, (batch, K, N) if layout == "kn" else (batch, N, K))
+    c = binding.gemm(to_cuda_bf16(a), to_cuda_bf16(b), b_layout=layout)
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0
+    got = to_host_f64(c).reshape(batch, M, N)
+    for bi in range(batch):
+        rows = np.arange(M) if rows_per_batch is None or rows_per_batch >= M else \
+            np.unique(np.concatenate([[0, M - 1], rng.integers(0, M, rows_per_batch)]))
+        ref = go.matmul_rows(a[bi], b[bi], M, N, K, rows, layout)
+        # fp32 accumulation of K products of size ~1, then one bf16 rounding of a value of size ~sqrt(K)
+        tol = 2.0 ** -8 * np.maximum(np.abs(ref), 1.0) + 1e-5 * math.sqrt(K)
+        err = np.abs(got[bi][rows] - ref)
+        assert (err <= tol).all(), (layout, batch, M, N, K, float(err.max()), float(np.abs(ref).max()))
+
+
+@pytest.mark.parametrize("layout", ["kn", "nk"])
+@pytest.mark.parametrize("batch,M,N,K", [
+    (1, 256, 256, 64), (1, 256, 256, 256), (1, 512, 768, 192), (2, 384, 520, 136), (1, 1, 8, 8), (3, 130, 264, 72),
+    (1, 1000, 1000, 1000), (1, 2048, 128, 2048)])
+def test_matrix_product_matches_oracle(env, layout, batch, M, N, K):
+    _check_product(env, batch, M, N, K, layout, seed=1)
+
+
+@pytest.mark.parametrize("layout", ["kn", "nk"])
+def test_structured_products(env, layout):
+    """Identity, a single one, and an index pattern: operand order and the two storage layouts of B."""
+    torch, go, binding = env
+    M = N = K = 320
+    rng = np.random.default_rng(4)
+    a = _rand_bits(rng, (M, K))
+    eye = synth.f32_to_bf16_bits(np.eye(K, dtype=np.float32))
+    c = to_host_f64(binding.gemm(to_cuda_bf16(a), to_cuda_bf16(eye), b_layout=layout)).reshape(M, N)
+    assert np.array_equal(c, go.bf16_bits_to_f64(a).reshape(M, K))
+    # B[k][j] (as a matrix, whatever its storage) = 1 if k == 2 j' pattern: picks columns of A
+    bm = np.zeros((K, N), np.float32)
+    bm[(np.arange(N) * 7) % K, np.arange(N)] = 1.0
+    b_store = bm if layout == "kn" else np.ascontiguousarray(bm.T)
+    c = to_host_f64(binding.gemm(to_cuda_bf16(a), to_cuda_bf16(synth.f32_to_bf16_bits(b_store)), b_layout=layout)).reshape(M, N)
+    assert np.array_equal(c, go.bf16_bits_to_f64(a).reshape(M, K)[:, (np.arange(N) * 7) % K])
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0
+
+
+def test_matrix_product_full_size_sampled(env):
+    """The paper's 4096^3 shape, rows sampled."""
+    _check_product(env, 1, 4096, 4096, 4096, "kn", seed=2, rows_per_batch=48)
+
+
+@pytest.mark.parametrize("rows,cols", [(4, 8), (7, 256), (33, 2048), (5, 2056), (3, 16384), (2, 32768), (9, 1000)])
+def test_row_softmax_matches_oracle(env, rows, cols):
+    torch, go, binding = env
+    rng = np.random.default_rng([rows, cols])
+    s = _rand_bits(rng, (rows, cols), sigma=6.0)
+    scale = 0.37
+    ref = go.softmax_rows(go.bf16_bits_to_f64(s).reshape(rows, cols), scale)
+    st = to_cuda_bf16(s)
+    p = binding.softmax_rows(st, scale)
+    got = to_host_f64(p).reshape(rows, cols)
+    assert np.abs(got - ref).max() <= 2.0 ** -8 * ref.max() + 1e-6
+    assert np.abs(got.sum(axis=1) - 1.0).max() <= 1e-2
+    p2 = binding.softmax_rows(st, scale, out=st)                 # in place
+    assert torch.equal(p2, p)
+
+
+@pytest.mark.parametrize("B,H,L,d", [(1, 1, 256, 64), (1, 2, 1024, 128), (2, 2, 520, 64), (1, 1, 4096, 128)])
+def test_unfused_attention_matches_its_oracle_and_the_fused_kernel(env, B, H, L, d):
+    torch, go, binding = env
+    from oracle import attn_oracle as orc
+
+    case = synth.AttnCase("unfused", B, H, L, d)
+    q, k, v = synth.make_qkv(case, seed=5)
+    tq, tk, tv = (to_cuda_bf16(x) for x in (q, k, v))
+    scores = torch.empty(B * H * L * L, dtype=torch.bfloat16, device="cuda")
+    o = binding.forward_unfused(tq, tk, tv, scores)
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0
+    got = to_host_f64(o).reshape(B * H, L, d)
+    rows = np.unique(np.concatenate([[0, L - 1], np.random.default_rng(L).integers(0, L, 40)]))
+    qh, kh, vh = (x.reshape(B * H, L, d) for x in (q, k, v))
+    for bh in range(B * H):
+        u = go.unfused_attention_rows(qh[bh], kh[bh], vh[bh], L, d, rows)
+        err = np.abs(got[bh][rows] - u["o"])
+        # same three steps and the same two bf16 roundings; what remains is fp32 accumulation, exp2 and the
+        # final bf16 rounding of the output
+        assert err.max() <= 1e-2 and np.linalg.norm(err) / np.linalg.norm(u["o"]) <= 5e-3
+    # and the definition itself (the fused kernel's oracle), at the looser bound the two extra roundings cost
+    ref = orc.attention_rows(q, k, v, B, H, L, d, rows.astype(np.int32)).reshape(B * H, len(rows), d)
+    assert np.abs(got[:, rows] - ref).max() <= 3e-2

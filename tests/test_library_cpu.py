@@ -23,18 +23,41 @@ def binding():
 
 
 def _declared_functions():
-    text = open(os.path.join(ROOT, "include", "attn.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(attn_[a-z0-9_]+)\s*\(", text)))
+    names = set()
+    for header in ("attn.h", "gemm.h"):
+        text = open(os.path.join(ROOT, "include", header)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b((?:attn|gemm|softmax)_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_every_declared_symbol_is_exported(binding):
     names = _declared_functions()
-    assert len(names) >= 12
+    assert len(names) >= 16
     L = binding.lib()
     for n in names:
-        assert hasattr(L, n), f"{n} declared in include/attn.h but not exported"
+        assert hasattr(L, n), f"{n} declared in include/*.h but not exported"
     assert set(names) == set(binding.EXPORTED_SYMBOLS)
+
+
+def test_gemm_plan_closed_form(binding):
+    """Tile derivation of the matrix product (Eq. 2, Eq. 3 re-read for tensor memory), retyped from the header's formula
+    with the B200 constants, and its reaction to a changed descriptor."""
+    desc = binding.hw_desc_b200()
+    t = binding.gemm_plan(desc, 1, 4096, 4096, 4096)
+    # 512 accumulator columns / 256 = 2 sub-tiles; stage = (256 + 256) * 64 * 2 = 65536; staging 2 * 128 * 128
+    assert (t.tile_m, t.tile_n, t.tile_k, t.n_sub) == (256, 256, 64, 2)
+    assert t.stages == (232448 - 32768 - 1024) // 65536 == 3 and t.smem_bytes == 3 * 65536 + 32768 + 1024
+    assert (t.tiles, t.ctas, t.feasible, t.tmem_columns) == (256, 148, 1, 512)
+    assert t.wave_efficiency == pytest.approx(256 / (2 * 148))
+    t = binding.gemm_plan(desc, 3, 1000, 520, 64)
+    assert (t.tiles, t.ctas) == (3 * 4 * 3, 36)
+    desc.acc_mem_columns = 256                      # half the tensor memory: one sub-tile
+    t = binding.gemm_plan(desc, 1, 4096, 4096, 4096)
+    assert (t.n_sub, t.tile_m, t.stages) == (1, 128, (232448 - 16384 - 1024) // 49152)
+    desc.local_mem_bytes = 101376                   # a small shared memory: the ring no longer fits twice
+    t = binding.gemm_plan(desc, 1, 4096, 4096, 4096)
+    assert t.feasible == 0 or t.stages >= 2
 
 
 def test_struct_sizes_match_the_header(binding):
