@@ -469,29 +469,30 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
   gemm_tiles t;
   if ((rc = gemm_plan(&st->desc, batch, M, N, K, &t)) != ATTN_OK) return rc;
   // the kernel is compiled for exactly the tile shape the derivation gives on this architecture
-  if (!t.feasible || t.tile_m != gemm::kTileM || t.tile_n != gemm::kTileN || t.tile_k != gemm::kTileK ||
+  if (!t.feasible || t.tile_m != gemm::kTileM || (t.tile_n != 128 && t.tile_n != 256) || t.tile_k != gemm::kTileK ||
       t.stages > gemm::kMaxStages)
     return ATTN_ERR_INFEASIBLE_PLAN;
   CUtensorMap ta, tb, tc;
   if ((rc = make_tmap_mat(&ta, a, batch, M, K, attn::kSub)) != ATTN_OK) return rc;
   if (b_layout == 0) rc = make_tmap_mat(&tb, b, batch, K, N, gemm::kTileK);    // [K][N]: box 64 columns x 64 k-rows
-  else rc = make_tmap_mat(&tb, b, batch, N, K, gemm::kTileN);                  // [N][K]: box 64 k-columns x 256 rows
+  else rc = make_tmap_mat(&tb, b, batch, N, K, t.tile_n);                      // [N][K]: box 64 k-columns x tile_n rows
   if (rc != ATTN_OK) return rc;
   if ((rc = make_tmap_mat(&tc, c, batch, M, N, attn::kSub)) != ATTN_OK) return rc;
   gemm::GemmParams p;
   p.M = M; p.N = N; p.K = K; p.batch = batch;
   p.m_tiles = (M + gemm::kTileM - 1) / gemm::kTileM;
-  p.n_tiles = (N + gemm::kTileN - 1) / gemm::kTileN;
+  p.n_tiles = (N + t.tile_n - 1) / t.tile_n;
   p.k_steps = (K + gemm::kTileK - 1) / gemm::kTileK;
   p.stages = t.stages;
-  const int smem = gemm::smem_total(t.stages);
-  if (b_layout == 0) {
-    ATTN_CUDA_TRY(cudaFuncSetAttribute(gemm::gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    gemm::gemm_kernel<true><<<t.ctas, gemm::kThreads, smem, stream>>>(ta, tb, tc, p);
-  } else {
-    ATTN_CUDA_TRY(cudaFuncSetAttribute(gemm::gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    gemm::gemm_kernel<false><<<t.ctas, gemm::kThreads, smem, stream>>>(ta, tb, tc, p);
-  }
+  const int smem = gemm::smem_total(t.stages, t.tile_n);
+  auto launch = [&](auto kernel) -> int {
+    ATTN_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    kernel<<<t.ctas, gemm::kThreads, smem, stream>>>(ta, tb, tc, p);
+    return ATTN_OK;
+  };
+  if (t.tile_n == 256) rc = (b_layout == 0) ? launch(gemm::gemm_kernel<true, 256>) : launch(gemm::gemm_kernel<false, 256>);
+  else rc = (b_layout == 0) ? launch(gemm::gemm_kernel<true, 128>) : launch(gemm::gemm_kernel<false, 128>);
+  if (rc != ATTN_OK) return rc;
   ATTN_CUDA_TRY(cudaGetLastError());
   ++t_launch_count;
   return ATTN_OK;
@@ -502,16 +503,17 @@ int softmax_launch(const void* s, void* pout, long long rows, int cols, float sc
   if ((cols & 7) || cols > 32768 || rows > 0x7FFFFFFFLL) return ATTN_ERR_UNSUPPORTED_SHAPE;
   if (((uintptr_t)s | (uintptr_t)pout) & 15u) return ATTN_ERR_MISALIGNED;
   const float scale_log2 = scale * 1.4426950408889634f;
-  const int nvec = cols / 8;
-  const int vpt = (nvec + gemm::kSoftmaxThreads - 1) / gemm::kSoftmaxThreads;
+  const int nvec = cols / 8;                        // 16-byte vectors per row
   const __nv_bfloat16* sp = static_cast<const __nv_bfloat16*>(s);
   __nv_bfloat16* pp = static_cast<__nv_bfloat16*>(pout);
   const dim3 grid((unsigned)rows);
-  if (vpt <= 1) gemm::softmax_rows_kernel<1><<<grid, gemm::kSoftmaxThreads, 0, stream>>>(sp, pp, cols, scale_log2);
-  else if (vpt <= 2) gemm::softmax_rows_kernel<2><<<grid, gemm::kSoftmaxThreads, 0, stream>>>(sp, pp, cols, scale_log2);
-  else if (vpt <= 4) gemm::softmax_rows_kernel<4><<<grid, gemm::kSoftmaxThreads, 0, stream>>>(sp, pp, cols, scale_log2);
-  else if (vpt <= 8) gemm::softmax_rows_kernel<8><<<grid, gemm::kSoftmaxThreads, 0, stream>>>(sp, pp, cols, scale_log2);
-  else gemm::softmax_rows_kernel<16><<<grid, gemm::kSoftmaxThreads, 0, stream>>>(sp, pp, cols, scale_log2);
+  // threads x vectors per thread >= nvec, with at most four vectors per thread (register-light: several rows per SM)
+  if (nvec <= 128) gemm::softmax_rows_kernel<1, 128><<<grid, 128, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (nvec <= 256) gemm::softmax_rows_kernel<1, 256><<<grid, 256, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (nvec <= 512) gemm::softmax_rows_kernel<2, 256><<<grid, 256, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (nvec <= 1024) gemm::softmax_rows_kernel<2, 512><<<grid, 512, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (nvec <= 2048) gemm::softmax_rows_kernel<4, 512><<<grid, 512, 0, stream>>>(sp, pp, cols, scale_log2);
+  else gemm::softmax_rows_kernel<4, 1024><<<grid, 1024, 0, stream>>>(sp, pp, cols, scale_log2);
   ATTN_CUDA_TRY(cudaGetLastError());
   ++t_launch_count;
   return ATTN_OK;

@@ -282,8 +282,9 @@ extern "C" int gemm_plan(const attn_hw_desc* desc, int batch, int M, int N, int 
   const attn_hw_desc& h = *desc;
   out->binding_constraint = ATTN_BIND_TMEM;
   if (h.acc_mem_columns <= 0 || h.atom_n_max <= 0 || h.elem_bytes <= 0) return ATTN_OK;   // not a tensor-memory machine
-  const int tile_n = h.atom_n_max;
-  int n_sub = h.acc_mem_columns / tile_n;      // fp32 accumulator columns: one per output column and sub-tile
+  // N of one instruction: the largest the atom allows, or half of it when the output is no wider than that
+  const int tile_n = (N <= h.atom_n_max / 2) ? h.atom_n_max / 2 : h.atom_n_max;
+  int n_sub = h.acc_mem_columns / h.atom_n_max;   // fp32 accumulator columns: one per output column and sub-tile
   if (n_sub > 2) n_sub = 2;
   if (n_sub < 1) return ATTN_OK;
   const int tile_m = n_sub * h.atom_m;

@@ -19,23 +19,22 @@ using namespace sm100;
 using attn::kSub;
 
 constexpr int kTileM = 2 * kSub;   // two 128-row sub-tiles share every B tile
-constexpr int kTileN = 256;        // largest N of one matrix instruction
+constexpr int kTileNMax = 256;     // largest N of one matrix instruction; narrow outputs (N <= 128) use 128
 constexpr int kTileK = 64;         // one 128-byte swizzle row of bf16
 constexpr int kStageA = kTileM * kTileK * 2;
-constexpr int kStageB = kTileN * kTileK * 2;
-constexpr int kStageBytes = kStageA + kStageB;
+__host__ __device__ constexpr int stage_bytes(int tile_n) { return kStageA + tile_n * kTileK * 2; }
 constexpr int kOutBytes = 2 * kSub * 128;    // per sub-tile one [128 rows][64 columns] bf16 staging chunk
 constexpr int kMiscBytes = 1024;
 constexpr int kMaxStages = 8;
 constexpr int kThreads = 320;      // producer warp, MMA warp, eight epilogue warps
-__host__ __device__ constexpr int smem_total(int stages) { return stages * kStageBytes + kOutBytes + kMiscBytes; }
+__host__ __device__ constexpr int smem_total(int stages, int tile_n) { return stages * stage_bytes(tile_n) + kOutBytes + kMiscBytes; }
 
 enum Role : uint32_t { kRoleGemmLoad = 6, kRoleGemmMma = 7, kRoleGemmEpi = 8 };
 
 struct GemmParams {
   int M, N, K;
   int batch;
-  int m_tiles, n_tiles;   // ceil(M / 256), ceil(N / 256)
+  int m_tiles, n_tiles;   // ceil(M / 256), ceil(N / tile_n)
   int k_steps;            // ceil(K / 64)
   int stages;
 };
@@ -53,10 +52,12 @@ static_assert(sizeof(GemmMisc) <= kMiscBytes, "misc region too large");
 
 // B_KN: B is stored [K][N] row-major (C = A B; the MN-major operand form, as V in P V);
 // otherwise B is stored [N][K] row-major (C = A B^T; K-major, as K in Q K^T).
-template <bool B_KN>
+template <bool B_KN, int kTileN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
             const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
+  static_assert(kTileN == 128 || kTileN == 256, "tile N");
+  constexpr int kStageBytes = stage_bytes(kTileN);
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t smem_base = smem_u32(smem_raw);
   const uint32_t out_smem = smem_base + p.stages * kStageBytes;
@@ -222,13 +223,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
 }
 
 // ---------------------------------------------------------------------------
-// Row softmax of scale * S, bf16 in and out (in place allowed).  One CTA per row; thread t holds VPT
-// vectors of 8 consecutive columns (vector v covers columns (v * 256 + t) * 8 ...).  Each thread keeps
+// Row softmax of scale * S, bf16 in and out (in place allowed).  One CTA of THREADS threads per row; thread t
+// holds VPT vectors of 8 consecutive columns (vector v covers columns (v * THREADS + t) * 8 ...).  Each thread keeps
 // the running statistics (m, d) of its columns; partials are merged with
 //   (m1, d1) (+) (m2, d2) = (max(m1, m2), d1 2^(m1 - m) + d2 2^(m2 - m))
 // first across the warp by shuffles, then across warps through shared memory.
 // ---------------------------------------------------------------------------
-constexpr int kSoftmaxThreads = 256;
 
 __device__ __forceinline__ void merge_md(float& m, float& d, float m2, float d2) {
   const float mn = fmaxf(m, m2);
@@ -239,10 +239,10 @@ __device__ __forceinline__ void merge_md(float& m, float& d, float m2, float d2)
   d = t1 + t2;
 }
 
-template <int VPT>
-__global__ void __launch_bounds__(kSoftmaxThreads)
+template <int VPT, int THREADS>
+__global__ void __launch_bounds__(THREADS, 2048 / THREADS)
 softmax_rows_kernel(const __nv_bfloat16* s, __nv_bfloat16* pout, int cols, float scale_log2) {
-  __shared__ float sm_m[kSoftmaxThreads / 32], sm_d[kSoftmaxThreads / 32];
+  __shared__ float sm_m[THREADS / 32], sm_d[THREADS / 32];
   const size_t row = blockIdx.x;
   const uint4* src = reinterpret_cast<const uint4*>(s + row * (size_t)cols);
   uint4* dst = reinterpret_cast<uint4*>(pout + row * (size_t)cols);
@@ -251,7 +251,7 @@ softmax_rows_kernel(const __nv_bfloat16* s, __nv_bfloat16* pout, int cols, float
   float m = -INFINITY;
 #pragma unroll
   for (int v = 0; v < VPT; ++v) {
-    const int idx = v * kSoftmaxThreads + threadIdx.x;
+    const int idx = v * THREADS + threadIdx.x;
     if (idx < nvec) {
       const uint4 w = src[idx];
       const uint32_t u[4] = {w.x, w.y, w.z, w.w};
@@ -263,12 +263,18 @@ softmax_rows_kernel(const __nv_bfloat16* s, __nv_bfloat16* pout, int cols, float
       }
     }
   }
+  // this thread's statistics; the exponentials are kept (relative to the thread's own maximum) and only
+  // rescaled once the row's maximum is known: one exponential per element
+  const float m_own = m;
   float d = 0.f;
 #pragma unroll
   for (int v = 0; v < VPT; ++v)
-    if (v * kSoftmaxThreads + threadIdx.x < nvec) {
+    if (v * THREADS + threadIdx.x < nvec) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) d += exp2f(x[v][e] - m);
+      for (int e = 0; e < 8; ++e) {
+        x[v][e] = ex2_approx(x[v][e] - m_own);
+        d += x[v][e];
+      }
     }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
@@ -279,17 +285,17 @@ softmax_rows_kernel(const __nv_bfloat16* s, __nv_bfloat16* pout, int cols, float
   __syncthreads();
   float mr = sm_m[0], dr = sm_d[0];
 #pragma unroll
-  for (int w = 1; w < kSoftmaxThreads / 32; ++w) merge_md(mr, dr, sm_m[w], sm_d[w]);
-  const float inv = 1.0f / dr;
+  for (int w = 1; w < THREADS / 32; ++w) merge_md(mr, dr, sm_m[w], sm_d[w]);
+  const float f = (m_own == -INFINITY) ? 0.f : exp2f(m_own - mr) / dr;
 #pragma unroll
   for (int v = 0; v < VPT; ++v) {
-    const int idx = v * kSoftmaxThreads + threadIdx.x;
+    const int idx = v * THREADS + threadIdx.x;
     if (idx < nvec) {
       uint4 w;
-      w.x = pack_bf16x2(exp2f(x[v][0] - mr) * inv, exp2f(x[v][1] - mr) * inv);
-      w.y = pack_bf16x2(exp2f(x[v][2] - mr) * inv, exp2f(x[v][3] - mr) * inv);
-      w.z = pack_bf16x2(exp2f(x[v][4] - mr) * inv, exp2f(x[v][5] - mr) * inv);
-      w.w = pack_bf16x2(exp2f(x[v][6] - mr) * inv, exp2f(x[v][7] - mr) * inv);
+      w.x = pack_bf16x2(x[v][0] * f, x[v][1] * f);
+      w.y = pack_bf16x2(x[v][2] * f, x[v][3] * f);
+      w.z = pack_bf16x2(x[v][4] * f, x[v][5] * f);
+      w.w = pack_bf16x2(x[v][6] * f, x[v][7] * f);
       dst[idx] = w;
     }
   }
