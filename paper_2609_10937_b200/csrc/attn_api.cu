@@ -123,7 +123,7 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   if ((rc = make_tmap(&tq, q, BH, L, D, attn::kSub)) != ATTN_OK) return rc;
   if ((rc = make_tmap(&tk, k, BH, L, D, TKV)) != ATTN_OK) return rc;
   if ((rc = make_tmap(&tv, v, BH, L, D, TKV)) != ATTN_OK) return rc;
-  if ((rc = make_tmap(&to, o, BH, L, D, attn::kSub)) != ATTN_OK) return rc;
+  if ((rc = make_tmap(&to, o, BH, L, D, 32)) != ATTN_OK) return rc;    // every warp stores its own 32 rows
 
   attn::FwdParams p;
   p.L = L;
@@ -140,9 +140,10 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   p.ws = ws ? ws + attn::kCounterBytes / sizeof(float) : nullptr;    // partial results follow
   const int grid = t.ctas;
   const long long total_units = p.head_units * BH;
-  // at least one KV step per CTA; two arrival counters per CTA must fit the counter block
+  // at least one KV step per CTA; when Q tiles are shared, the counters of every (CTA, sub-tile, warp) --
+  // two each -- must fit the counter block
   if (grid < 1 || (long long)grid > total_units) return ATTN_ERR_BAD_TILES;
-  if ((size_t)grid * NQ > attn::kCounterBytes / sizeof(unsigned int)) return ATTN_ERR_BAD_TILES;
+  if (ws && (size_t)grid * NQ * 8 > attn::kCounterBytes / sizeof(unsigned int)) return ATTN_ERR_BAD_TILES;
   const int smem = SM::total(t.kv_stages);
   if (p.causal) {
     auto kern = attn::attn_fwd_kernel<D, TKV, NQ, true>;

@@ -260,11 +260,9 @@ struct FwdMisc {               // lives in the last 3072 bytes of dynamic shared
   uint64_t p_half[2];          // second half of P written
   uint64_t o_full[2];
   uint64_t alpha_full[2];
-  uint64_t epi_sync[2];        // softmax warpgroup rendezvous in the epilogue
   uint64_t q_empty;            // every product that reads the Q tile of a segment has finished
   uint64_t o_free[2];          // the epilogue of a segment has read its O accumulator
   uint64_t dbg_bar[2];         // trace builds only: completion of the first half of P V
-  uint32_t ticket[2];          // arrival order of this CTA among the splits of its Q sub-tile
   uint32_t tmem_slot;
   int abort_flag;
 };
@@ -422,7 +420,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(smem_u32(&misc->p_half[i]), kSub);
       mbar_init(smem_u32(&misc->o_full[i]), 1);
       mbar_init(smem_u32(&misc->alpha_full[i]), kSub);
-      mbar_init(smem_u32(&misc->epi_sync[i]), kSub);
       mbar_init(smem_u32(&misc->dbg_bar[i]), 1);
       mbar_init(smem_u32(&misc->o_free[i]), kSub);
     }
@@ -458,18 +455,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t bar_p = smem_u32(&misc->p_full[i]);
     const uint32_t bar_h = smem_u32(&misc->p_half[i]);
     const uint32_t bar_a = smem_u32(&misc->alpha_full[i]);
-    const uint32_t bar_e = smem_u32(&misc->epi_sync[i]);
     const float scale = p.scale_log2;
     const ExpConsts ek = make_exp_consts(scale);
     const size_t per_sub = ws_floats_per_sub(D);
     const int kv_tail = p.L % TKV;                     // valid keys in a ragged last KV tile (0: none ragged)
-    uint32_t ep_phase = 0;
-    auto wg_sync = [&](uint32_t tag) -> bool {          // all 128 threads of this warpgroup, bounded
-      mbar_arrive(bar_e);
-      const bool r = wait_bar_warp(bar_e, ep_phase, abort_flag, wait_info(kRoleSoftmax, kBarSync, tag));
-      ep_phase ^= 1u;
-      return r;
-    };
     bool ok = run;
     uint32_t g = 0;
     if (ok) {
@@ -586,138 +575,255 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
       // ----------------------------------------------------- end of segment
+      // Each warp finishes its own 32 rows without meeting the other warps of its warpgroup.
       if (warp == 0) ATTN_TRACE_MARK(3);
       if (ok) ok = wait_bar_warp(smem_u32(&misc->o_full[i]), (g - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, g));
       if (!ok) break;
       tc_fence_after();
       if (warp == 0) ATTN_TRACE_MARK(4);
+      const int wq = warp & 3;                               // which 32 rows of the sub-tile
+      // This warp's staging: [32 rows][64 columns] bf16 chunks.  Before the CTA's last segment there is one
+      // (the next Q tile may already be arriving in the Q buffer) and the two halves of a 128-wide row take
+      // turns; for a whole tile on the last segment the warp's slice of its sub-tile's dead Q buffer holds all
+      // halves at once (when the last segment ends in a merge, that slice receives the other parts instead).
       const bool last_seg = (u >= u_hi);                     // u was advanced past this segment already
-      // Normalised values of one 32-column chunk of this thread's output row -> memory, always through
-      // shared memory and a TMA store (coalesced, and rows past the end of the sequence are clipped by the
-      // tensor map).  On the CTA's last segment the Q buffer is dead and takes the whole sub-tile; before
-      // that the next segment's Q tile may already be arriving there, so the rows go through this
-      // warpgroup's [128][64] staging chunk, one 64-column half of the row at a time.
-      auto put_chunk = [&](int c, const float (&val)[32]) -> bool {
-        if (last_seg) {
-          stage_row_chunk(q_smem + i * (kSub * D * 2), c, row, val);
-          return true;
-        }
-        const uint32_t stage_out = out_smem + i * (kSub * 128);
-        stage_row_chunk(stage_out, c & 1, row, val);
-        if ((c & 1) == 0) return true;
+      const bool q_stage = last_seg && sg.full;
+      const uint32_t stage_w = q_stage ? q_smem + warp * (KCH * 4096) : out_smem + warp * 4096;
+      // 64 normalised columns of this warp's rows -> memory through the staging chunk and a TMA store
+      // (coalesced; rows past the end of the sequence are clipped by the tensor map).
+      auto store_half = [&](int h, const float (&v0)[32], const float (&v1)[32]) {
+        const uint32_t dst = q_stage ? stage_w + h * 4096 : stage_w;
+        stage_row_chunk(dst, 0, lane, v0);
+        stage_row_chunk(dst, 1, lane, v1);
+        if (q_stage && h < KCH - 1) return;
         fence_proxy_async_smem();
-        bool r = wg_sync(4);
-        if (r && (warp & 3) == 0 && lane == 0) {
-          tma_store_3d(&tm_o, stage_out, (c >> 1) * 64, q_row0 + i * kSub, bh);
-          tma_store_commit();
-          tma_store_wait_read();
-        }
-        if (r) r = wg_sync(5);                               // the staging chunk may be written again
-        return r;
-      };
-      auto finish_rows = [&]() -> bool {                     // after put_chunk on the last segment
-        if (!last_seg) return true;
-        const uint32_t stage_out = q_smem + i * (kSub * D * 2);
-        fence_proxy_async_smem();
-        const bool r = wg_sync(3);
-        if (r && (warp & 3) == 0 && lane == 0) {
+        __syncwarp();
+        if (lane == 0) {
+          if (q_stage) {
 #pragma unroll
-          for (int c = 0; c < KCH; ++c)
-            tma_store_3d(&tm_o, stage_out + c * (kSub * 128), c * 64, q_row0 + i * kSub, bh);
+            for (int hh = 0; hh < KCH; ++hh)
+              tma_store_3d(&tm_o, stage_w + hh * 4096, hh * 64, q_row0 + i * kSub + wq * 32, bh);
+          } else {
+            tma_store_3d(&tm_o, stage_w, h * 64, q_row0 + i * kSub + wq * 32, bh);
+          }
           tma_store_commit();
           tma_store_wait_read();
         }
-        return r;
+        __syncwarp();                                        // the staging chunk may be written again
       };
       if (sg.full) {
         // The whole Q tile was processed here: normalise and store.
         const float inv = 1.0f / delta;
 #pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t r[32];
-          float val[32];
-          tmem_ld32(o_tmem + c * 32, r);
-#pragma unroll
-          for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(r[k]) * inv;
-          if (!put_chunk(c, val)) { ok = false; break; }
-        }
-        tc_fence_before();
-        mbar_arrive(smem_u32(&misc->o_free[i]));             // O may be overwritten by the next segment
-        if (ok) ok = finish_rows();
-      } else {
-        // Part of a Q tile: un-normalised partial (O, m, delta) of this key range.  A CTA has at most two
-        // such pieces, its first and its last segment: slots 2*cta and 2*cta + 1.
-        float* ws = p.ws + ((size_t)(2 * cta + (seg == 0 ? 0 : 1)) * NQ + i) * per_sub;
-        {
-          uint32_t r[D];
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) tmem_ld32_nowait(o_tmem + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[c * 32]));
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&r[c * 32]));
-#pragma unroll
-          for (int gq = 0; gq < D / 4; ++gq) {
-            float4 v4 = make_float4(__uint_as_float(r[gq * 4]), __uint_as_float(r[gq * 4 + 1]),
-                                    __uint_as_float(r[gq * 4 + 2]), __uint_as_float(r[gq * 4 + 3]));
-            reinterpret_cast<float4*>(ws)[(size_t)gq * kSub + row] = v4;
+        for (int h = 0; h < KCH; ++h) {
+          uint32_t r0[32], r1[32];
+          float v0[32], v1[32];
+          tmem_ld32_nowait(o_tmem + h * 64, r0);
+          tmem_ld32_nowait(o_tmem + h * 64 + 32, r1);
+          tmem_ld_fence(r0);
+          tmem_ld_fence(r1);
+          if (h == KCH - 1) {
+            tc_fence_before();
+            mbar_arrive(smem_u32(&misc->o_free[i]));         // O may be overwritten by the next segment
           }
+#pragma unroll
+          for (int k = 0; k < 32; ++k) { v0[k] = __uint_as_float(r0[k]) * inv; v1[k] = __uint_as_float(r1[k]) * inv; }
+          store_half(h, v0, v1);
         }
-        tc_fence_before();
-        mbar_arrive(smem_u32(&misc->o_free[i]));             // O may be overwritten by the next segment
-        ws[(size_t)kSub * D + row] = m_run;
-        ws[(size_t)kSub * D + kSub + row] = delta;
-        __threadfence();
-        if (warp == 0) ATTN_TRACE_MARK(5);
-        // CTAs that share this Q tile: those whose ranges meet the tile's units; the first of them owns
-        // the tile's arrival counter.
+      } else {
+        // Part of a Q tile shared with other CTAs (those whose ranges meet the tile's units; the first of
+        // them owns the tile's counters).  Per warp: counter A orders the CTAs by when they finished their
+        // key range; all but the last publish their un-normalised partial (O, m, delta) -- slots 2*cta and
+        // 2*cta+1: a CTA has at most two partial pieces, its first and its last segment -- and signal that on
+        // counter B without waiting; the last one keeps its part in tensor memory, waits for B and merges
+        // all parts in ascending key order (the merge operator of the online softmax), so the result does
+        // not depend on who merges.
         const int c_first = cta_of_unit(sg.unit0, T, G);
         const int c_last = cta_of_unit(sg.unit0 + sg.steps_t - 1, T, G);
-        ok = wg_sync(1);
-        if (ok) {
-          if (row == 0) misc->ticket[i] = atomicAdd(&p.counters[c_first * NQ + i], 1u);
-          ok = wg_sync(2);
-        }
-        if (!ok) break;
-        if (warp == 0) ATTN_TRACE_MARK(6);
-        if (*reinterpret_cast<volatile uint32_t*>(&misc->ticket[i]) == (uint32_t)(c_last - c_first)) {
-          // Last one to finish: merge all parts in ascending key order (the merge operator of the
-          // online softmax), independent of arrival order, and write the rows of this sub-tile.
-          if (row == 0) p.counters[c_first * NQ + i] = 0u;
+        const int parts = c_last - c_first + 1, mine = cta - c_first;
+        unsigned int* ctr = p.counters + (((size_t)(c_first * NQ + i) * 4 + wq) << 1);
+        uint32_t order = 0;
+        if (lane == 0) order = atomicAdd(&ctr[0], 1u);
+        order = __shfl_sync(0xffffffffu, order, 0);
+        if (warp == 0) ATTN_TRACE_MARK(5);
+        if (order != (uint32_t)(parts - 1)) {
+          float* ws = p.ws + ((size_t)(2 * cta + (seg == 0 ? 0 : 1)) * NQ + i) * per_sub;
+#pragma unroll 1
+          for (int hcol = 0; hcol < D / 64; ++hcol) {
+            uint32_t r[64];
+            tmem_ld32_nowait(o_tmem + hcol * 64, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+            tmem_ld32_nowait(o_tmem + hcol * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+            tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+            tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+#pragma unroll
+            for (int gq = 0; gq < 16; ++gq) {
+              float4 v4 = make_float4(__uint_as_float(r[gq * 4]), __uint_as_float(r[gq * 4 + 1]),
+                                      __uint_as_float(r[gq * 4 + 2]), __uint_as_float(r[gq * 4 + 3]));
+              reinterpret_cast<float4*>(ws)[(size_t)(hcol * 16 + gq) * kSub + row] = v4;
+            }
+          }
+          tc_fence_before();
+          mbar_arrive(smem_u32(&misc->o_free[i]));           // O may be overwritten by the next segment
+          ws[(size_t)kSub * D + row] = m_run;
+          ws[(size_t)kSub * D + kSub + row] = delta;
           __threadfence();
-          const int parts = c_last - c_first + 1;
+          __syncwarp();                                      // the lanes' stores are ordered before lane 0's release
+          if (lane == 0) red_release_gpu_inc(&ctr[1]);
+        } else {
+          // wait (bounded) until the other parts are published
+          uint32_t seen = 1;
+          if (lane == 0) {
+            const long long t0 = clock64();
+            while (ld_acquire_gpu(&ctr[1]) < (uint32_t)(parts - 1)) {
+              if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { seen = 0; break; }
+              __nanosleep(100);                              // the publishers update this cache line: poll gently
+            }
+            if (!seen && !*abort_flag) {
+              report_timeout(wait_info(kRoleSoftmax, kBarSync, 0x7000 | (uint32_t)wq));
+              *abort_flag = 1;
+            }
+          }
+          seen = __shfl_sync(0xffffffffu, seen, 0);
+          if (!seen) { ok = false; break; }
+          __threadfence();
+          if (lane == 0) { ctr[0] = 0u; ctr[1] = 0u; }       // ready for the next launch
+          if (warp == 0) ATTN_TRACE_MARK(6);
           // part sp comes from CTA c_first + sp: its first piece if its range starts inside this tile
           auto part_ptr = [&](int sp) -> const float* {
             const int c = c_first + sp;
             const int slot = (range_begin(c, T, G) >= sg.unit0) ? 0 : 1;
             return p.ws + ((size_t)(2 * c + slot) * NQ + i) * per_sub;
           };
-          float m_all = -INFINITY;
-#pragma unroll 4
-          for (int sp = 0; sp < parts; ++sp) m_all = fmaxf(m_all, __ldcg(part_ptr(sp) + (size_t)kSub * D + row));
-          // whole output row accumulated in registers: per part all loads are independent and in flight together
-          float val[D];
+          if (last_seg && parts <= 4) {
+            // Usual case.  The other CTAs' parts are copied asynchronously, 32 columns of this warp's rows at
+            // a time, into the warp's slice of the dead Q buffer while the previous piece is accumulated, so
+            // that the round trips to L2 overlap instead of following one another.
+            constexpr int NBUF = KCH;                         // 4 KB pieces the slice holds
+            const uint32_t inb = q_smem + warp * (KCH * 4096) + lane * 16;
+            const float* pp[4];
 #pragma unroll
-          for (int k = 0; k < D; ++k) val[k] = 0.f;
-          float d_all = 0.f;
-          for (int sp = 0; sp < parts; ++sp) {
-            const float* b = part_ptr(sp);
-            const float w = exp2f(__ldcg(b + (size_t)kSub * D + row) - m_all);
-            d_all += __ldcg(b + (size_t)kSub * D + kSub + row) * w;
+            for (int sp = 0; sp < 4; ++sp) pp[sp] = part_ptr(sp < parts ? sp : 0);
+            const int n_other = parts - 1, n_items = (D / 32) * n_other;
+            auto issue = [&](int k) {                         // item k: chunk k / n_other of the (k % n_other)-th other part
+              const int c = k / n_other, o = k - c * n_other, sp = o < mine ? o : o + 1;
+              const float* base = sp == 0 ? pp[0] : sp == 1 ? pp[1] : sp == 2 ? pp[2] : pp[3];
+              const float4* src = reinterpret_cast<const float4*>(base) + (size_t)(c * 8) * kSub + row;
+              const uint32_t dst = inb + (uint32_t)(k % NBUF) * 4096;
 #pragma unroll
-            for (int gq = 0; gq < D / 4; ++gq) {
-              const float4 v4 = __ldcg(reinterpret_cast<const float4*>(b) + (size_t)gq * kSub + row);
-              val[gq * 4 + 0] += w * v4.x;
-              val[gq * 4 + 1] += w * v4.y;
-              val[gq * 4 + 2] += w * v4.z;
-              val[gq * 4 + 3] += w * v4.w;
+              for (int gq = 0; gq < 8; ++gq) cp_async16(dst + gq * 512, src + (size_t)gq * kSub);
+              cp_async_commit();
+            };
+            for (int k = 0; k < NBUF && k < n_items; ++k) issue(k);
+            float mm[4], dd[4], ww[4];
+#pragma unroll
+            for (int sp = 0; sp < 4; ++sp) {
+              mm[sp] = -INFINITY;
+              dd[sp] = 0.f;
+              if (sp < parts) {
+                mm[sp] = (sp == mine) ? m_run : __ldcg(pp[sp] + (size_t)kSub * D + row);
+                dd[sp] = (sp == mine) ? delta : __ldcg(pp[sp] + (size_t)kSub * D + kSub + row);
+              }
             }
+            const float m_all = fmaxf(fmaxf(mm[0], mm[1]), fmaxf(mm[2], mm[3]));
+            float d_all = 0.f;
+#pragma unroll
+            for (int sp = 0; sp < 4; ++sp) {                   // ascending key order
+              ww[sp] = (sp < parts) ? exp2f(mm[sp] - m_all) : 0.f;
+              if (sp < parts) d_all += dd[sp] * ww[sp];
+            }
+            const float inv = 1.0f / d_all;
+            int k = 0;
+#pragma unroll 1
+            for (int h = 0; h < KCH; ++h) {
+              float val[64];
+#pragma unroll
+              for (int cc = 0; cc < 2; ++cc) {
+                float* v = &val[cc * 32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[e] = 0.f;
+#pragma unroll
+                for (int sp = 0; sp < 4; ++sp) {
+                  if (sp >= parts) continue;
+                  if (sp == mine) {
+                    uint32_t r[32];
+                    tmem_ld32(o_tmem + h * 64 + cc * 32, r);
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] += ww[sp] * __uint_as_float(r[e]);
+                  } else {
+                    if (NBUF == 2 && k + 1 < n_items) cp_async_wait<1>(); else cp_async_wait<0>();
+                    const uint32_t src = inb + (uint32_t)(k % NBUF) * 4096;
+#pragma unroll
+                    for (int gq = 0; gq < 8; ++gq) {
+                      const float4 v4 = ld_shared_f4(src + gq * 512);
+                      v[gq * 4 + 0] += ww[sp] * v4.x;
+                      v[gq * 4 + 1] += ww[sp] * v4.y;
+                      v[gq * 4 + 2] += ww[sp] * v4.z;
+                      v[gq * 4 + 3] += ww[sp] * v4.w;
+                    }
+                    if (k + NBUF < n_items) issue(k + NBUF);
+                    ++k;
+                  }
+                }
+              }
+              if (h == KCH - 1) {
+                tc_fence_before();
+                mbar_arrive(smem_u32(&misc->o_free[i]));     // O may be overwritten by the next segment
+              }
+#pragma unroll
+              for (int e = 0; e < 64; ++e) val[e] *= inv;
+              store_half(h, *reinterpret_cast<float(*)[32]>(&val[0]), *reinterpret_cast<float(*)[32]>(&val[32]));
+            }
+          } else {
+          // General case (a merge before the CTA's last segment, or more than four parts): from registers.
+          float m_all = m_run;
+#pragma unroll 4
+          for (int sp = 0; sp < parts; ++sp)
+            if (sp != mine) m_all = fmaxf(m_all, __ldcg(part_ptr(sp) + (size_t)kSub * D + row));
+          float d_all = 0.f;
+          for (int sp = 0; sp < parts; ++sp) {                // ascending key order, own part in its place
+            const float* b = part_ptr(sp);
+            const float m_sp = (sp == mine) ? m_run : __ldcg(b + (size_t)kSub * D + row);
+            const float d_sp = (sp == mine) ? delta : __ldcg(b + (size_t)kSub * D + kSub + row);
+            d_all += d_sp * exp2f(m_sp - m_all);
           }
           const float inv = 1.0f / d_all;
+#pragma unroll 1
+          for (int h = 0; h < KCH; ++h) {
+            float val[64];
 #pragma unroll
-          for (int k = 0; k < D; ++k) val[k] *= inv;
+            for (int k = 0; k < 64; ++k) val[k] = 0.f;
+            for (int sp = 0; sp < parts; ++sp) {
+              const float* b = part_ptr(sp);
+              if (sp == mine) {
+                const float w = exp2f(m_run - m_all);
+                uint32_t r[64];
+                tmem_ld32_nowait(o_tmem + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+                tmem_ld32_nowait(o_tmem + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+                tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+                tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&r[32]));
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c)
-            if (ok) ok = put_chunk(c, *reinterpret_cast<float(*)[32]>(&val[c * 32]));
-          if (ok) ok = finish_rows();
+                for (int k = 0; k < 64; ++k) val[k] += w * __uint_as_float(r[k]);
+              } else {
+                const float w = exp2f(__ldcg(b + (size_t)kSub * D + row) - m_all);
+#pragma unroll
+                for (int gq = 0; gq < 16; ++gq) {
+                  const float4 v4 = __ldcg(reinterpret_cast<const float4*>(b) + (size_t)(h * 16 + gq) * kSub + row);
+                  val[gq * 4 + 0] += w * v4.x;
+                  val[gq * 4 + 1] += w * v4.y;
+                  val[gq * 4 + 2] += w * v4.z;
+                  val[gq * 4 + 3] += w * v4.w;
+                }
+              }
+            }
+            if (h == KCH - 1) {
+              tc_fence_before();
+              mbar_arrive(smem_u32(&misc->o_free[i]));       // O may be overwritten by the next segment
+            }
+#pragma unroll
+            for (int k = 0; k < 64; ++k) val[k] *= inv;
+            store_half(h, *reinterpret_cast<float(*)[32]>(&val[0]), *reinterpret_cast<float(*)[32]>(&val[32]));
+          }
+          }
         }
       }
       }
