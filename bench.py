@@ -274,6 +274,24 @@ def run_ours(args):
             "compulsory_traffic_bytes": traffic.fused_bytes(case.B, case.H, case.L, case.d, 2),
         },
     }
+    if world == 1 and not args.no_extras:
+        # Context beside the headline (not part of the timed region above): the same problem through the
+        # unfused three-kernel path, and the paper's other workload, the 4096^3 matrix product.
+        scores = torch.empty(case.B * case.H * case.L * case.L, dtype=torch.bfloat16, device="cuda")
+        u_ms, _, _, _ = timed(lambda: binding.forward_unfused(dq, dk, dv, scores, do), 10, 3)
+        del scores
+        line["unfused_baseline"] = {
+            "ms_per_step": u_ms, "value": flops / (u_ms * 1e-3) / 1e12, "unit": UNIT, "kernels_per_step": 3,
+            "fused_speedup": u_ms / ms,
+            "path": "attn_forward_unfused: S = Q K^T to HBM (bf16), row softmax in place, P V; same inputs",
+            "analytic_traffic_bytes": traffic.unfused_bytes(case.B, case.H, case.L, case.d, 2, 2)}
+        ga = torch.randn(4096, 4096, device="cuda").to(torch.bfloat16)
+        gb = torch.randn(4096, 4096, device="cuda").to(torch.bfloat16)
+        gc = torch.empty(4096, 4096, dtype=torch.bfloat16, device="cuda")
+        g_ms, _, _, _ = timed(lambda: binding.gemm(ga, gb, gc), 20, 3)
+        g_tf = 2.0 * 4096 ** 3 / (g_ms * 1e-3) / 1e12
+        line["gemm"] = {"workload": "C = A B, 4096 x 4096 x 4096, bf16 in/out, fp32 accumulate, closed-form tiles",
+                        "ms_per_step": g_ms, "value": g_tf, "unit": UNIT, "frac_of_measured_peak": g_tf / peaks["bf16_tflops"]}
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = {k_: v_ for k_, v_ in cpu_baseline(case, q, k, v).items() if k_ != "seconds"}
     print(json.dumps(line), flush=True)
@@ -289,6 +307,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the unfused-path and matrix-product context numbers")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
