@@ -145,15 +145,17 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   if (grid < 1 || (long long)grid > total_units) return ATTN_ERR_BAD_TILES;
   if (ws && (size_t)grid * NQ * 8 > attn::kCounterBytes / sizeof(unsigned int)) return ATTN_ERR_BAD_TILES;
   const int smem = SM::total(t.kv_stages);
-  if (p.causal) {
-    auto kern = attn::attn_fwd_kernel<D, TKV, NQ, true>;
+  // uniform key split (k CTAs per tile, all parts of a tile finish together): the eager-publish instantiation
+  const bool eager = !p.causal && t.ctas > t.tiles && t.ctas % t.tiles == 0;
+  auto launch = [&](auto kern) -> int {
     ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
-  } else {
-    auto kern = attn::attn_fwd_kernel<D, TKV, NQ, false>;
-    ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
-  }
+    return ATTN_OK;
+  };
+  if (p.causal) rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, true, false>);
+  else if (eager) rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, false, true>);
+  else rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, false, false>);
+  if (rc != ATTN_OK) return rc;
   ATTN_CUDA_TRY(cudaGetLastError());
   t_launch_count = 1;
   return ATTN_OK;

@@ -364,7 +364,7 @@ __device__ __forceinline__ void stage_row_chunk(uint32_t stage_out, int c, int r
   }
 }
 
-template <int D, int TKV, int NQ, bool CAUSAL>
+template <int D, int TKV, int NQ, bool CAUSAL, bool EAGER>
 __global__ void __launch_bounds__(512, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -642,11 +642,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int c_last = cta_of_unit(sg.unit0 + sg.steps_t - 1, T, G);
         const int parts = c_last - c_first + 1, mine = cta - c_first;
         unsigned int* ctr = p.counters + (((size_t)(c_first * NQ + i) * 4 + wq) << 1);
-        uint32_t order = 0;
-        if (lane == 0) order = atomicAdd(&ctr[0], 1u);
-        order = __shfl_sync(0xffffffffu, order, 0);
-        if (warp == 0) ATTN_TRACE_MARK(5);
-        if (order != (uint32_t)(parts - 1)) {
+        auto write_partial = [&]() {
           float* ws = p.ws + ((size_t)(2 * cta + (seg == 0 ? 0 : 1)) * NQ + i) * per_sub;
 #pragma unroll 1
           for (int hcol = 0; hcol < D / 64; ++hcol) {
@@ -662,10 +658,23 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               reinterpret_cast<float4*>(ws)[(size_t)(hcol * 16 + gq) * kSub + row] = v4;
             }
           }
-          tc_fence_before();
-          mbar_arrive(smem_u32(&misc->o_free[i]));           // O may be overwritten by the next segment
           ws[(size_t)kSub * D + row] = m_run;
           ws[(size_t)kSub * D + kSub + row] = delta;
+        };
+        uint32_t order = 0;
+        if (lane == 0) order = atomicAdd(&ctr[0], 1u);
+        // When all parts of a tile finish together (a uniform key split: the EAGER instantiation), the partial
+        // is written while that answer is on its way -- the last finisher then writes it in vain, but nobody
+        // waits for a publisher that has not even started.  With staggered finishes (balanced ranges) only the
+        // publishers write.
+        // EAGER instantiation: the partial is written while the answer is on its way.
+        if constexpr (EAGER) write_partial();
+        order = __shfl_sync(0xffffffffu, order, 0);
+        if (warp == 0) ATTN_TRACE_MARK(5);
+        if (order != (uint32_t)(parts - 1)) {
+          if constexpr (!EAGER) write_partial();
+          tc_fence_before();
+          mbar_arrive(smem_u32(&misc->o_free[i]));           // O may be overwritten by the next segment
           __threadfence();
           __syncwarp();                                      // the lanes' stores are ordered before lane 0's release
           if (lane == 0) red_release_gpu_inc(&ctr[1]);
