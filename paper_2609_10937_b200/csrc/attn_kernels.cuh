@@ -180,12 +180,21 @@ __host__ __device__ __forceinline__ int tile_steps(int n_steps, int ratio, int c
   const long long s = (long long)(q + 1) * ratio;
   return s < n_steps ? (int)s : n_steps;
 }
-// Units of Q tiles 0..q-1 of one head (closed form: a triangular number until the step count saturates).
+// Causal tiles are short at the start of a head, and starting and finishing a piece of a tile costs a CTA
+// about as much as a few KV steps.  So that equal ranges of the line mean equal time, every causal tile is
+// preceded on the line by kCausalTileCost units that stand for that cost: a CTA whose range covers them
+// simply has fewer real steps.  (Non-causal tiles all have the same length: nothing to even out.)
+#ifndef ATTN_CAUSAL_TILE_COST
+#define ATTN_CAUSAL_TILE_COST 3
+#endif
+constexpr int kCausalTileCost = ATTN_CAUSAL_TILE_COST;
+// Units of Q tiles 0..q-1 of one head (closed form: a triangular number until the step count saturates;
+// causal: plus the cost units of those tiles).
 __host__ __device__ __forceinline__ long long tile_prefix(int n_steps, int ratio, int causal, int q) {
   if (!causal) return (long long)q * n_steps;
   long long qc = n_steps / ratio;
   if (qc > q) qc = q;
-  return (long long)ratio * qc * (qc + 1) / 2 + (long long)(q - qc) * n_steps;
+  return (long long)ratio * qc * (qc + 1) / 2 + (long long)(q - qc) * n_steps + (long long)kCausalTileCost * q;
 }
 __device__ __forceinline__ long long range_begin(long long c, long long T, long long G) { return (c * T) / G; }
 __device__ __forceinline__ int cta_of_unit(long long u, long long T, long long G) {
@@ -193,7 +202,7 @@ __device__ __forceinline__ int cta_of_unit(long long u, long long T, long long G
 }
 template <bool V>
 struct MaskTag { static constexpr bool value = V; };
-struct Segment { int tile, q, j0, j1, n, bh, q_row0, seg, steps_t; bool full; long long unit0; };
+struct Segment { int tile, q, j0, j1, n, bh, q_row0, seg, steps_t; bool full; long long unit0; };   // unit0: the tile's first real unit
 // Q tile (head, index) that owns unit u, and the unit at which that tile starts.
 // Next piece of the unit range [u, u_hi) that lies inside one Q tile; advances u and the segment counter.
 // (Scalar arguments and straight-line code on purpose: the non-causal instantiation must stay as lean as
@@ -209,27 +218,38 @@ __device__ __forceinline__ bool next_segment(long long& u, long long u_hi, int& 
     sg.q = sg.tile % q_tiles;
     sg.steps_t = n_steps;
     sg.unit0 = (long long)sg.tile * n_steps;
+    const long long left = u_hi - u;
+    sg.j1 = (left < (long long)(sg.steps_t - sg.j0)) ? sg.j0 + (int)left : sg.steps_t;
+    sg.n = sg.j1 - sg.j0;
+    u += sg.n;
   } else {
-    sg.bh = (int)(u / head_units);
-    const long long r = u - (long long)sg.bh * head_units;
-    int lo = 0, hi = q_tiles - 1;                     // largest q with tile_prefix(q) <= r
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (tile_prefix(n_steps, ratio, 1, mid) <= r) lo = mid; else hi = mid - 1;
+    for (;;) {
+      sg.bh = (int)(u / head_units);
+      const long long r = u - (long long)sg.bh * head_units;
+      int lo = 0, hi = q_tiles - 1;                     // largest q with tile_prefix(q) <= r
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (tile_prefix(n_steps, ratio, 1, mid) <= r) lo = mid; else hi = mid - 1;
+      }
+      sg.q = lo;
+      sg.tile = sg.bh * q_tiles + lo;
+      const long long start = (long long)sg.bh * head_units + tile_prefix(n_steps, ratio, 1, lo);   // cost units first
+      sg.unit0 = start + kCausalTileCost;
+      sg.steps_t = tile_steps(n_steps, ratio, 1, lo);
+      long long end = sg.unit0 + sg.steps_t;
+      if (end > u_hi) end = u_hi;
+      const long long x0 = u - sg.unit0, x1 = end - sg.unit0;   // negative inside the cost units
+      sg.j0 = x0 > 0 ? (int)x0 : 0;
+      sg.j1 = x1 > 0 ? (int)x1 : 0;
+      sg.n = sg.j1 - sg.j0;
+      u = end;
+      if (sg.n > 0) break;
+      if (u >= u_hi) return false;                      // the range ended inside a tile's cost units
     }
-    sg.q = lo;
-    sg.tile = sg.bh * q_tiles + lo;
-    sg.unit0 = (long long)sg.bh * head_units + tile_prefix(n_steps, ratio, 1, lo);
-    sg.steps_t = tile_steps(n_steps, ratio, 1, lo);
-    sg.j0 = (int)(u - sg.unit0);
   }
-  const long long left = u_hi - u;
-  sg.j1 = (left < (long long)(sg.steps_t - sg.j0)) ? sg.j0 + (int)left : sg.steps_t;
-  sg.n = sg.j1 - sg.j0;
   sg.full = (sg.j0 == 0 && sg.j1 == sg.steps_t);
   sg.q_row0 = sg.q * tile_rows;
   sg.seg = seg_ctr++;
-  u += sg.n;
   return true;
 }
 
@@ -700,7 +720,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           // part sp comes from CTA c_first + sp: its first piece if its range starts inside this tile
           auto part_ptr = [&](int sp) -> const float* {
             const int c = c_first + sp;
-            const int slot = (range_begin(c, T, G) >= sg.unit0) ? 0 : 1;
+            const int slot = (range_begin(c, T, G) >= sg.unit0 - (CAUSAL ? kCausalTileCost : 0)) ? 0 : 1;
             return p.ws + ((size_t)(2 * c + slot) * NQ + i) * per_sub;
           };
           if (last_seg && parts <= 4) {
