@@ -297,3 +297,16 @@ def test_host_buffer_entry_point(env):
     got = (ho.view(torch.int16).numpy().view(np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
     ref = orc.attention_rows(q, k, v, 1, 2, 512, 128, np.arange(512, dtype=np.int32))
     assert_close(got.reshape(2, 512, 128), ref, "host entry")
+
+
+def test_shared_tile_counters_bound_the_grid(env):
+    """Grids whose CTAs share Q tiles keep two counters per warp of every (CTA, sub-tile) in the 64 KB counter block:
+    more than 1024 such CTAs are refused, not run."""
+    torch, _, binding = env
+    case = _case("limit", 1, 1, 8192, 64)                # 32 Q tiles x 128 steps of 64 keys = 4096 units
+    q, k, v = (to_cuda_bf16(x) for x in synth.make_qkv(case, 0))
+    with pytest.raises(binding.AttnError) as err:
+        binding.forward_tiles(q, k, v, ctas=1500, tile_kv=64)
+    assert err.value.code == binding.ERR_BAD_TILES
+    rows = synth.sample_rows(case.L)
+    _run_and_compare(env, case, lambda a, b, c: binding.forward_tiles(a, b, c, ctas=1024, tile_kv=64), rows=rows)

@@ -96,7 +96,7 @@ def test_row_softmax_matches_oracle(env, rows, cols):
     assert torch.equal(p2, p)
 
 
-@pytest.mark.parametrize("B,H,L,d", [(1, 1, 256, 64), (1, 2, 1024, 128), (2, 2, 520, 64), (1, 1, 4096, 128)])
+@pytest.mark.parametrize("B,H,L,d", [(1, 1, 256, 64), (1, 2, 1024, 128), (2, 2, 520, 64), (1, 1, 4096, 128), (1, 1, 16384, 128)])
 def test_unfused_attention_matches_its_oracle_and_the_fused_kernel(env, B, H, L, d):
     torch, go, binding = env
     from oracle import attn_oracle as orc
