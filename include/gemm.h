@@ -44,7 +44,8 @@ typedef struct gemm_tiles {
 /*
  * Tiles for C[batch][M][N] = A[batch][M][K] B (Eq. 2 and Eq. 3 re-derived for
  * tensor memory): tile_n = atom_n_max (atom_n_max / 2 if N <= atom_n_max / 2);
- * n_sub = min(2, acc_mem_columns / atom_n_max);
+ * n_sub = min(2, acc_mem_columns / atom_n_max), reduced to 1 if two-sub-tile blocks
+ * would be fewer than the compute units (occupancy);
  * tile_k = 128 bytes / elem_bytes; stages = min(8, (local_mem - staging - 1024)
  * / ((tile_m + tile_n) * tile_k * elem_bytes)), at least 2.  Pure host
  * arithmetic.  Returns ATTN_OK (then check out->feasible) or

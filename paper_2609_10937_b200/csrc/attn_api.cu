@@ -472,7 +472,8 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
   gemm_tiles t;
   if ((rc = gemm_plan(&st->desc, batch, M, N, K, &t)) != ATTN_OK) return rc;
   // the kernel is compiled for exactly the tile shape the derivation gives on this architecture
-  if (!t.feasible || t.tile_m != gemm::kTileM || (t.tile_n != 128 && t.tile_n != 256) || t.tile_k != gemm::kTileK ||
+  if (!t.feasible || (t.n_sub != 1 && t.n_sub != 2) || t.tile_m != t.n_sub * attn::kSub || (t.tile_n != 128 && t.tile_n != 256) ||
+      t.tile_k != gemm::kTileK ||
       t.stages > gemm::kMaxStages)
     return ATTN_ERR_INFEASIBLE_PLAN;
   CUtensorMap ta, tb, tc;
@@ -483,7 +484,8 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
   if ((rc = make_tmap_mat(&tc, c, batch, M, N, attn::kSub)) != ATTN_OK) return rc;
   gemm::GemmParams p;
   p.M = M; p.N = N; p.K = K; p.batch = batch;
-  p.m_tiles = (M + gemm::kTileM - 1) / gemm::kTileM;
+  p.n_sub = t.n_sub;
+  p.m_tiles = (M + t.tile_m - 1) / t.tile_m;
   p.n_tiles = (N + t.tile_n - 1) / t.tile_n;
   p.k_steps = (K + gemm::kTileK - 1) / gemm::kTileK;
   p.stages = t.stages;

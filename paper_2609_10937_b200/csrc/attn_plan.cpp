@@ -287,10 +287,14 @@ extern "C" int gemm_plan(const attn_hw_desc* desc, int batch, int M, int N, int 
   int n_sub = h.acc_mem_columns / h.atom_n_max;   // fp32 accumulator columns: one per output column and sub-tile
   if (n_sub > 2) n_sub = 2;
   if (n_sub < 1) return ATTN_OK;
+  // Occupancy: if two-sub-tile blocks would leave compute units without a tile, one sub-tile per block
+  // (twice as many blocks) is used instead -- the paper's "reduce tiles until occupancy is acceptable".
+  if (n_sub == 2 && (long long)batch * ceil_div(M, 2 * h.atom_m) * ceil_div(N, tile_n) < h.num_units) n_sub = 1;
   const int tile_m = n_sub * h.atom_m;
   const int tile_k = 128 / h.elem_bytes;       // one swizzle row
-  const int stage = (tile_m + tile_n) * tile_k * h.elem_bytes;
-  const int staging = n_sub * h.atom_m * 128;  // per sub-tile one 64-column chunk of the output rows
+  const int a_rows = (h.acc_mem_columns / h.atom_n_max >= 2 ? 2 : 1) * h.atom_m;   // the stage layout keeps room for two sub-tiles
+  const int stage = (a_rows + tile_n) * tile_k * h.elem_bytes;
+  const int staging = (a_rows / h.atom_m) * h.atom_m * 128;  // per sub-tile one 64-column chunk of the output rows
   int stages = (h.local_mem_bytes - staging - 1024) / stage;
   if (stages > 8) stages = 8;
   if (stages < 2) { out->binding_constraint = ATTN_BIND_SMEM; return ATTN_OK; }

@@ -34,7 +34,8 @@ enum Role : uint32_t { kRoleGemmLoad = 6, kRoleGemmMma = 7, kRoleGemmEpi = 8 };
 struct GemmParams {
   int M, N, K;
   int batch;
-  int m_tiles, n_tiles;   // ceil(M / 256), ceil(N / tile_n)
+  int n_sub;              // 128-row sub-tiles per CTA (1 or 2)
+  int m_tiles, n_tiles;   // ceil(M / (128 n_sub)), ceil(N / tile_n)
   int k_steps;            // ceil(K / 64)
   int stages;
 };
@@ -77,7 +78,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
       mbar_init(smem_u32(&misc->empty[s]), 1);
     }
     mbar_init(smem_u32(&misc->acc_full), 1);
-    mbar_init(smem_u32(&misc->acc_empty), 2 * kSub);
+    mbar_init(smem_u32(&misc->acc_empty), p.n_sub * kSub);
     mbar_init(smem_u32(&misc->epi_sync[0]), kSub);
     mbar_init(smem_u32(&misc->epi_sync[1]), kSub);
     fence_mbar_init();
@@ -94,6 +95,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
   tc_fence_after();
   const uint32_t tmem_base = misc->tmem_slot;
   const long long tiles = (long long)p.batch * p.m_tiles * p.n_tiles;
+  const int tile_m = p.n_sub * kSub;
   const bool run = (*abort_flag == 0);
 
   if (warp == 0) {
@@ -108,9 +110,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
           if (!attn::wait_bar(smem_u32(&misc->empty[stage]), phase ^ 1u, abort_flag, attn::wait_info(kRoleGemmLoad, 1, ks))) { ok = false; break; }
           const uint32_t bar = smem_u32(&misc->full[stage]);
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kStageA;
-          mbar_arrive_expect_tx(bar, kStageBytes);
-          tma_load_3d(a_dst, &tm_a, ks * kTileK, mt * kTileM, b, bar);
-          tma_load_3d(a_dst + kSub * 128, &tm_a, ks * kTileK, mt * kTileM + kSub, b, bar);
+          mbar_arrive_expect_tx(bar, kStageBytes - (2 - p.n_sub) * (kSub * kTileK * 2));
+          tma_load_3d(a_dst, &tm_a, ks * kTileK, mt * tile_m, b, bar);
+          if (p.n_sub == 2) tma_load_3d(a_dst + kSub * 128, &tm_a, ks * kTileK, mt * tile_m + kSub, b, bar);
           if (B_KN) {
 #pragma unroll
             for (int c = 0; c < kTileN / 64; ++c)
@@ -153,6 +155,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
           const uint32_t b_lo = B_KN ? attn::desc_lo(b_smem, kTileK * 128) : attn::desc_lo(b_smem, 16);
 #pragma unroll
           for (int sub = 0; sub < 2; ++sub) {
+            if (sub >= p.n_sub) break;
             const uint32_t a_lo = attn::desc_lo(a_smem + sub * (kSub * 128), 16);
 #pragma unroll
             for (int k16 = 0; k16 < kTileK / 16; ++k16) {
@@ -178,7 +181,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     const uint32_t stage_out = out_smem + sub * (kSub * 128);
     const bool leader = ((warp - 2) & 3) == 0 && lane == 0;
     uint32_t ep_phase = 0, tile_ctr = 0;
-    bool ok = run;
+    bool ok = run && sub < p.n_sub;
     auto group_sync = [&](uint32_t tag) -> bool {
       mbar_arrive(bar_e);
       const bool r = attn::wait_bar_warp(bar_e, ep_phase, abort_flag, attn::wait_info(kRoleGemmEpi, 3, tag));
@@ -206,7 +209,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         fence_proxy_async_smem();
         if (!(ok = group_sync(c))) break;
         if (leader) {
-          tma_store_3d(&tm_c, stage_out, nt * kTileN + (c >> 1) * 64, mt * kTileM + sub * kSub, b);
+          tma_store_3d(&tm_c, stage_out, nt * kTileN + (c >> 1) * 64, mt * tile_m + sub * kSub, b);
           tma_store_commit();
           tma_store_wait_read();
         }

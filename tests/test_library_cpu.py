@@ -50,8 +50,11 @@ def test_gemm_plan_closed_form(binding):
     assert t.stages == (232448 - 32768 - 1024) // 65536 == 3 and t.smem_bytes == 3 * 65536 + 32768 + 1024
     assert (t.tiles, t.ctas, t.feasible, t.tmem_columns) == (256, 148, 1, 512)
     assert t.wave_efficiency == pytest.approx(256 / (2 * 148))
+    # fewer two-sub-tile blocks than SMs (3 * 4 * 3 = 36 < 148): one sub-tile per block, twice as many blocks
     t = binding.gemm_plan(desc, 3, 1000, 520, 64)
-    assert (t.tiles, t.ctas) == (3 * 4 * 3, 36)
+    assert (t.n_sub, t.tile_m, t.tiles, t.ctas) == (1, 128, 3 * 8 * 3, 72)
+    t = binding.gemm_plan(desc, 1, 16384, 128, 16384)        # P V of the unfused path: 64 blocks -> 128
+    assert (t.n_sub, t.tile_n, t.tiles, t.ctas) == (1, 128, 128, 128)
     desc.acc_mem_columns = 256                      # half the tensor memory: one sub-tile
     t = binding.gemm_plan(desc, 1, 4096, 4096, 4096)
     assert (t.n_sub, t.tile_m, t.stages) == (1, 128, (232448 - 16384 - 1024) // 49152)
