@@ -120,12 +120,16 @@ def cpu_baseline(case, q, k, v, target_seconds=12.0):
     dt = max(time.perf_counter() - t0, 1e-6)
     n_rows = int(min(case.L, max(256, len(probe) * target_seconds / dt)))
     rows = np.unique(np.linspace(0, case.L - 1, n_rows).astype(np.int32))
-    t0 = time.perf_counter()
-    orc.attention_rows(q, k, v, case.B, case.H, case.L, case.d, rows)
-    dt = time.perf_counter() - t0
-    flops = 4.0 * case.B * case.H * len(rows) * case.L * case.d
+    # when even all rows take less than the target, the pass is repeated (at most 8 times) and the mean is reported
+    reps, dt = 0, 0.0
+    while reps < 8 and (reps == 0 or (len(rows) == case.L and dt < 0.8 * target_seconds)):
+        t0 = time.perf_counter()
+        orc.attention_rows(q, k, v, case.B, case.H, case.L, case.d, rows)
+        dt += time.perf_counter() - t0
+        reps += 1
+    flops = 4.0 * case.B * case.H * len(rows) * case.L * case.d * reps
     return {"value": flops / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{len(rows)} of {case.L} query rows per head, all keys, fp64, {dt:.2f} s",
+            "sample": f"{len(rows)} of {case.L} query rows per head, all keys, fp64, {reps} pass(es), {dt:.2f} s in all",
             "seconds": dt}
 
 
