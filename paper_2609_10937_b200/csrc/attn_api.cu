@@ -512,13 +512,15 @@ int softmax_launch(const void* s, void* pout, long long rows, int cols, float sc
   const __nv_bfloat16* sp = static_cast<const __nv_bfloat16*>(s);
   __nv_bfloat16* pp = static_cast<__nv_bfloat16*>(pout);
   const dim3 grid((unsigned)rows);
-  // threads x vectors per thread >= nvec, with at most four vectors per thread (register-light: several rows per SM)
+  // threads x vectors per thread >= nvec.  Small blocks (128 or 256 threads, the row in up to 8 -- for the widest
+  // rows 32 -- vectors per thread): several rows are then in flight per SM in different phases (load, reduce, store),
+  // which one large block per row does not give (measured: 1024-thread blocks reach half the bandwidth).
   if (nvec <= 128) gemm::softmax_rows_kernel<1, 128><<<grid, 128, 0, stream>>>(sp, pp, cols, scale_log2);
-  else if (nvec <= 256) gemm::softmax_rows_kernel<1, 256><<<grid, 256, 0, stream>>>(sp, pp, cols, scale_log2);
-  else if (nvec <= 512) gemm::softmax_rows_kernel<2, 256><<<grid, 256, 0, stream>>>(sp, pp, cols, scale_log2);
-  else if (nvec <= 1024) gemm::softmax_rows_kernel<2, 512><<<grid, 512, 0, stream>>>(sp, pp, cols, scale_log2);
-  else if (nvec <= 2048) gemm::softmax_rows_kernel<4, 512><<<grid, 512, 0, stream>>>(sp, pp, cols, scale_log2);
-  else gemm::softmax_rows_kernel<4, 1024><<<grid, 1024, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (nvec <= 256) gemm::softmax_rows_kernel<2, 128><<<grid, 128, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (nvec <= 512) gemm::softmax_rows_kernel<4, 128><<<grid, 128, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (nvec <= 1024) gemm::softmax_rows_kernel<4, 256><<<grid, 256, 0, stream>>>(sp, pp, cols, scale_log2);
+  else if (nvec <= 2048) gemm::softmax_rows_kernel<8, 256><<<grid, 256, 0, stream>>>(sp, pp, cols, scale_log2);
+  else gemm::softmax_rows_kernel<32, 128><<<grid, 128, 0, stream>>>(sp, pp, cols, scale_log2);
   ATTN_CUDA_TRY(cudaGetLastError());
   ++t_launch_count;
   return ATTN_OK;

@@ -243,63 +243,75 @@ __device__ __forceinline__ void merge_md(float& m, float& d, float m2, float d2)
 }
 
 template <int VPT, int THREADS>
-__global__ void __launch_bounds__(THREADS, 2048 / THREADS)
+__global__ void __launch_bounds__(THREADS)
 softmax_rows_kernel(const __nv_bfloat16* s, __nv_bfloat16* pout, int cols, float scale_log2) {
   __shared__ float sm_m[THREADS / 32], sm_d[THREADS / 32];
   const size_t row = blockIdx.x;
   const uint4* src = reinterpret_cast<const uint4*>(s + row * (size_t)cols);
   uint4* dst = reinterpret_cast<uint4*>(pout + row * (size_t)cols);
   const int nvec = cols / 8;
-  float x[VPT][8];
-  float m = -INFINITY;
+  // Pass 1 on the packed bf16 words: load, running maximum per lane pair (scale > 0 keeps the order).
+  uint32_t w[VPT][4];
+  uint32_t mx2 = 0xFF80FF80u;                               // (-inf, -inf) in bf16
 #pragma unroll
   for (int v = 0; v < VPT; ++v) {
     const int idx = v * THREADS + threadIdx.x;
     if (idx < nvec) {
-      const uint4 w = src[idx];
-      const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+      const uint4 q = src[idx];
+      w[v][0] = q.x; w[v][1] = q.y; w[v][2] = q.z; w[v][3] = q.w;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        x[v][2 * e] = __uint_as_float(u[e] << 16) * scale_log2;
-        x[v][2 * e + 1] = __uint_as_float(u[e] & 0xFFFF0000u) * scale_log2;
-        m = fmaxf(m, fmaxf(x[v][2 * e], x[v][2 * e + 1]));
-      }
+      for (int e = 0; e < 4; ++e) mx2 = max_bf16x2(mx2, w[v][e]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) w[v][e] = 0xFF80FF80u;    // -inf: weight 0
     }
   }
+  float m = fmaxf(__uint_as_float(mx2 << 16), __uint_as_float(mx2 & 0xFFFF0000u)) * scale_log2;
   // this thread's statistics; the exponentials are kept (relative to the thread's own maximum) and only
   // rescaled once the row's maximum is known: one exponential per element
   const float m_own = m;
-  float d = 0.f;
+  const float neg_m = (m_own == -INFINITY) ? 0.f : -m_own;
+  const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2), negm2 = pack_f32x2(neg_m, neg_m);
+  uint64_t x[VPT][4];
+  uint64_t d2 = 0ull;
 #pragma unroll
-  for (int v = 0; v < VPT; ++v)
-    if (v * THREADS + threadIdx.x < nvec) {
+  for (int v = 0; v < VPT; ++v) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        x[v][e] = ex2_approx(x[v][e] - m_own);
-        d += x[v][e];
-      }
+    for (int e = 0; e < 4; ++e) {
+      const uint64_t t = fma_f32x2(pack_f32x2(__uint_as_float(w[v][e] << 16), __uint_as_float(w[v][e] & 0xFFFF0000u)), scale2, negm2);
+      float t0, t1;
+      unpack_f32x2(t, t0, t1);
+      x[v][e] = pack_f32x2(ex2_approx(t0), ex2_approx(t1));
+      d2 = add_f32x2(d2, x[v][e]);
     }
+  }
+  float d0, d1;
+  unpack_f32x2(d2, d0, d1);
+  float d = d0 + d1;
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
-    const float m2 = __shfl_xor_sync(0xffffffffu, m, off), d2 = __shfl_xor_sync(0xffffffffu, d, off);
-    merge_md(m, d, m2, d2);
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, off), dd = __shfl_xor_sync(0xffffffffu, d, off);
+    merge_md(m, d, m2, dd);
   }
   if ((threadIdx.x & 31) == 0) { sm_m[threadIdx.x >> 5] = m; sm_d[threadIdx.x >> 5] = d; }
   __syncthreads();
   float mr = sm_m[0], dr = sm_d[0];
 #pragma unroll
-  for (int w = 1; w < THREADS / 32; ++w) merge_md(mr, dr, sm_m[w], sm_d[w]);
+  for (int k = 1; k < THREADS / 32; ++k) merge_md(mr, dr, sm_m[k], sm_d[k]);
   const float f = (m_own == -INFINITY) ? 0.f : exp2f(m_own - mr) / dr;
+  const uint64_t f2 = pack_f32x2(f, f);
 #pragma unroll
   for (int v = 0; v < VPT; ++v) {
     const int idx = v * THREADS + threadIdx.x;
     if (idx < nvec) {
-      uint4 w;
-      w.x = pack_bf16x2(x[v][0] * f, x[v][1] * f);
-      w.y = pack_bf16x2(x[v][2] * f, x[v][3] * f);
-      w.z = pack_bf16x2(x[v][4] * f, x[v][5] * f);
-      w.w = pack_bf16x2(x[v][6] * f, x[v][7] * f);
-      dst[idx] = w;
+      uint32_t o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float a0, a1;
+        unpack_f32x2(mul_f32x2(x[v][e], f2), a0, a1);
+        o[e] = pack_bf16x2(a0, a1);
+      }
+      dst[idx] = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
 }
