@@ -194,6 +194,22 @@ int attn_forward_simple(const void *q, const void *k, const void *v, void *o,
                         void *cuda_stream);
 
 /*
+ * attn_forward (causal == 0) or attn_forward_causal (causal != 0) with the tiles
+ * derived from a caller-supplied descriptor instead of the device's own: the
+ * paper's portability claim -- changing the hardware descriptor re-runs the same
+ * derivation, no code changes -- carried through to the launch.  `desc` must
+ * describe the current device or a smaller machine of the same architecture
+ * (no more compute units, local memory, registers or tensor-memory columns than
+ * the device has; same instruction atom), else ATTN_ERR_INVALID_ARG; a plan that
+ * no compiled kernel variant covers gives ATTN_ERR_BAD_TILES, one that does not
+ * fit gives ATTN_ERR_INFEASIBLE_PLAN.  Workspace as for attn_forward, sized with
+ * attn_workspace_bytes for the plan of that descriptor.  Other errors as
+ * attn_forward.
+ */
+int attn_forward_desc(const attn_hw_desc *desc, const void *q, const void *k, const void *v, void *o,
+                      int B, int H, int L, int d, int causal, void *cuda_stream);
+
+/*
  * Host-buffer form of attn_forward (the end-to-end path of Figure 2: Q, K, V
  * come from host memory, R goes back to it).  q_host, k_host, v_host, o_host
  * are HOST pointers (pinned memory for the copies to be asynchronous) in the

@@ -22,7 +22,7 @@ BIND_NAMES = ("none", "smem", "tmem", "reg", "atom", "shape")
 
 EXPORTED_SYMBOLS = (
     "attn_hw_desc_b200", "attn_hw_desc_query", "attn_plan", "attn_plan_ex", "attn_workspace_bytes",
-    "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_static_scratch",
+    "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_static_scratch", "attn_forward_desc",
     "attn_last_device_status",
     "attn_last_launch_count", "attn_status_string", "attn_last_cuda_error",
     "gemm_plan", "gemm_forward", "softmax_rows_forward", "attn_forward_unfused",
@@ -91,6 +91,7 @@ def lib() -> ctypes.CDLL:
         L.attn_forward_simple.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
         L.attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_size_t, vp]
         L.attn_forward_static_scratch.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+        L.attn_forward_desc.argtypes = [ctypes.POINTER(AttnHwDesc), vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.attn_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.attn_last_launch_count.argtypes = []
         L.attn_status_string.argtypes = [i32]
@@ -217,6 +218,20 @@ def forward_static_scratch(q, k, v, o):
     with torch.cuda.device(dev):
         _check(lib().attn_forward_static_scratch(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
                                                  B, H, L, d, stream), "attn_forward_static_scratch")
+    return o
+
+
+def forward_desc(desc: AttnHwDesc, q, k, v, o=None, causal=False):
+    """forward() with the tiles derived from `desc` (this device or a smaller machine of its architecture)."""
+    import torch
+
+    o, B, H, L, d, dev, stream = _prep(q, k, v, o)
+    with torch.cuda.device(dev):
+        t = plan(desc, B, H, L, d, causal=causal)
+        if t.feasible:
+            ensure_workspace(dev, workspace_bytes(t, B, H, L, d))
+        _check(lib().attn_forward_desc(ctypes.byref(desc), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                       B, H, L, d, 1 if causal else 0, stream), "attn_forward_desc")
     return o
 
 

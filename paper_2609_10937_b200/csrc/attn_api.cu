@@ -181,15 +181,27 @@ int dispatch_fwd(const void* q, const void* k, const void* v, void* o, int B, in
 bool plan_needs_workspace(const attn_tiles& t) { return t.causal != 0 || t.ctas != t.tiles; }
 
 int forward_impl(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d, int causal,
-                 const attn_tiles* ovr, void* cuda_stream) {
+                 const attn_tiles* ovr, void* cuda_stream, const attn_hw_desc* plan_desc = nullptr) {
   t_launch_count = 0;
   int rc = check_args(q, k, v, o, B, H, L, d);
   if (rc != ATTN_OK) return rc;
   DeviceState* st = nullptr;
   if ((rc = device_state(&st)) != ATTN_OK) return rc;
   if (ovr && ovr->causal) causal = 1;
+  if (plan_desc) {
+    // a caller-supplied descriptor must describe this device or a smaller machine of the same architecture
+    const attn_hw_desc& a = *plan_desc;
+    const attn_hw_desc& dv = st->desc;
+    if (a.struct_bytes != (int32_t)sizeof(attn_hw_desc)) return ATTN_ERR_INVALID_ARG;
+    if (a.num_units < 1 || a.num_units > dv.num_units || a.local_mem_bytes > dv.local_mem_bytes ||
+        a.regs_per_unit > dv.regs_per_unit || a.acc_mem_columns > dv.acc_mem_columns || a.acc_mem_columns <= 0 ||
+        a.acc_mem_lanes != dv.acc_mem_lanes || a.atom_m != dv.atom_m || a.atom_n != dv.atom_n || a.atom_k != dv.atom_k ||
+        a.atom_n_max > dv.atom_n_max || a.elem_bytes != dv.elem_bytes || a.simd_width != dv.simd_width)
+      return ATTN_ERR_INVALID_ARG;
+  }
+  const attn_hw_desc& desc = plan_desc ? *plan_desc : st->desc;
   attn_tiles t;
-  if ((rc = attn_plan_ex(&st->desc, B, H, L, d, causal, &t)) != ATTN_OK) return rc;
+  if ((rc = attn_plan_ex(&desc, B, H, L, d, causal, &t)) != ATTN_OK) return rc;
   if (!t.feasible) return ATTN_ERR_INFEASIBLE_PLAN;
   if (ovr) {
     if (ovr->n_q > 0) t.n_q = ovr->n_q;
@@ -198,7 +210,7 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
     if (t.tile_kv != 64 && t.tile_kv != 128) return ATTN_ERR_BAD_TILES;
     const int q_bytes = t.n_q * 128 * d * 2, stage = t.tile_kv * d * 2;
     const int reserve = 3072 + t.n_q * 128 * 128;   // barriers etc. + output staging (see FwdSmem)
-    int max_stages = (st->desc.local_mem_bytes - q_bytes - reserve) / stage;
+    int max_stages = (desc.local_mem_bytes - q_bytes - reserve) / stage;
     if (max_stages > attn::kMaxStages) max_stages = attn::kMaxStages;
     t.kv_stages = ovr->kv_stages > 0 ? ovr->kv_stages : max_stages;
     if (t.kv_stages < 2 || t.kv_stages > max_stages) return ATTN_ERR_BAD_TILES;
@@ -212,8 +224,8 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
     } else if (ovr->kv_splits > 0) {
       t.ctas = t.tiles * ovr->kv_splits;
     } else {
-      t.ctas = attn_internal::grid_size(st->desc, B * H, (L + t.tile_q - 1) / t.tile_q, steps, t.tile_q / t.tile_kv, causal,
-                                        2LL * L * d * st->desc.elem_bytes);
+      t.ctas = attn_internal::grid_size(desc, B * H, (L + t.tile_q - 1) / t.tile_q, steps, t.tile_q / t.tile_kv, causal,
+                                        2LL * L * d * desc.elem_bytes);
     }
     t.kv_splits = (t.ctas + t.tiles - 1) / t.tiles;
     if (t.ctas < 1) return ATTN_ERR_BAD_TILES;
@@ -297,6 +309,12 @@ extern "C" int attn_forward(const void* q, const void* k, const void* v, void* o
 extern "C" int attn_forward_causal(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
                                    void* cuda_stream) {
   return forward_impl(q, k, v, o, B, H, L, d, 1, nullptr, cuda_stream);
+}
+
+extern "C" int attn_forward_desc(const attn_hw_desc* desc, const void* q, const void* k, const void* v, void* o, int B, int H,
+                                 int L, int d, int causal, void* cuda_stream) {
+  if (!desc) return ATTN_ERR_INVALID_ARG;
+  return forward_impl(q, k, v, o, B, H, L, d, causal ? 1 : 0, nullptr, cuda_stream, desc);
 }
 
 extern "C" int attn_forward_tiles(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,

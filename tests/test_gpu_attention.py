@@ -317,3 +317,35 @@ def test_shared_tile_counters_bound_the_grid(env):
     assert err.value.code == binding.ERR_BAD_TILES
     rows = synth.sample_rows(case.L)
     _run_and_compare(env, case, lambda a, b, c: binding.forward_tiles(a, b, c, ctas=1024, tile_kv=64), rows=rows)
+
+
+@pytest.mark.parametrize("field,value,expect", [
+    ("num_units", 74, dict(ctas=64)),                                  # half the SMs: two CTAs per Q tile instead of four
+    ("local_mem_bytes", 166912, dict(tile_kv=64, binding_constraint=1)),   # less shared memory: smaller K/V tiles
+    ("acc_mem_columns", 256, dict(n_q=1)),                             # half the tensor memory: one Q sub-tile per CTA
+    ("cache_bytes", 0, dict()),                                        # no cache model
+])
+def test_other_descriptors_run_with_no_code_change(env, field, value, expect):
+    """The paper's portability claim carried to the launch: a changed descriptor re-runs the derivation and the same
+    kernels run with the tiles it gives (here: descriptors of smaller machines, on the B200 itself)."""
+    torch, _, binding = env
+    desc = binding.hw_desc_query(0)
+    setattr(desc, field, value)
+    case = _case("desc", 1, 2, 4096, 128)
+    plan = binding.plan(desc, case.B, case.H, case.L, case.d)
+    assert plan.feasible
+    for key, want in expect.items():
+        assert getattr(plan, key) == want, (key, getattr(plan, key))
+    _run_and_compare(env, case, lambda a, b, c: binding.forward_desc(desc, a, b, c), rows=synth.sample_rows(case.L))
+    _run_and_compare(env, case, lambda a, b, c: binding.forward_desc(desc, a, b, c, causal=True),
+                     rows=synth.sample_rows(case.L), causal=True)
+
+
+def test_descriptor_of_a_larger_machine_is_refused(env):
+    torch, _, binding = env
+    desc = binding.hw_desc_query(0)
+    desc.num_units += 1
+    case = _case("desc", 1, 1, 512, 64)
+    with pytest.raises(binding.AttnError) as err:
+        binding.forward_desc(desc, *(to_cuda_bf16(x) for x in synth.make_qkv(case, 0)))
+    assert err.value.code == -1
