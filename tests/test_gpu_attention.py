@@ -349,3 +349,15 @@ def test_descriptor_of_a_larger_machine_is_refused(env):
     with pytest.raises(binding.AttnError) as err:
         binding.forward_desc(desc, *(to_cuda_bf16(x) for x in synth.make_qkv(case, 0)))
     assert err.value.code == -1
+
+
+@pytest.mark.parametrize("B,H,L,d", [(1, 20, 2000, 128), (2, 40, 2047, 64), (1, 37, 1025, 128), (3, 50, 777, 64)])
+def test_persistent_grid_with_ragged_lengths(env, B, H, L, d):
+    """More Q tiles than SMs and little K/V per head: one persistent CTA per SM walks whole tiles and shares the ones at
+    its range ends; the ragged last Q tile is clipped by the staged TMA stores, the ragged last KV tile masked."""
+    _, _, binding = env
+    plan = binding.plan(binding.hw_desc_query(0), B, H, L, d)
+    assert plan.tiles > plan.ctas == binding.hw_desc_query(0).num_units
+    case = _case("persistent", B, H, L, d)
+    _run_and_compare(env, case, binding.forward)
+    _run_and_compare(env, case, lambda a, b, c: binding.forward(a, b, c, causal=True), causal=True)
