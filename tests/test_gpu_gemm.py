@@ -120,3 +120,34 @@ def test_unfused_attention_matches_its_oracle_and_the_fused_kernel(env, B, H, L,
     # and the definition itself (the fused kernel's oracle), at the looser bound the two extra roundings cost
     ref = orc.attention_rows(q, k, v, B, H, L, d, rows.astype(np.int32)).reshape(B * H, len(rows), d)
     assert np.abs(got[:, rows] - ref).max() <= 3e-2
+
+
+def test_unfused_entry_points_refuse_bad_arguments(env):
+    torch, _, binding = env
+    a = torch.zeros(64, 72, dtype=torch.bfloat16, device="cuda")
+    b = torch.zeros(72, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.AttnError) as err:                       # K = 70 is not a multiple of 8
+        binding.gemm(a[:, :70].contiguous(), b[:70].contiguous())
+    assert err.value.code == -2
+    with pytest.raises(binding.AttnError) as err:                       # c overlaps a
+        L = binding.lib()
+        rc = L.gemm_forward(a.data_ptr(), b.data_ptr(), a.data_ptr(), 1, 64, 64, 72, 0, None)
+        binding._check(rc, "gemm_forward")
+    assert err.value.code == -4
+    flat = torch.zeros(64 * 72 + 8, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.AttnError) as err:                       # pointer not 16-byte aligned
+        rc = binding.lib().gemm_forward(flat.data_ptr() + 2, b.data_ptr(), torch.empty(64, 64, dtype=torch.bfloat16, device="cuda").data_ptr(),
+                                        1, 64, 64, 72, 0, None)
+        binding._check(rc, "gemm_forward")
+    assert err.value.code == -3
+    s = torch.zeros(4, 100, dtype=torch.bfloat16, device="cuda")        # 100 columns: not a multiple of 8
+    with pytest.raises(binding.AttnError) as err:
+        binding.softmax_rows(s, 1.0)
+    assert err.value.code == -2
+    q = torch.zeros(1, 1, 256, 64, dtype=torch.bfloat16, device="cuda")
+    small = torch.empty(10, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.AttnError) as err:                       # score buffer too small
+        binding.forward_unfused(q, q.clone(), q.clone(), small)
+    assert err.value.code == -1
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0
