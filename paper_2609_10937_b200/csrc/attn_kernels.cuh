@@ -10,9 +10,10 @@
 //                          memory -> second tcgen05.mma (O += P V, A operand
 //                          read from tensor memory) ; a correction warpgroup
 //                          rescales O when the running maximum moved.
-//                          When CTAs split the key axis, each writes its partial
-//                          (O, m, delta) and the last one to finish merges them
-//                          with the merge operator of the online softmax.
+//                          CTAs walk equal ranges of the (Q tile, KV step) line.  Where
+//                          several CTAs share a Q tile, all but the last to finish publish
+//                          their partial (O, m, delta) and the last one merges them, per
+//                          warp, with the merge operator of the online softmax.
 //   attn_fwd_simple_kernel the same algorithm with nothing overlapped; used to
 //                          cross-check the pipelined kernel and the layouts.
 //
