@@ -98,7 +98,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     }
   }
 }
-// Same, for roles whose warps run warp-collective instructions afterwards: the verdict is made warp-uniform.
+// Same, for roles whose warps run warp-collective instructions afterwards: the outcome is made warp-uniform.
 __device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t info) {
   return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_flag, info) ? 1 : 0) != 0;
 }
