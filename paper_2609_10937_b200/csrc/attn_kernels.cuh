@@ -10,6 +10,9 @@
 //                          memory -> second tcgen05.mma (O += P V, A operand
 //                          read from tensor memory) ; a correction warpgroup
 //                          rescales O when the running maximum moved.
+//                          d = 64: P has tensor-memory columns of its own, so the
+//                          next step's Q K^T is issued as soon as the softmax
+//                          warpgroup holds the scores in registers.
 //                          CTAs walk equal ranges of the (Q tile, KV step) line.  Where
 //                          several CTAs share a Q tile, all but the last to finish publish
 //                          their partial (O, m, delta) and the last one merges them, per
@@ -283,6 +286,7 @@ struct FwdMisc {               // lives in the last 3072 bytes of dynamic shared
   uint64_t alpha_full[2];
   uint64_t q_empty;            // every product that reads the Q tile of a segment has finished
   uint64_t o_free[2];          // the epilogue of a segment has read its O accumulator
+  uint64_t s_free[2];          // d = 64: the softmax warpgroup holds the step's scores in registers
   uint64_t dbg_bar[2];         // trace builds only: completion of the first half of P V
   uint32_t tmem_slot;
   int abort_flag;
@@ -397,10 +401,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   constexpr int O_COL0 = NQ * S_COLS;                 // O accumulators follow the score buffers
   constexpr int NCH = TKV / 32;                       // 32-column chunks of one score row
   constexpr int kPoly = (D == 128) ? ATTN_POLY_PAIRS_D128 : ATTN_POLY_PAIRS_D64;   // polynomial pairs per 8
-  constexpr int TMEM_COLS = (NQ * (S_COLS + D) <= 32) ? 32
-                          : (NQ * (S_COLS + D) <= 64) ? 64
-                          : (NQ * (S_COLS + D) <= 128) ? 128
-                          : (NQ * (S_COLS + D) <= 256) ? 256 : 512;
+  // d = 64 leaves tensor memory for P next to S and O.  The score buffer is then free as soon as the softmax
+  // warpgroup has read it into registers, and the next step's Q K^T runs during this step's exponentials instead
+  // of after this step's P V.  (d = 128 fills tensor memory: P overwrites the front of the score buffer.)
+  constexpr bool kSplitP = (D == 64) && NQ == 2 && (NQ * (S_COLS + D) + NQ * (TKV / 2) <= 512);
+  constexpr int P_COL0 = NQ * (S_COLS + D);           // kSplitP: bf16 P, TKV / 2 columns per sub-tile
+  constexpr int kTmemUsed = NQ * (S_COLS + D) + (kSplitP ? NQ * (TKV / 2) : 0);
+  constexpr int TMEM_COLS = (kTmemUsed <= 32) ? 32 : (kTmemUsed <= 64) ? 64 : (kTmemUsed <= 128) ? 128
+                          : (kTmemUsed <= 256) ? 256 : 512;
   using SM = FwdSmem<D, TKV, NQ>;
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -443,6 +451,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(smem_u32(&misc->alpha_full[i]), kSub);
       mbar_init(smem_u32(&misc->dbg_bar[i]), 1);
       mbar_init(smem_u32(&misc->o_free[i]), kSub);
+      mbar_init(smem_u32(&misc->s_free[i]), kSub);
     }
     mbar_init(smem_u32(&misc->q_empty), 1);
     fence_mbar_init();
@@ -471,6 +480,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t s_tmem = lane_base + i * S_COLS;
+    const uint32_t p_tmem = kSplitP ? lane_base + P_COL0 + i * (TKV / 2) : s_tmem;   // else P aliases the front of S
     const uint32_t o_tmem = lane_base + O_COL0 + i * D;
     const uint32_t bar_s = smem_u32(&misc->s_full[i]);
     const uint32_t bar_p = smem_u32(&misc->p_full[i]);
@@ -490,6 +500,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
       float m_run = -INFINITY, delta = 0.f;
+      const uint32_t g_seg0 = g;                         // first step of this segment
+      (void)g_seg0;
       // One KV step of this sub-tile.  The masked variant (a ragged last KV tile, or a causal step that
       // reaches past the sub-tile's first row) is compiled separately so that the common step pays
       // nothing for it; `lim` is the last key column of this step the thread's row may attend to.
@@ -519,6 +531,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
         for (int c = NCH / 2; c < NCH; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
         if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 1);
+        if constexpr (kSplitP) {
+          tc_fence_before();
+          mbar_arrive(smem_u32(&misc->s_free[i]));         // the scores are in registers: the buffer may be overwritten
+        }
         if constexpr (kMasked) {
 #pragma unroll
           for (int k = TKV / 2; k < TKV; ++k)
@@ -549,11 +565,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint64_t neg_m2 = pack_f32x2(-m_new, -m_new);
         uint64_t sum_a = 0ull, sum_b = 0ull;               // packed (0.f, 0.f)
         uint32_t pk[16];
+        if constexpr (kSplitP) {
+          // P has its own columns: the previous step's P V must have read them (it finished long ago as a rule)
+          if (g != g_seg0) {
+            if (!wait_bar_warp(smem_u32(&misc->o_full[i]), (g - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, 0x4000 | g))) return false;
+            tc_fence_after();
+          }
+        }
         // first half of the row: the second product may start on it while the rest is computed
 #pragma unroll
         for (int c = 0; c < NCH / 2; ++c) {
           exp_chunk<kPoly>(&s[c * 32], ek, neg_m2, sum_a, pk);
-          tmem_st16(s_tmem + c * 16, pk);                  // P aliases the front of the S buffer
+          tmem_st16(p_tmem + c * 16, pk);
         }
         uint32_t pk2[16];
         exp_chunk<kPoly>(&s[(NCH / 2) * 32], ek, neg_m2, sum_b, pk2);
@@ -562,11 +585,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tc_fence_before();
         mbar_arrive(bar_p);
         if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 4);
-        tmem_st16(s_tmem + (NCH / 2) * 16, pk2);
+        tmem_st16(p_tmem + (NCH / 2) * 16, pk2);
 #pragma unroll
         for (int c = NCH / 2 + 1; c < NCH; ++c) {
           exp_chunk<kPoly>(&s[c * 32], ek, neg_m2, sum_b, pk);
-          tmem_st16(s_tmem + c * 16, pk);
+          tmem_st16(p_tmem + c * 16, pk);
         }
         float sa0, sa1, sb0, sb1;
         unpack_f32x2(sum_a, sa0, sa1);
@@ -942,7 +965,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!ok) break;
         tc_fence_after();
       }
-      if (elect_one()) {
+      const int k0_stage = stage;
+      // kSplitP: nothing ties the two sub-tiles to each other any more, so the half-step offset between their
+      // softmax warpgroups (one computes exponentials while the other loads, reduces and stores) is set up here:
+      // sub-tile 1's first scores are produced only after the first half of sub-tile 0's first P (short segments
+      // start both at once; holding K_0 that long while K_1 is awaited needs a third ring stage).
+      const bool defer_q1 = kSplitP && n >= 4 && p.stages >= 3;
+      if (!defer_q1 && elect_one()) {
         if (NQ == 2) {
           issue_qk<D, TKV>(tmem_base + S_COLS, q_smem + kSub * D * 2, ring_smem + stage * SM::kStageBytes);
           umma_commit(smem_u32(&misc->s_full[1]));
@@ -962,6 +991,62 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (more) advance();
         const uint32_t v_smem = ring_smem + v_stage * SM::kStageBytes;
         const uint32_t k_smem = ring_smem + k_stage * SM::kStageBytes;
+        if constexpr (kSplitP) {
+          // Products are issued in the order in which their operands become ready when sub-tile 1 runs half a
+          // step behind sub-tile 0.
+          const uint32_t p0 = tmem_base + P_COL0, p1 = p0 + TKV / 2, o0 = tmem_base + O_COL0, o1 = o0 + D;
+          const uint32_t q1_smem = q_smem + kSub * D * 2;
+          auto W = [&](uint64_t* bar, uint32_t par, uint32_t tag) -> bool {
+            if (!wait_bar_warp(smem_u32(bar), par, abort_flag, wait_info(kRoleMma, kBarPFull, tag))) { ok = false; return false; }
+            tc_fence_after();
+            return true;
+          };
+          if (more) {                                                        // A0: scores of sub-tile 0, next step
+            if (!W(&misc->s_free[0], g & 1, 0x100) || !W(&misc->kv_full[k_stage], k_phase, 0x101)) break;
+            if (elect_one()) { issue_qk<D, TKV>(tmem_base, q_smem, k_smem); umma_commit(smem_u32(&misc->s_full[0])); }
+            __syncwarp();
+          }
+          if (!W(&misc->kv_full[v_stage], v_phase, 0x102) || !W(&misc->p_full[0], g & 1, 0x103)) break;
+          if (jj == 0 && seg > 0 && !W(&misc->o_free[0], (seg - 1) & 1, 0x104)) break;
+          if (elect_one()) issue_pv<D, TKV>(o0, p0, v_smem, jj > 0, TKV * 128, 1024, 0, TKV / 32);   // B0a
+          __syncwarp();
+          if (jj == 0 && defer_q1) {                                         // first scores of sub-tile 1
+            if (elect_one()) {
+              issue_qk<D, TKV>(tmem_base + S_COLS, q1_smem, ring_smem + k0_stage * SM::kStageBytes);
+              umma_commit(smem_u32(&misc->s_full[1]));
+              umma_commit(smem_u32(&misc->kv_empty[k0_stage]));
+            }
+            __syncwarp();
+          }
+          if (more) {                                                        // A1
+            if (!W(&misc->s_free[1], g & 1, 0x105)) break;
+            if (elect_one()) {
+              issue_qk<D, TKV>(tmem_base + S_COLS, q1_smem, k_smem);
+              umma_commit(smem_u32(&misc->s_full[1]));
+              umma_commit(smem_u32(&misc->kv_empty[k_stage]));
+              if (jj + 2 == n) umma_commit(smem_u32(&misc->q_empty));
+            }
+            __syncwarp();
+          }
+          if (!W(&misc->p_half[0], g & 1, 0x106)) break;                     // B0b
+          if (elect_one()) {
+            issue_pv<D, TKV>(o0, p0, v_smem, true, TKV * 128, 1024, TKV / 32, TKV / 16);
+            umma_commit(smem_u32(&misc->o_full[0]));
+          }
+          __syncwarp();
+          if (!W(&misc->p_full[1], g & 1, 0x107)) break;                     // B1a
+          if (jj == 0 && seg > 0 && !W(&misc->o_free[1], (seg - 1) & 1, 0x108)) break;
+          if (elect_one()) issue_pv<D, TKV>(o1, p1, v_smem, jj > 0, TKV * 128, 1024, 0, TKV / 32);
+          __syncwarp();
+          if (!W(&misc->p_half[1], g & 1, 0x109)) break;                     // B1b
+          if (elect_one()) {
+            issue_pv<D, TKV>(o1, p1, v_smem, true, TKV * 128, 1024, TKV / 32, TKV / 16);
+            umma_commit(smem_u32(&misc->o_full[1]));
+            umma_commit(smem_u32(&misc->kv_empty[v_stage]));
+          }
+          __syncwarp();
+          continue;
+        }
         if (!wait_bar_warp(smem_u32(&misc->kv_full[v_stage]), v_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, g))) { ok = false; break; }
 #pragma unroll
         for (int i = 0; i < NQ; ++i) {
