@@ -145,7 +145,7 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   if (grid < 1 || (long long)grid > total_units) return ATTN_ERR_BAD_TILES;
   if (ws && (size_t)grid * NQ * 8 > attn::kCounterBytes / sizeof(unsigned int)) return ATTN_ERR_BAD_TILES;
   const int smem = SM::total(t.kv_stages);
-  // uniform key split (k CTAs per tile, all parts of a tile finish together): the eager-publish instantiation
+  // uniform key split (k CTAs per tile, all parts of a tile finish together): the instantiation with fixed merge roles
   const bool eager = !p.causal && t.ctas > t.tiles && t.ctas % t.tiles == 0;
   auto launch = [&](auto kern) -> int {
     ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));

@@ -676,10 +676,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       } else {
         // Part of a Q tile shared with other CTAs (those whose ranges meet the tile's units; the first of
-        // them owns the tile's counters).  Per warp: counter A orders the CTAs by when they finished their
-        // key range; all but the last publish their un-normalised partial (O, m, delta) -- slots 2*cta and
+        // them owns the tile's counters).  Per warp: one of the tile's CTAs merges (see "Who merges" below:
+        // counter A orders the CTAs by when they finished their key range); all but that one publish their un-normalised partial (O, m, delta) -- slots 2*cta and
         // 2*cta+1: a CTA has at most two partial pieces, its first and its last segment -- and signal that on
-        // counter B without waiting; the last one keeps its part in tensor memory, waits for B and merges
+        // counter B without waiting; the merging one keeps its part in tensor memory, waits for B and merges
         // all parts in ascending key order (the merge operator of the online softmax), so the result does
         // not depend on who merges.
         const int c_first = cta_of_unit(sg.unit0, T, G);
@@ -705,18 +705,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           ws[(size_t)kSub * D + row] = m_run;
           ws[(size_t)kSub * D + kSub + row] = delta;
         };
-        uint32_t order = 0;
-        if (lane == 0) order = atomicAdd(&ctr[0], 1u);
-        // When all parts of a tile finish together (a uniform key split: the EAGER instantiation), the partial
-        // is written while that answer is on its way -- the last finisher then writes it in vain, but nobody
-        // waits for a publisher that has not even started.  With staggered finishes (balanced ranges) only the
-        // publishers write.
-        // EAGER instantiation: the partial is written while the answer is on its way.
-        if constexpr (EAGER) write_partial();
-        order = __shfl_sync(0xffffffffu, order, 0);
+        // Who merges.  Balanced ranges: the parts of a tile finish at different times, so the last finisher
+        // (by counter A) merges and nobody waits for a part that has not started.  Uniform key split (the EAGER
+        // instantiation): all parts finish together, so the roles are fixed in advance -- the tile's 32-row
+        // groups are dealt out to the parts in turn; a warp publishes its rows unless its own part owns them.
+        // Every CTA then writes and reads only its share, all parts merge in parallel, and nobody waits for
+        // the answer of an atomic.
+        bool merges;
+        if constexpr (EAGER) {
+          const int rg = i * 4 + wq;
+          merges = (mine == (parts <= NQ * 4 ? rg % parts : rg));
+        } else {
+          uint32_t order = 0;
+          if (lane == 0) order = atomicAdd(&ctr[0], 1u);
+          order = __shfl_sync(0xffffffffu, order, 0);
+          merges = (order == (uint32_t)(parts - 1));
+        }
         if (warp == 0) ATTN_TRACE_MARK(5);
-        if (order != (uint32_t)(parts - 1)) {
-          if constexpr (!EAGER) write_partial();
+        if (!merges) {
+          write_partial();
           tc_fence_before();
           mbar_arrive(smem_u32(&misc->o_free[i]));           // O may be overwritten by the next segment
           __threadfence();
