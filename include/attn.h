@@ -265,6 +265,11 @@ int attn_last_device_status(void *cuda_stream, uint32_t *detail);
 /* Number of kernels the last attn_forward* call on this thread launched. */
 int attn_last_launch_count(void);
 
+/* CTAs per thread-block cluster of the last fused launch on this thread: k if the plan was a
+ * uniform key split of k CTAs per Q tile and those were launched as one cluster each (their
+ * partial results then travel through distributed shared memory), 0 otherwise. */
+int attn_last_cluster_size(void);
+
 /* Static description of a status code; never NULL. */
 const char *attn_status_string(int status);
 

@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "attn_hw_desc_b200", "attn_hw_desc_query", "attn_plan", "attn_plan_ex", "attn_workspace_bytes",
     "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_static_scratch", "attn_forward_desc",
     "attn_last_device_status",
-    "attn_last_launch_count", "attn_status_string", "attn_last_cuda_error",
+    "attn_last_launch_count", "attn_last_cluster_size", "attn_status_string", "attn_last_cuda_error",
     "gemm_plan", "gemm_forward", "softmax_rows_forward", "attn_forward_unfused",
 )
 
@@ -94,6 +94,7 @@ def lib() -> ctypes.CDLL:
         L.attn_forward_desc.argtypes = [ctypes.POINTER(AttnHwDesc), vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.attn_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.attn_last_launch_count.argtypes = []
+        L.attn_last_cluster_size.argtypes = []
         L.attn_status_string.argtypes = [i32]
         L.attn_status_string.restype = ctypes.c_char_p
         L.attn_last_cuda_error.argtypes = []
@@ -311,6 +312,11 @@ def last_device_status(device=None):
 
 def last_launch_count() -> int:
     return int(lib().attn_last_launch_count())
+
+
+def last_cluster_size() -> int:
+    """CTAs per thread-block cluster of the last fused launch (0: launched without clusters)."""
+    return int(lib().attn_last_cluster_size())
 
 
 # ----------------------------------------------------------------- unfused path

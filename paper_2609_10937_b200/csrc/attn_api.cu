@@ -20,6 +20,7 @@ namespace {
 
 thread_local char t_cuda_error[256] = "";
 thread_local int t_launch_count = 0;
+thread_local int t_cluster_size = 0;   // CTAs per thread-block cluster of the last fused launch (0: no clusters)
 
 int cuda_fail(cudaError_t e, const char* what) {
   std::snprintf(t_cuda_error, sizeof t_cuda_error, "%s: %s", what, cudaGetErrorString(e));
@@ -152,8 +153,58 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
     kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
     return ATTN_OK;
   };
+  // Uniform key split with few parts: the k CTAs of a tile are launched as one thread-block cluster and exchange
+  // their partial results through distributed shared memory (landing areas in the K/V ring: the groups of rows one
+  // CTA merges, times the k-1 parts it receives for each, must fit).  Used only if all clusters can be resident at
+  // once, like the CTAs of the plain launch; otherwise, or if the cluster launch is not possible, the partials go
+  // through the workspace.
+  p.cluster_k = 0;
+  t_cluster_size = 0;
+  auto launch_eager = [&](auto kern, auto kern_cluster) -> int {
+    ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+#ifndef ATTN_NO_CLUSTER
+    ATTN_CUDA_TRY(cudaFuncSetAttribute(kern_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    const int kk = t.ctas / t.tiles;
+    const size_t landing = (size_t)((4 * NQ + kk - 1) / kk) * (kk - 1) * (32 * D * 4 + 256);
+    if (kk >= 2 && kk <= 8 && landing <= (size_t)t.kv_stages * SM::kStageBytes) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(grid);
+      cfg.blockDim = dim3(512);
+      cfg.dynamicSmemBytes = smem;
+      cfg.stream = stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = kk;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      static int resident[9][kMaxDevices] = {};          // clusters of kk CTAs that fit at once (+1; 0 = not asked yet)
+      int dev = 0;
+      ATTN_CUDA_TRY(cudaGetDevice(&dev));
+      if (dev >= 0 && dev < kMaxDevices) {
+        if (resident[kk][dev] == 0) {
+          int n = 0;
+          if (cudaOccupancyMaxActiveClusters(&n, kern_cluster, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+          resident[kk][dev] = n + 1;
+        }
+        if ((long long)(resident[kk][dev] - 1) * kk >= grid) {
+          attn::FwdParams pc = p;
+          pc.cluster_k = kk;
+          if (cudaLaunchKernelEx(&cfg, kern_cluster, tq, tk, tv, to, pc) == cudaSuccess) {
+            t_cluster_size = kk;
+            return ATTN_OK;
+          }
+          (void)cudaGetLastError();                       // fall through to the plain launch
+        }
+      }
+    }
+#endif
+    kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
+    return ATTN_OK;
+  };
   if (p.causal) rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, true, false>);
-  else if (eager) rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, false, true>);
+  else if (eager) rc = launch_eager(attn::attn_fwd_kernel<D, TKV, NQ, false, true>, attn::attn_fwd_kernel<D, TKV, NQ, false, true, true>);
   else rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, false, false>);
   if (rc != ATTN_OK) return rc;
   ATTN_CUDA_TRY(cudaGetLastError());
@@ -446,6 +497,7 @@ extern "C" int attn_debug_read_cta_times(unsigned long long* out, int n) {
 #endif
 
 extern "C" int attn_last_launch_count(void) { return t_launch_count; }
+extern "C" int attn_last_cluster_size(void) { return t_cluster_size; }
 
 extern "C" const char* attn_last_cuda_error(void) { return t_cuda_error; }
 

@@ -16,7 +16,10 @@
 //                          CTAs walk equal ranges of the (Q tile, KV step) line.  Where
 //                          several CTAs share a Q tile, all but the last to finish publish
 //                          their partial (O, m, delta) and the last one merges them, per
-//                          warp, with the merge operator of the online softmax.
+//                          warp, with the merge operator of the online softmax.  Under a
+//                          uniform key split the CTAs of a tile can run as one thread-block
+//                          cluster: the partials then go from tensor memory straight into the
+//                          merging CTA's shared memory (st.async), not through L2.
 //   attn_fwd_simple_kernel the same algorithm with nothing overlapped; used to
 //                          cross-check the pipelined kernel and the layouts.
 //
@@ -172,6 +175,7 @@ struct FwdParams {
   __nv_bfloat16* o;        // output, written directly when a result cannot go through the Q buffer
   float* ws;               // partial results of Q tiles shared by several CTAs
   unsigned int* counters;  // arrival counters of shared Q tiles; zero between launches
+  int cluster_k;           // > 1: the k CTAs of a Q tile are one thread-block cluster (uniform key split only)
 };
 
 // Work decomposition.  A work unit is one KV step of one Q tile.  Q tile q of a head needs
@@ -287,6 +291,8 @@ struct FwdMisc {               // lives in the last 3072 bytes of dynamic shared
   uint64_t q_empty;            // every product that reads the Q tile of a segment has finished
   uint64_t o_free[2];          // the epilogue of a segment has read its O accumulator
   uint64_t s_free[2];          // d = 64: the softmax warpgroup holds the step's scores in registers
+  uint64_t peers_ready;        // cluster: every other CTA of the tile has finished with its K/V ring
+  uint64_t data_ready[8][2];   // cluster: the other CTAs' parts of softmax warp w's rows have landed ([1]: columns 64..)
   uint64_t dbg_bar[2];         // trace builds only: completion of the first half of P V
   uint32_t tmem_slot;
   int abort_flag;
@@ -389,7 +395,7 @@ __device__ __forceinline__ void stage_row_chunk(uint32_t stage_out, int c, int r
   }
 }
 
-template <int D, int TKV, int NQ, bool CAUSAL, bool EAGER>
+template <int D, int TKV, int NQ, bool CAUSAL, bool EAGER, bool CLUSTER = false>
 __global__ void __launch_bounds__(512, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -406,6 +412,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // of after this step's P V.  (d = 128 fills tensor memory: P overwrites the front of the score buffer.)
   constexpr bool kSplitP = (D == 64) && NQ == 2 && (NQ * (S_COLS + D) + NQ * (TKV / 2) <= 512);
   constexpr int P_COL0 = NQ * (S_COLS + D);           // kSplitP: bf16 P, TKV / 2 columns per sub-tile
+  constexpr uint32_t kPartBytes = 32 * D * 4 + 256;   // cluster: one warp's part -- O of 32 rows, then m and delta
   constexpr int kTmemUsed = NQ * (S_COLS + D) + (kSplitP ? NQ * (TKV / 2) : 0);
   constexpr int TMEM_COLS = (kTmemUsed <= 32) ? 32 : (kTmemUsed <= 64) ? 64 : (kTmemUsed <= 128) ? 128
                           : (kTmemUsed <= 256) ? 256 : 512;
@@ -454,6 +461,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(smem_u32(&misc->s_free[i]), kSub);
     }
     mbar_init(smem_u32(&misc->q_empty), 1);
+    if constexpr (CLUSTER) {
+      {
+        // Partials travel through distributed shared memory (see the end of a segment).  The merging warps of
+        // this CTA -- warp w merges if w mod k is this CTA's rank -- expect the parts of the k-1 other CTAs.
+        mbar_init(smem_u32(&misc->peers_ready), p.cluster_k - 1);
+        for (int w = 0; w < 4 * NQ; ++w) {
+          mbar_init(smem_u32(&misc->data_ready[w][0]), 1);
+          mbar_init(smem_u32(&misc->data_ready[w][1]), 1);
+          if (w % p.cluster_k == cta % p.cluster_k) {
+            // first the statistics and columns 0..63 of every part, then (d = 128) columns 64..127
+            mbar_arrive_expect_tx(smem_u32(&misc->data_ready[w][0]), (uint32_t)(p.cluster_k - 1) * (32 * 64 * 4 + 256));
+            if (KCH == 2) mbar_arrive_expect_tx(smem_u32(&misc->data_ready[w][1]), (uint32_t)(p.cluster_k - 1) * (32 * 64 * 4));
+          }
+        }
+      }
+    }
     fence_mbar_init();
     prefetch_tmap(&tm_q);
     prefetch_tmap(&tm_k);
@@ -467,6 +490,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // every CTA's barriers must exist before a peer touches them: arrive here, wait where the first peer access is
+  bool cluster_waited = false;                           // this thread has completed the wait of that barrier
+  (void)cluster_waited;
+  if constexpr (CLUSTER) cluster_arrive();
   const uint32_t tmem_base = misc->tmem_slot;
   const bool run = (*abort_flag == 0) && u_hi > u_lo;
   if (threadIdx.x == 0) ATTN_TRACE_MARK(1);
@@ -621,6 +648,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // ----------------------------------------------------- end of segment
       // Each warp finishes its own 32 rows without meeting the other warps of its warpgroup.
       if (warp == 0) ATTN_TRACE_MARK(3);
+      if constexpr (CLUSTER) {
+        // The peers' barriers exist (arrival at kernel start).  Two parts: what a CTA receives lands in its Q
+        // buffer, which is dead one step before the end -- its peers may be told so right away.
+        if (ok) {
+          cluster_wait();
+          cluster_waited = true;
+          if (p.cluster_k == 2 && warp == 0) {
+            ok = wait_bar_warp(smem_u32(&misc->q_empty), 0, abort_flag, wait_info(kRoleSoftmax, kBarQ, 0x2000));
+            if (ok && lane < 2 && lane != (cta & 1)) mbar_arrive_peer(map_to_cta(smem_u32(&misc->peers_ready), lane));
+          }
+        }
+      }
       if (ok) ok = wait_bar_warp(smem_u32(&misc->o_full[i]), (g - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, g));
       if (!ok) break;
       tc_fence_after();
@@ -682,6 +721,117 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // counter B without waiting; the merging one keeps its part in tensor memory, waits for B and merges
         // all parts in ascending key order (the merge operator of the online softmax), so the result does
         // not depend on who merges.
+        if constexpr (CLUSTER) {
+          {
+            const int mine = cta % p.cluster_k;
+            // Uniform key split with the tile's k CTAs as one thread-block cluster (rank = `mine`): the parts go
+            // from tensor memory straight into the merging CTA's shared memory -- no trip through L2, no flag
+            // in global memory.  Roles as below ("Who merges"): softmax warp w belongs to rank w mod k.  The
+            // landing areas lie in the K/V ring, which is dead in a CTA once the last product of both its
+            // sub-tiles has finished; every CTA tells its peers when that is so.
+            const int k = p.cluster_k;
+            const int owner = warp % k, ms = warp / k;
+            // Two parts: what a CTA receives fits its Q buffer (O) and the idle staging chunks of its publishing
+            // warps (m, delta), and the Q buffer is dead one step before the end.  More parts: the K/V ring,
+            // dead once the last product of the other sub-tile has finished too.
+            const bool q_land = (k == 2);
+            if (!q_land) {
+              if (NQ == 2 &&
+                  !wait_bar_warp(smem_u32(&misc->o_full[1 - i]), (g - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, 0x2000 | g))) { ok = false; break; }
+              if (warp == 0 && lane < k && lane != mine) mbar_arrive_peer(map_to_cta(smem_u32(&misc->peers_ready), lane));
+            }
+            if (warp == 0) ATTN_TRACE_MARK(5);
+            // landing area of part `src` (index among the k-1 other parts) of this warp's rows, as local addresses
+            auto o_land = [&](int src) -> uint32_t {
+              return q_land ? q_smem + (uint32_t)ms * (32 * D * 4) : ring_smem + (uint32_t)(ms * (k - 1) + src) * kPartBytes;
+            };
+            auto s_land = [&](int src) -> uint32_t {
+              return q_land ? out_smem + (uint32_t)(warp ^ 1) * 4096 : o_land(src) + 32 * D * 4;
+            };
+            if (owner != mine) {
+              if (!wait_bar_warp(smem_u32(&misc->peers_ready), 0, abort_flag, wait_info(kRoleSoftmax, kBarSync, 0x6000 | (uint32_t)warp))) { ok = false; break; }
+              const int src = mine < owner ? mine : mine - 1;
+              const uint32_t land = map_to_cta(o_land(src), owner), sland = map_to_cta(s_land(src), owner);
+              const uint32_t rbar0 = map_to_cta(smem_u32(&misc->data_ready[warp][0]), owner);
+              st_peer_f1(sland + lane * 4, m_run, rbar0);
+              st_peer_f1(sland + 128 + lane * 4, delta, rbar0);
+#pragma unroll 1
+              for (int hcol = 0; hcol < D / 64; ++hcol) {
+                const uint32_t rbar = rbar0 + hcol * 8;
+                uint32_t r[64];
+                tmem_ld32_nowait(o_tmem + hcol * 64, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+                tmem_ld32_nowait(o_tmem + hcol * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+                tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+                tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+#pragma unroll
+                for (int gq = 0; gq < 16; ++gq)
+                  st_peer_f4(land + (uint32_t)((hcol * 16 + gq) * 32 + lane) * 16, __uint_as_float(r[gq * 4]),
+                             __uint_as_float(r[gq * 4 + 1]), __uint_as_float(r[gq * 4 + 2]), __uint_as_float(r[gq * 4 + 3]), rbar);
+              }
+              tc_fence_before();
+              mbar_arrive(smem_u32(&misc->o_free[i]));
+            } else {
+              if (!wait_bar_warp(smem_u32(&misc->data_ready[warp][0]), 0, abort_flag, wait_info(kRoleSoftmax, kBarSync, 0x5000 | (uint32_t)warp))) { ok = false; break; }
+              if (warp == 0) ATTN_TRACE_MARK(6);
+              // part q (ascending key order) of this warp's rows: own part in tensor memory, the others landed
+              auto part = [&](int q) -> const float* {           // O of part q: [column / 4][lane] float4
+                return reinterpret_cast<const float*>(smem_raw + (o_land(q < mine ? q : q - 1) - smem_base));
+              };
+              auto stat = [&](int q) -> const float* {           // m[32], delta[32] of part q
+                return reinterpret_cast<const float*>(smem_raw + (s_land(q < mine ? q : q - 1) - smem_base));
+              };
+              float m_all = m_run;
+              for (int q = 0; q < k; ++q)
+                if (q != mine) m_all = fmaxf(m_all, stat(q)[lane]);
+              float d_all = 0.f;
+              for (int q = 0; q < k; ++q) {
+                const float m_q = (q == mine) ? m_run : stat(q)[lane];
+                const float d_q = (q == mine) ? delta : stat(q)[32 + lane];
+                d_all += d_q * exp2f(m_q - m_all);
+              }
+              const float inv = 1.0f / d_all;
+#pragma unroll 1
+              for (int h = 0; h < KCH; ++h) {
+                if (h == 1 &&
+                    !wait_bar_warp(smem_u32(&misc->data_ready[warp][1]), 0, abort_flag, wait_info(kRoleSoftmax, kBarSync, 0x5800 | (uint32_t)warp))) { ok = false; break; }
+                float val[64];
+#pragma unroll
+                for (int e = 0; e < 64; ++e) val[e] = 0.f;
+                for (int q = 0; q < k; ++q) {
+                  if (q == mine) {
+                    const float w = exp2f(m_run - m_all);
+                    uint32_t r[64];
+                    tmem_ld32_nowait(o_tmem + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+                    tmem_ld32_nowait(o_tmem + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+                    tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+                    tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+#pragma unroll
+                    for (int e = 0; e < 64; ++e) val[e] += w * __uint_as_float(r[e]);
+                  } else {
+                    const float* b = part(q);
+                    const float w = exp2f(stat(q)[lane] - m_all);
+#pragma unroll
+                    for (int gq = 0; gq < 16; ++gq) {
+                      const float4 v4 = reinterpret_cast<const float4*>(b)[(h * 16 + gq) * 32 + lane];
+                      val[gq * 4 + 0] += w * v4.x;
+                      val[gq * 4 + 1] += w * v4.y;
+                      val[gq * 4 + 2] += w * v4.z;
+                      val[gq * 4 + 3] += w * v4.w;
+                    }
+                  }
+                }
+                if (h == KCH - 1) {
+                  tc_fence_before();
+                  mbar_arrive(smem_u32(&misc->o_free[i]));
+                }
+#pragma unroll
+                for (int e = 0; e < 64; ++e) val[e] *= inv;
+                store_half(h, *reinterpret_cast<float(*)[32]>(&val[0]), *reinterpret_cast<float(*)[32]>(&val[32]));
+              }
+              if (!ok) break;
+            }
+          }
+        } else {
         const int c_first = cta_of_unit(sg.unit0, T, G);
         const int c_last = cta_of_unit(sg.unit0 + sg.steps_t - 1, T, G);
         const int parts = c_last - c_first + 1, mine = cta - c_first;
@@ -884,6 +1034,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             store_half(h, *reinterpret_cast<float(*)[32]>(&val[0]), *reinterpret_cast<float(*)[32]>(&val[32]));
           }
           }
+        }
         }
       }
       }
@@ -1172,6 +1323,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   if (warp == 0) ATTN_TRACE_MARK(7);
   tc_fence_before();
   __syncthreads();
+  if constexpr (CLUSTER) {
+    if (!cluster_waited) cluster_wait();                 // (the softmax warps waited at the end of their segment)
+    cluster_arrive();                                    // no CTA leaves while a peer may still write to it
+    cluster_wait();
+  }
   if (warp == 15) {
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);

@@ -232,6 +232,32 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
                : "memory");
 }
 
+// -------------------------------------------- thread-block clusters: barrier, peer addresses, peer stores
+// (relaxed: what a peer must see before it passes the barrier -- the mbarrier initialisations -- is released by
+// fence.mbarrier_init.release.cluster)
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// Address of the same shared-memory location in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+// One arrival on an mbarrier of another CTA of the cluster (release at cluster scope).
+__device__ __forceinline__ void mbar_arrive_peer(uint32_t peer_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(peer_bar) : "memory");
+}
+// Asynchronous stores into another CTA's shared memory; the bytes are counted on that CTA's mbarrier
+// (complete_tx), whose waiter then sees the data -- the same contract as a bulk copy.
+__device__ __forceinline__ void st_peer_f4(uint32_t peer_addr, float a, float b, float c, float d, uint32_t peer_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(peer_addr), "f"(a), "f"(b), "f"(c), "f"(d), "r"(peer_bar) : "memory");
+}
+__device__ __forceinline__ void st_peer_f1(uint32_t peer_addr, float a, uint32_t peer_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];"
+               ::"r"(peer_addr), "f"(a), "r"(peer_bar) : "memory");
+}
+
 // -------------------------------------------- per-thread asynchronous 16-byte copies (L2 -> shared)
 __device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");

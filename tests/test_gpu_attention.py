@@ -120,6 +120,38 @@ def test_pipelined_kernel_matches_oracle_small(env, B, H, L, d):
     _run_and_compare(env, _case("small", B, H, L, d), binding.forward)
 
 
+@pytest.mark.parametrize("d,n_q,kv_splits,L,cluster", [
+    (128, 2, 2, 2100, 2),     # two parts: landing in the Q buffer, ready one step before the end; ragged L
+    (128, 2, 3, 1408, 3),     # three and four parts: landing in the K/V ring
+    (128, 2, 4, 2048, 4),
+    (128, 2, 5, 2560, 0),     # five parts of a two-sub-tile CTA do not fit the ring: through the workspace
+    (64, 2, 2, 1408, 2), (64, 2, 3, 1500, 3), (64, 2, 4, 2048, 4),
+    (128, 1, 2, 1408, 2), (128, 1, 4, 1408, 4), (64, 1, 3, 777, 3)])
+def test_uniform_split_through_clusters(env, d, n_q, kv_splits, L, cluster):
+    """Uniform key splits: the CTAs of a Q tile run as one thread-block cluster and exchange their partial results
+    through distributed shared memory where the landing areas fit; the result is the oracle's either way, the
+    same bits run to run, and the same bits as with one CTA per tile merged nowhere (up to the merge's rounding)."""
+    torch, _, binding = env
+    case = _case("cluster", 1, 3, L, d, sigma_qk=math.sqrt(3.0))
+    seen = []
+
+    def run(a, b, c):
+        o = binding.forward_tiles(a, b, c, n_q=n_q, kv_splits=kv_splits)
+        seen.append(binding.last_cluster_size())
+        return o
+
+    _run_and_compare(env, case, run)
+    assert seen == [cluster]
+    q, k, v = (to_cuda_bf16(x) for x in synth.make_qkv(case, seed=0))
+    o1 = binding.forward_tiles(q, k, v, n_q=n_q, kv_splits=kv_splits)
+    o2 = binding.forward_tiles(q, k, v, n_q=n_q, kv_splits=kv_splits)
+    whole = binding.forward_tiles(q, k, v, n_q=n_q, kv_splits=1)
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))
+    assert float((o1.float() - whole.float()).abs().max()) <= 2e-2
+
+
 @pytest.mark.parametrize("n_q,tile_kv,kv_stages,kv_splits", [
     (2, 128, 0, 1), (2, 128, 2, 1), (2, 128, 3, 3), (2, 64, 0, 1), (2, 64, 4, 5),
     (1, 128, 0, 1), (1, 64, 0, 2), (1, 128, 3, 7)])
