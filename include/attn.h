@@ -83,6 +83,8 @@ typedef struct attn_hw_desc {
   int32_t atom_n_max;          /* largest N of one instruction (256 | 16)             */
   int32_t elem_bytes;          /* operand element size (2 = bf16, 4 = fp32)           */
   int32_t cache_bytes;         /* last-level cache shared by all units (L2); 0 if not modelled */
+  int32_t max_clusters[8];     /* [k-1]: clusters of k CTAs (one CTA per unit, distributed shared    */
+                               /* memory between them) that can be resident at once; 0: none        */
   double hbm_gbps;             /* sustained HBM bandwidth, GB/s                       */
   double peak_tflops;          /* dense tensor peak for the operand type, TFLOP/s     */
   double sm_clock_mhz;         /* maximum SM clock                                    */

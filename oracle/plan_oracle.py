@@ -67,6 +67,12 @@ _MIN_STEPS_PER_SPLIT = 4
 _SEGMENT_OVERHEAD_STEPS = 3
 _CTA_OVERHEAD_STEPS = 2     # start and end of a CTA that handles one whole Q tile
 _TRANSITION_STEPS = 1       # a persistent CTA moving on to its next Q tile
+# fewer Q tiles than units: cost of the end of a CTA's work, in KV steps
+_MIN_STEPS_PER_CLUSTER_SPLIT = 2
+_CLUSTER_OVERHEAD_STEPS = 5      # k CTAs per tile as one cluster (partials through distributed shared memory)
+_WORKSPACE_OVERHEAD_STEPS = 8    # k CTAs per tile, partials through the workspace (plus k // 2)
+_BALANCED_OVERHEAD_STEPS = 12    # equal ranges of the unit line
+_LANDING_PART_EXTRA = 256        # m and delta of the 32 rows of one part
 
 
 def causal_head_units(q_tiles: int, steps: int, ratio: int) -> int:
@@ -119,15 +125,32 @@ def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal
         total = B * H * causal_head_units(-(-L // tile_q), steps, tile_q // tile_kv)
         ctas = max(1, min(total // _MIN_STEPS_PER_SPLIT, desc["num_units"]))
     elif under:
-        k = max(1, min(desc["num_units"] // tiles, steps // _MIN_STEPS_PER_SPLIT))
-        cost_uniform = -(-steps // k) + _SEGMENT_OVERHEAD_STEPS
+        # one CTA per tile; k CTAs per tile as one cluster; k CTAs per tile through the workspace; equal ranges.
+        # The cheapest wins, ties go to the earlier candidate.
+        units = desc["num_units"]
         total = tiles * steps
-        g = min(total // _MIN_STEPS_PER_SPLIT, desc["num_units"])
-        ctas = tiles * k
-        if g > tiles * k:
-            cost_balanced = -(-total // g) + 2 * _SEGMENT_OVERHEAD_STEPS
-            if cost_balanced < cost_uniform:
-                ctas = g
+        best = steps + _CTA_OVERHEAD_STEPS
+        clusters = list(desc.get("max_clusters", [0] * 8))
+        groups = 4 * n_q
+        part = 32 * 4 * d + _LANDING_PART_EXTRA
+        for k in range(2, 9):
+            if tiles * k > units or steps // k < _MIN_STEPS_PER_CLUSTER_SPLIT or clusters[k - 1] < tiles:
+                continue
+            if k > 2 and -(-groups // k) * (k - 1) * part > stages * stage:
+                continue
+            cost = -(-steps // k) + _CLUSTER_OVERHEAD_STEPS
+            if cost < best:
+                best, ctas = cost, tiles * k
+        k = min(units // tiles, steps // _MIN_STEPS_PER_SPLIT)
+        if k >= 2:
+            cost = -(-steps // k) + _WORKSPACE_OVERHEAD_STEPS + k // 2
+            if cost < best:
+                best, ctas = cost, tiles * k
+        g = min(total // _MIN_STEPS_PER_SPLIT, units)
+        if g > tiles:
+            cost = -(-total // g) + _BALANCED_OVERHEAD_STEPS
+            if cost < best:
+                best, ctas = cost, g
     else:
         # enough tiles for every unit: one CTA per tile (whole waves, each CTA its own start and end), or one
         # persistent CTA per unit on an equal range of the (tile, step) line -- only if the K/V of the heads

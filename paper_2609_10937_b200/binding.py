@@ -33,7 +33,7 @@ class AttnHwDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "struct_bytes", "num_units", "local_mem_bytes", "regs_per_unit", "max_regs_per_thread", "simd_width",
         "acc_mem_lanes", "acc_mem_columns", "atom_m", "atom_n", "atom_k", "atom_n_max", "elem_bytes", "cache_bytes",
-    )] + [("hbm_gbps", ctypes.c_double), ("peak_tflops", ctypes.c_double), ("sm_clock_mhz", ctypes.c_double)]
+    )] + [("max_clusters", ctypes.c_int32 * 8)] + [("hbm_gbps", ctypes.c_double), ("peak_tflops", ctypes.c_double), ("sm_clock_mhz", ctypes.c_double)]
 
 
 class AttnTiles(ctypes.Structure):

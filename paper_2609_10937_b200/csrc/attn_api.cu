@@ -276,7 +276,7 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
       t.ctas = t.tiles * ovr->kv_splits;
     } else {
       t.ctas = attn_internal::grid_size(desc, B * H, (L + t.tile_q - 1) / t.tile_q, steps, t.tile_q / t.tile_kv, causal,
-                                        2LL * L * d * desc.elem_bytes);
+                                        2LL * L * d * desc.elem_bytes, 4 * t.n_q, d, (long long)t.kv_stages * stage);
     }
     t.kv_splits = (t.ctas + t.tiles - 1) / t.tiles;
     if (t.ctas < 1) return ATTN_ERR_BAD_TILES;
@@ -336,6 +336,35 @@ extern "C" int attn_hw_desc_query(int device, attn_hw_desc* out) {
   out->sm_clock_mhz = clock_khz / 1000.0;
   // dense bf16: 8192 FLOP per clock per SM
   out->peak_tflops = 8192.0 * sms * (clock_khz * 1e3) / 1e12;
+  // Resident clusters of k CTAs, asked for the kernel that uses them at its largest shared-memory footprint.
+  {
+    int cur = 0;
+    ATTN_CUDA_TRY(cudaGetDevice(&cur));
+    if (cur != device) ATTN_CUDA_TRY(cudaSetDevice(device));
+    auto kern = attn::attn_fwd_kernel<128, 128, 2, false, true, true>;
+    const int smem = attn::FwdSmem<128, 128, 2>::total(4);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    for (int k = 1; k <= 8; ++k) {
+      int n = 0;
+      if (e == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(sms / k * k));
+        cfg.blockDim = dim3(512);
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = k;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) n = 0;
+      }
+      out->max_clusters[k - 1] = n;
+    }
+    (void)cudaGetLastError();
+    if (cur != device) ATTN_CUDA_TRY(cudaSetDevice(cur));
+  }
   return ATTN_OK;
 }
 

@@ -35,6 +35,12 @@ constexpr int kMinStepsPerSplit = 4;
 constexpr int kSegmentOverheadSteps = 3;  // Q load + first product + partial write/merge, in units of one KV step
 constexpr int kCtaOverheadSteps = 2;      // start and end of a CTA that handles one whole Q tile
 constexpr int kTransitionSteps = 1;       // a persistent CTA moving on to its next Q tile
+// Under-occupied grids (fewer Q tiles than units): cost of the end of a CTA's work in KV steps, measured on B200 --
+constexpr int kMinStepsPerClusterSplit = 2;
+constexpr int kClusterOverheadSteps = 5;     // k CTAs per tile as one cluster: partials through distributed shared memory
+constexpr int kWorkspaceOverheadSteps = 8;   // k CTAs per tile, partials through the workspace (plus k / 2: parts to merge)
+constexpr int kBalancedOverheadSteps = 12;   // equal ranges of the unit line: two partial pieces per CTA, staggered merges
+constexpr int kLandingPartExtra = 256;       // m and delta of the 32 rows of one part
 
 inline int floor_to(int x, int m) { return (x / m) * m; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -71,7 +77,7 @@ long long attn_internal::head_units(int q_tiles, int steps, int ratio, int causa
 
 // Occupancy step of the derivation (shared with the tile-override path of the launcher).
 int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int steps, int ratio, int causal,
-                             long long kv_bytes_per_head) {
+                             long long kv_bytes_per_head, int groups, int part_floats_per_row, long long ring_bytes) {
   const long long tiles_ll = (long long)heads * q_tiles;
   const long long total = (long long)heads * head_units(q_tiles, steps, ratio, causal);
   if (causal) {
@@ -95,17 +101,38 @@ int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int 
     if (cached && cost_balanced < cost_tiles) return (int)g;
     return (int)tiles_ll;
   }
-  int k = h.num_units / tiles;
-  const int k_max = steps / kMinStepsPerSplit;
-  if (k > k_max) k = k_max;
-  if (k < 1) k = 1;
-  const int cost_uniform = ceil_div(steps, k) + kSegmentOverheadSteps;
-  long long g = total / kMinStepsPerSplit;
-  if (g > h.num_units) g = h.num_units;
-  int ctas = tiles * k;
-  if (g > (long long)tiles * k) {
-    const int cost_balanced = (int)((total + g - 1) / g) + 2 * kSegmentOverheadSteps;
-    if (cost_balanced < cost_uniform) ctas = (int)g;
+  // Fewer tiles than units: k CTAs per tile along the key axis, or equal ranges of the unit line.  Costs in KV steps
+  // per CTA; the cheapest wins, ties go to the earlier candidate.
+  int ctas = tiles;                                          // one CTA per tile, nothing to merge
+  long long best = steps + kCtaOverheadSteps;
+  // (1) k CTAs per tile as one cluster: the tile's clusters must all be resident, every CTA needs a few steps, and
+  // what a CTA receives must fit its landing area -- for two parts the Q buffer, else the K/V ring: the 32-row
+  // groups one CTA merges, times the k-1 parts of each.
+  for (int k = 2; k <= 8; ++k) {
+    if ((long long)tiles * k > h.num_units || steps / k < kMinStepsPerClusterSplit || h.max_clusters[k - 1] < tiles) continue;
+    const long long landing = (long long)ceil_div(groups, k) * (k - 1) * (32LL * 4 * part_floats_per_row + kLandingPartExtra);
+    if (k > 2 && landing > ring_bytes) continue;
+    const long long cost = ceil_div(steps, k) + kClusterOverheadSteps;
+    if (cost < best) { best = cost; ctas = tiles * k; }
+  }
+  // (2) k CTAs per tile, partials through the workspace
+  {
+    int k = h.num_units / tiles;
+    const int k_max = steps / kMinStepsPerSplit;
+    if (k > k_max) k = k_max;
+    if (k >= 2) {
+      const long long cost = ceil_div(steps, k) + kWorkspaceOverheadSteps + k / 2;
+      if (cost < best) { best = cost; ctas = tiles * k; }
+    }
+  }
+  // (3) equal ranges
+  {
+    long long g = total / kMinStepsPerSplit;
+    if (g > h.num_units) g = h.num_units;
+    if (g > tiles) {
+      const long long cost = (total + g - 1) / g + kBalancedOverheadSteps;
+      if (cost < best) { best = cost; ctas = (int)g; }
+    }
   }
   return ctas;
 }
@@ -191,8 +218,9 @@ void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, int ca
   const int tiles = B * H * ceil_div(L, tile_q);
   const int steps = ceil_div(L, tile_kv);
   const int under = tiles < h.num_units;
+  // (4 n_q groups of 32 rows per tile; a part of one group is 32 rows of d fp32 values plus statistics)
   const int ctas = attn_internal::grid_size(h, B * H, ceil_div(L, tile_q), steps, tile_q / tile_kv, causal,
-                                             2LL * L * d * h.elem_bytes);
+                                             2LL * L * d * h.elem_bytes, 4 * n_q, d, (long long)stages * stage);
   const int kv_splits = ceil_div(ctas, tiles);
 
   t->feasible = 1;
@@ -234,6 +262,11 @@ extern "C" int attn_hw_desc_b200(attn_hw_desc* out) {
   out->atom_n = 16;
   out->atom_k = 16;
   out->atom_n_max = 256;
+  {
+    // resident clusters of k CTAs with one CTA per SM (the occupancy query on a B200: 8 GPCs of unequal size)
+    static const int kClusters[8] = {148, 74, 45, 33, 26, 22, 15, 15};
+    for (int k = 0; k < 8; ++k) out->max_clusters[k] = kClusters[k];
+  }
   out->elem_bytes = 2;
   out->cache_bytes = 126 << 20;   // L2
   out->hbm_gbps = 7700.0;

@@ -65,13 +65,13 @@ def test_gemm_plan_closed_form(binding):
 
 def test_struct_sizes_match_the_header(binding):
     d = binding.hw_desc_b200()
-    assert d.struct_bytes == ctypes.sizeof(binding.AttnHwDesc) == 80
+    assert d.struct_bytes == ctypes.sizeof(binding.AttnHwDesc) == 112
     assert ctypes.sizeof(binding.AttnTiles) == 72
     assert binding.AttnTiles.causal.offset == 68
 
 
 def _desc_dict(d):
-    return {n: getattr(d, n) for n, _ in d._fields_}
+    return {n: (list(getattr(d, n)) if n == "max_clusters" else getattr(d, n)) for n, _ in d._fields_}
 
 
 def test_b200_plan_equals_oracle_restatement(binding):

@@ -15,7 +15,8 @@ CDNA = dict(lds_bytes=64 * 1024, regs_per_thread=256, wavefront=64, atom_m=16, a
 
 B200 = dict(num_units=148, local_mem_bytes=232448, regs_per_unit=65536, max_regs_per_thread=255,
             simd_width=32, acc_mem_lanes=128, acc_mem_columns=512, atom_m=128, atom_n=16, atom_k=16,
-            atom_n_max=256, elem_bytes=2, cache_bytes=126 << 20)
+            atom_n_max=256, elem_bytes=2, cache_bytes=126 << 20,
+            max_clusters=[148, 74, 45, 33, 26, 22, 15, 15])
 
 
 def test_table2_register_use_and_feasibility():
@@ -81,7 +82,10 @@ def test_tmem_machine_capacity_invariants(B, H, L, d):
     assert 0 < t["wave_efficiency"] <= 1.0
     if t["ctas"] > t["tiles"]:
         assert t["under_occupied"] and t["ctas"] <= 148
-        assert t["tiles"] * math.ceil(L / t["tile_kv"]) // t["ctas"] >= 4      # at least 4 KV steps per CTA
+        k = t["ctas"] // t["tiles"]
+        clustered = t["ctas"] % t["tiles"] == 0 and B200["max_clusters"][k - 1] >= t["tiles"]
+        # at least 4 KV steps per CTA; 2 where the CTAs of a tile form a cluster
+        assert t["tiles"] * math.ceil(L / t["tile_kv"]) // t["ctas"] >= (2 if clustered else 4)
         assert t["ctas"] % t["tiles"] == 0 or t["ctas"] == 148                   # uniform split or one range per SM
 
 
@@ -103,5 +107,20 @@ def test_tmem_machine_expected_defaults_for_the_benchmark_shapes():
     t = po.derive_tiles_tmem_machine(B200, 1, 43, 4096, 128)                             # 86 MiB: over
     assert (t["tiles"], t["ctas"]) == (688, 688)
     assert po.derive_tiles_tmem_machine(dict(B200, cache_bytes=0), 1, 4, 16384, 128)["ctas"] == 256
+    # Fewer tiles than SMs.  Costs in KV steps per CTA: one CTA per tile steps + 2; k CTAs per tile as a cluster
+    # ceil(steps / k) + 5 (k <= 8, at least 2 steps each, that many clusters resident, landing areas fit);
+    # through the workspace ceil(steps / k) + 8 + k // 2 (at least 4 steps each); equal ranges ceil(total / g) + 12.
+    ctas = lambda B, H, L, d, desc=B200: po.derive_tiles_tmem_machine(desc, B, H, L, d)["ctas"]
+    assert ctas(1, 8, 2048, 128) == 128        # 64 tiles x 16 steps: clusters of 2 (8 + 5) against ranges (7 + 12)
+    assert ctas(1, 4, 1024, 128) == 64         # 16 tiles x 8 steps: clusters of 4, two steps each (2 + 5)
+    assert ctas(1, 1, 4096, 128) == 64         # 16 tiles x 32: clusters of 4 (8 + 5); 16 clusters of 8 are not resident (15)
+    assert ctas(1, 1, 2048, 128) == 64         # 8 tiles x 16: clusters of 8 fit the ring (1 group x 7 parts) and 15 >= 8 are resident
+    assert ctas(1, 3, 3000, 128) == 108        # 36 tiles: 36 clusters of 4 are not resident (33), 36 of 3 are
+    assert ctas(1, 2, 8192, 128) == 128        # 64 tiles x 64: clusters of 2 (32 + 5) against ranges (28 + 12)
+    assert ctas(1, 1, 16384, 128) == 148       # 64 tiles x 128: ranges (56 + 12) against clusters of 2 (64 + 5)
+    assert ctas(1, 4, 8192, 128) == 128        # 128 tiles: whole tiles (64 + 2) against ranges (56 + 12)
+    no_clusters = dict(B200, max_clusters=[0] * 8)
+    assert ctas(1, 8, 2048, 128, no_clusters) == 128   # workspace split in two: 8 + 8 + 1 against ranges 7 + 12
+    assert ctas(1, 1, 4096, 128, no_clusters) == 128   # 16 tiles x 32: eight parts through the workspace (4 + 8 + 4) = ranges (4 + 12): tie
     assert not po.derive_tiles_tmem_machine(B200, 1, 1, 1024, 72)["feasible"]          # d not a multiple of 16
     assert not po.derive_tiles_tmem_machine(B200, 1, 1, 1024, 512)["feasible"]         # d beyond the atom's N
