@@ -128,6 +128,13 @@ int attn_hw_desc_query(int device, attn_hw_desc *out);
  * CUDA calls, no search.  Fills *out and returns ATTN_OK even when the result
  * is infeasible (out->feasible == 0 and out->binding_constraint says why);
  * returns ATTN_ERR_INVALID_ARG for null pointers or a bad struct_bytes.
+ * Occupancy step with fewer Q tiles than units (costs in KV steps per CTA, the
+ * cheapest wins, ties to the earlier): one CTA per tile, steps + 2; k CTAs per
+ * tile along the keys as one thread-block cluster, ceil(steps / k) + 5 (2 <= k <= 8,
+ * tiles * k <= num_units, steps / k >= 2, max_clusters[k-1] >= tiles, landing areas
+ * fit); k CTAs per tile through the workspace, ceil(steps / k) + 8 + k / 2 with
+ * k = min(num_units / tiles, steps / 4); equal ranges of the (tile, step) line for
+ * G = min(num_units, tiles * steps / 4) CTAs, ceil(tiles * steps / G) + 12.
  */
 int attn_plan(const attn_hw_desc *desc, int B, int H, int L, int d, attn_tiles *out);
 
