@@ -272,7 +272,7 @@ def run_ours(args):
             "peak_source": f"{peaks['source']} cuBLAS bf16 burst (kernel timed alone)",
             "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
             "frac_of_nominal_2250": achieved / 2250.0,
-            "kernel": "attn_fwd_kernel<128,128,2,false> (one launch per step; split-key partials are merged in the same kernel)",
+            "kernel": "attn_fwd_kernel<128,128,2,false,false,false> (non-causal, balanced key ranges; one launch per step; split-key partials are merged in the same kernel)",
             "algorithmic_flops_per_launch": flops,
             "unfused_traffic_bytes_bf16_scores": traffic.unfused_bytes(case.B, case.H, case.L, case.d, 2, 2),
             "compulsory_traffic_bytes": traffic.fused_bytes(case.B, case.H, case.L, case.d, 2),
