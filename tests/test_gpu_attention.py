@@ -153,6 +153,19 @@ def test_uniform_split_through_clusters(env, d, n_q, kv_splits, L, cluster):
     assert float((o1.float() - whole.float()).abs().max()) <= 2e-2
 
 
+@pytest.mark.parametrize("B,H,L,d,k", [
+    (1, 4, 1024, 128, 4), (1, 1, 2048, 128, 8), (1, 1, 4096, 128, 4), (1, 3, 3000, 128, 3), (1, 2, 8192, 128, 2),
+    (1, 8, 1024, 64, 4), (1, 1, 2048, 64, 8), (2, 3, 1500, 64, 3), (1, 1, 520, 128, 1), (1, 12, 1100, 128, 2), (1, 5, 333, 128, 1)])
+def test_default_plan_of_under_occupied_shapes(env, B, H, L, d, k):
+    """Fewer Q tiles than SMs: the closed-form plan picks k CTAs per tile as one cluster; the launch follows it."""
+    torch, _, binding = env
+    t = binding.plan(binding.hw_desc_query(0), B, H, L, d)
+    assert t.tiles < 148 and t.ctas == t.tiles * k
+    rows = None if L <= 2048 else np.unique(np.concatenate([[0, L - 1], np.random.default_rng(L).integers(0, L, 96)])).astype(np.int32)
+    _run_and_compare(env, _case("under", B, H, L, d, sigma_qk=math.sqrt(3.0)), binding.forward, rows=rows)
+    assert binding.last_cluster_size() == (k if k > 1 else 0)
+
+
 @pytest.mark.parametrize("n_q,tile_kv,kv_stages,kv_splits", [
     (2, 128, 0, 1), (2, 128, 2, 1), (2, 128, 3, 3), (2, 64, 0, 1), (2, 64, 4, 5),
     (1, 128, 0, 1), (1, 64, 0, 2), (1, 128, 3, 7)])
