@@ -139,7 +139,24 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   p.o = reinterpret_cast<__nv_bfloat16*>(o);
   p.counters = reinterpret_cast<unsigned int*>(ws);                   // head of the workspace
   p.ws = ws ? ws + attn::kCounterBytes / sizeof(float) : nullptr;    // partial results follow
-  const int grid = t.ctas;
+  int grid = t.ctas;
+  p.seg_skip = 0;
+#ifndef ATTN_NO_STRIDED
+  // One CTA per tile with more tiles than SMs: a persistent grid of one CTA per SM runs them in the same order.
+  if (!p.causal && t.ctas == t.tiles) {
+    int dev = 0, sms = 0;
+    ATTN_CUDA_TRY(cudaGetDevice(&dev));
+    static int sm_count[kMaxDevices] = {};
+    if (dev >= 0 && dev < kMaxDevices) {
+      if (sm_count[dev] == 0) ATTN_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+      sms = sm_count[dev];
+    }
+    if (sms > 0 && t.tiles > sms) {
+      grid = sms;
+      p.seg_skip = (long long)(grid - 1) * p.n_steps;
+    }
+  }
+#endif
   const long long total_units = p.head_units * BH;
   // at least one KV step per CTA; when Q tiles are shared, the counters of every (CTA, sub-tile, warp) --
   // two each -- must fit the counter block

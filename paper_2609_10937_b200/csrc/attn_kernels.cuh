@@ -176,6 +176,7 @@ struct FwdParams {
   float* ws;               // partial results of Q tiles shared by several CTAs
   unsigned int* counters;  // arrival counters of shared Q tiles; zero between launches
   int cluster_k;           // > 1: the k CTAs of a Q tile are one thread-block cluster (uniform key split only)
+  long long seg_skip;      // > 0: (gridDim.x - 1) * n_steps -- CTA c walks the whole tiles c, c + gridDim.x, ...
 };
 
 // Work decomposition.  A work unit is one KV step of one Q tile.  Q tile q of a head needs
@@ -217,7 +218,8 @@ struct Segment { int tile, q, j0, j1, n, bh, q_row0, seg, steps_t; bool full; lo
 // it was before causal support existed -- measured, helper structs here cost several per cent.)
 template <bool CAUSAL>
 __device__ __forceinline__ bool next_segment(long long& u, long long u_hi, int& seg_ctr, int n_steps, int q_tiles,
-                                             int ratio, long long head_units, int tile_rows, Segment& sg) {
+                                             int ratio, long long head_units, int tile_rows, Segment& sg,
+                                             long long skip) {
   if (u >= u_hi) return false;
   if constexpr (!CAUSAL) {
     sg.tile = (int)(u / n_steps);
@@ -229,7 +231,7 @@ __device__ __forceinline__ bool next_segment(long long& u, long long u_hi, int& 
     const long long left = u_hi - u;
     sg.j1 = (left < (long long)(sg.steps_t - sg.j0)) ? sg.j0 + (int)left : sg.steps_t;
     sg.n = sg.j1 - sg.j0;
-    u += sg.n;
+    u += sg.n + skip;                                   // skip > 0: whole tiles, every gridDim.x-th one
   } else {
     for (;;) {
       sg.bh = (int)(u / head_units);
@@ -434,7 +436,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int cta = blockIdx.x;
   const long long G = gridDim.x;
   const long long T = p.head_units * (p.tiles / p.q_tiles);
-  const long long u_lo = range_begin(cta, T, G), u_hi = range_begin(cta + 1, T, G);
+  // (seg_skip > 0: one CTA per tile executed by a persistent grid -- CTA c takes the whole tiles c, c + G, c + 2G, ...,
+  // the order in which the hardware would have started one CTA per tile, without a CTA's start and end per tile)
+  const long long u_lo = p.seg_skip ? (long long)cta * p.n_steps : range_begin(cta, T, G);
+  const long long u_hi = p.seg_skip ? T : range_begin(cta + 1, T, G);
 
   ATTN_TRACE_CTA(0);
   if (threadIdx.x == 0) {
@@ -523,7 +528,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       long long u = u_lo;
       int seg_ctr = 0;
       Segment sg;
-      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg)) {
+      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg, p.seg_skip)) {
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
       float m_run = -INFINITY, delta = 0.f;
@@ -1050,7 +1055,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       long long u = u_lo;
       int seg_ctr = 0;
       Segment sg;
-      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg)) {
+      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg, p.seg_skip)) {
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
       for (int jj = 0; ok && jj < n; ++jj, ++g) {
@@ -1106,7 +1111,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       long long u = u_lo;
       int seg_ctr = 0;
       Segment sg;
-      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg)) {
+      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg, p.seg_skip)) {
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
       ok = wait_bar_warp(smem_u32(&misc->q_full[0]), seg & 1, abort_flag, wait_info(kRoleMma, kBarQ, seg));
@@ -1267,7 +1272,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       long long u = u_lo;
       int seg_ctr = 0;
       Segment sg;
-      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg)) {
+      while (ok && next_segment<CAUSAL>(u, u_hi, seg_ctr, p.n_steps, p.q_tiles, p.ratio, p.head_units, NQ * kSub, sg, p.seg_skip)) {
         const int tile = sg.tile, j0 = sg.j0, j1 = sg.j1, n = sg.n, bh = sg.bh, q_row0 = sg.q_row0, seg = sg.seg;
         (void)tile; (void)j0; (void)j1; (void)bh; (void)q_row0; (void)seg;
         if (seg > 0 &&
