@@ -636,7 +636,12 @@ int softmax_launch(const void* s, void* pout, long long rows, int cols, float sc
   else if (nvec <= 512) gemm::softmax_rows_kernel<4, 128><<<grid, 128, 0, stream>>>(sp, pp, cols, scale_log2);
   else if (nvec <= 1024) gemm::softmax_rows_kernel<4, 256><<<grid, 256, 0, stream>>>(sp, pp, cols, scale_log2);
   else if (nvec <= 2048) gemm::softmax_rows_kernel<8, 256><<<grid, 256, 0, stream>>>(sp, pp, cols, scale_log2);
-  else gemm::softmax_rows_kernel<32, 128><<<grid, 128, 0, stream>>>(sp, pp, cols, scale_log2);
+  else {
+    // wider than the registers of one block hold: the row is staged in shared memory (2 bytes per column)
+    auto kern = gemm::softmax_rows_staged_kernel<256>;
+    ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
+    kern<<<grid, 256, cols * 2, stream>>>(sp, pp, cols, scale_log2);
+  }
   ATTN_CUDA_TRY(cudaGetLastError());
   ++t_launch_count;
   return ATTN_OK;

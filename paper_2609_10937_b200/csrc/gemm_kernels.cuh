@@ -7,6 +7,7 @@
 //                 sub-tiles x 256 columns accumulated in tensor memory) -> eight epilogue warps
 //                 (tensor memory -> bf16 -> shared-memory staging -> TMA store).
 //   softmax_rows_kernel  one CTA per row, the row held in registers: one read, one write.
+//   softmax_rows_staged_kernel  the same for rows too wide for registers: staged in shared memory.
 //
 // Every device-side wait is bounded (see attn_kernels.cuh).
 #pragma once
@@ -313,6 +314,74 @@ softmax_rows_kernel(const __nv_bfloat16* s, __nv_bfloat16* pout, int cols, float
       }
       dst[idx] = make_uint4(o[0], o[1], o[2], o[3]);
     }
+  }
+}
+
+// Rows too wide for registers (more than 2048 vectors of 8 columns): the row is staged in shared memory (2 bytes per
+// column) -- still one read and one write of the matrix.  Pass 1: global -> shared, running maximum on the packed
+// words; pass 2: sum of exp2(scale x - m) from shared memory; pass 3: the exponentials again, normalised, to global
+// (two exponentials per element cost less than a second trip to HBM or than fp32 staging, which would halve the rows
+// in flight per SM).
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS)
+softmax_rows_staged_kernel(const __nv_bfloat16* s, __nv_bfloat16* pout, int cols, float scale_log2) {
+  extern __shared__ __align__(16) uint8_t smem_row[];
+  __shared__ float sm_m[THREADS / 32], sm_d[THREADS / 32];
+  const size_t row = blockIdx.x;
+  const uint4* src = reinterpret_cast<const uint4*>(s + row * (size_t)cols);
+  uint4* dst = reinterpret_cast<uint4*>(pout + row * (size_t)cols);
+  uint4* stage = reinterpret_cast<uint4*>(smem_row);
+  const int nvec = cols / 8;
+  uint32_t mx2 = 0xFF80FF80u;                               // (-inf, -inf) in bf16
+#pragma unroll 4
+  for (int idx = threadIdx.x; idx < nvec; idx += THREADS) {
+    const uint4 q = src[idx];
+    stage[idx] = q;                                         // (each thread re-reads only what it wrote: no barrier)
+    mx2 = max_bf16x2(max_bf16x2(mx2, q.x), max_bf16x2(max_bf16x2(q.y, q.z), q.w));
+  }
+  float m = fmaxf(__uint_as_float(mx2 << 16), __uint_as_float(mx2 & 0xFFFF0000u)) * scale_log2;
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+  if ((threadIdx.x & 31) == 0) sm_m[threadIdx.x >> 5] = m;
+  __syncthreads();
+  float mr = sm_m[0];
+#pragma unroll
+  for (int k = 1; k < THREADS / 32; ++k) mr = fmaxf(mr, sm_m[k]);
+  const float neg_m = (mr == -INFINITY) ? 0.f : -mr;
+  const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2), negm2 = pack_f32x2(neg_m, neg_m);
+  auto exp_pair = [&](uint32_t w) -> uint64_t {
+    const uint64_t t = fma_f32x2(pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u)), scale2, negm2);
+    float t0, t1;
+    unpack_f32x2(t, t0, t1);
+    return pack_f32x2(ex2_approx(t0), ex2_approx(t1));
+  };
+  uint64_t d2 = 0ull;
+#pragma unroll 2
+  for (int idx = threadIdx.x; idx < nvec; idx += THREADS) {
+    const uint4 q = stage[idx];
+    d2 = add_f32x2(d2, add_f32x2(add_f32x2(exp_pair(q.x), exp_pair(q.y)), add_f32x2(exp_pair(q.z), exp_pair(q.w))));
+  }
+  float d0, d1;
+  unpack_f32x2(d2, d0, d1);
+  float d = d0 + d1;
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+  if ((threadIdx.x & 31) == 0) sm_d[threadIdx.x >> 5] = d;
+  __syncthreads();
+  float dr = sm_d[0];
+#pragma unroll
+  for (int k = 1; k < THREADS / 32; ++k) dr += sm_d[k];
+  const float inv = 1.0f / dr;
+  const uint64_t inv2 = pack_f32x2(inv, inv);
+  auto out_pair = [&](uint32_t w) -> uint32_t {
+    float a0, a1;
+    unpack_f32x2(mul_f32x2(exp_pair(w), inv2), a0, a1);
+    return pack_bf16x2(a0, a1);
+  };
+#pragma unroll 2
+  for (int idx = threadIdx.x; idx < nvec; idx += THREADS) {
+    const uint4 q = stage[idx];
+    dst[idx] = make_uint4(out_pair(q.x), out_pair(q.y), out_pair(q.z), out_pair(q.w));
   }
 }
 
