@@ -80,7 +80,8 @@ def test_matrix_product_full_size_sampled(env):
     _check_product(env, 1, 4096, 4096, 4096, "kn", seed=2, rows_per_batch=48)
 
 
-@pytest.mark.parametrize("rows,cols", [(4, 8), (7, 256), (33, 2048), (5, 2056), (3, 16384), (2, 32768), (9, 1000)])
+@pytest.mark.parametrize("rows,cols", [(4, 8), (7, 256), (33, 2048), (5, 2056), (3, 16384), (2, 32768), (9, 1000),
+                                       (3, 16392), (2, 20000), (5, 32760)])   # the last three: staged in shared memory
 def test_row_softmax_matches_oracle(env, rows, cols):
     torch, go, binding = env
     rng = np.random.default_rng([rows, cols])
