@@ -127,13 +127,14 @@ def test_pipelined_kernel_matches_oracle_small(env, B, H, L, d):
     (128, 2, 5, 2560, 0),     # five parts of a two-sub-tile CTA do not fit the ring: through the workspace
     (64, 2, 2, 1408, 2), (64, 2, 3, 1500, 3), (64, 2, 4, 2048, 4),
     (64, 2, 5, 1280, 5), (64, 2, 8, 1024, 8),      # half the bytes per part at d = 64: up to eight parts fit the ring
-    (128, 1, 2, 1408, 2), (128, 1, 4, 1408, 4), (64, 1, 3, 777, 3)])
+    (128, 1, 2, 1408, 2), (128, 1, 4, 1408, 4), (64, 1, 3, 777, 3),
+    (128, 1, 5, -1408, 5), (64, 1, 8, -1100, 8)])  # (one head) more CTAs than 32-row groups: the last ranks only publish
 def test_uniform_split_through_clusters(env, d, n_q, kv_splits, L, cluster):
     """Uniform key splits: the CTAs of a Q tile run as one thread-block cluster and exchange their partial results
     through distributed shared memory where the landing areas fit; the result is the oracle's either way, the
     same bits run to run, and the same bits as with one CTA per tile merged nowhere (up to the merge's rounding)."""
     torch, _, binding = env
-    case = _case("cluster", 1, 3, L, d, sigma_qk=math.sqrt(3.0))
+    case = _case("cluster", 1, 3 if L > 0 else 1, abs(L), d, sigma_qk=math.sqrt(3.0))
     seen = []
 
     def run(a, b, c):
