@@ -220,7 +220,29 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
     kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
     return ATTN_OK;
   };
-  if (p.causal) rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, true, false>);
+  if (p.causal && t.ctas == 2 * t.tiles && p.ratio >= 2) {
+    // causal, two CTAs per tile as one cluster: each half of the tile's own key steps (no other way to run this grid)
+    auto kern = attn::attn_fwd_kernel<D, TKV, NQ, true, true, true>;
+    ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(512);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    attn::FwdParams pc = p;
+    pc.cluster_k = 2;
+    pc.seg_skip = -1;
+    ATTN_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, to, pc));
+    t_cluster_size = 2;
+    rc = ATTN_OK;
+  } else if (p.causal) rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, true, false>);
   else if (eager) rc = launch_eager(attn::attn_fwd_kernel<D, TKV, NQ, false, true>, attn::attn_fwd_kernel<D, TKV, NQ, false, true, true>);
   else rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, false, false>);
   if (rc != ATTN_OK) return rc;

@@ -177,6 +177,7 @@ struct FwdParams {
   unsigned int* counters;  // arrival counters of shared Q tiles; zero between launches
   int cluster_k;           // > 1: the k CTAs of a Q tile are one thread-block cluster (uniform key split only)
   long long seg_skip;      // > 0: (gridDim.x - 1) * n_steps -- CTA c walks the whole tiles c, c + gridDim.x, ...
+                           // < 0 (causal, clusters of two): CTA c takes half of the key steps of tile c / 2
 };
 
 // Work decomposition.  A work unit is one KV step of one Q tile.  Q tile q of a head needs
@@ -232,6 +233,20 @@ __device__ __forceinline__ bool next_segment(long long& u, long long u_hi, int& 
     sg.j1 = (left < (long long)(sg.steps_t - sg.j0)) ? sg.j0 + (int)left : sg.steps_t;
     sg.n = sg.j1 - sg.j0;
     u += sg.n + skip;                                   // skip > 0: whole tiles, every gridDim.x-th one
+  } else if (skip < 0) {
+    // causal, two CTAs per tile as one cluster (u = the CTA's index): each takes half of the tile's own key steps --
+    // at least one each, a tile has at least `ratio` >= 2 of them
+    const int t_lin = (int)(u >> 1), part = (int)(u & 1);
+    sg.bh = t_lin / q_tiles;
+    sg.q = t_lin % q_tiles;
+    sg.tile = t_lin;
+    sg.steps_t = tile_steps(n_steps, ratio, 1, sg.q);
+    sg.unit0 = 0;
+    const int half = (sg.steps_t + 1) >> 1;
+    sg.j0 = part ? half : 0;
+    sg.j1 = part ? sg.steps_t : half;
+    sg.n = sg.j1 - sg.j0;
+    u = u_hi;
   } else {
     for (;;) {
       sg.bh = (int)(u / head_units);
@@ -438,8 +453,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const long long T = p.head_units * (p.tiles / p.q_tiles);
   // (seg_skip > 0: one CTA per tile executed by a persistent grid -- CTA c takes the whole tiles c, c + G, c + 2G, ...,
   // the order in which the hardware would have started one CTA per tile, without a CTA's start and end per tile)
-  const long long u_lo = p.seg_skip ? (long long)cta * p.n_steps : range_begin(cta, T, G);
-  const long long u_hi = p.seg_skip ? T : range_begin(cta + 1, T, G);
+  // (seg_skip < 0, causal: two CTAs per tile -- the "range" is the CTA's index)
+  const long long u_lo = p.seg_skip > 0 ? (long long)cta * p.n_steps : p.seg_skip < 0 ? (long long)cta : range_begin(cta, T, G);
+  const long long u_hi = p.seg_skip > 0 ? T : p.seg_skip < 0 ? (long long)cta + 1 : range_begin(cta + 1, T, G);
 
   ATTN_TRACE_CTA(0);
   if (threadIdx.x == 0) {

@@ -41,6 +41,9 @@ constexpr int kClusterOverheadSteps = 5;     // k CTAs per tile as one cluster: 
 constexpr int kWorkspaceOverheadSteps = 8;   // k CTAs per tile, partials through the workspace (plus k / 2: parts to merge)
 constexpr int kBalancedOverheadSteps = 12;   // equal ranges of the unit line: two partial pieces per CTA, staggered merges
 constexpr int kLandingPartExtra = 256;       // m and delta of the 32 rows of one part
+constexpr int kCausalTileCostUnits = 3;      // cost units that precede every causal tile on the unit line (kernel constant)
+constexpr int kCausalRangesOverheadSteps = 15;   // causal, equal ranges: many short pieces per CTA, merges through the workspace
+constexpr int kCausalPairsOverheadSteps = 6;     // causal, two CTAs per tile as one cluster
 
 inline int floor_to(int x, int m) { return (x / m) * m; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -81,9 +84,17 @@ int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int 
   const long long tiles_ll = (long long)heads * q_tiles;
   const long long total = (long long)heads * head_units(q_tiles, steps, ratio, causal);
   if (causal) {
+    // Equal ranges of the unit line (every tile preceded by kCausalTileCostUnits cost units, as in the kernel), or -- few
+    // and short tiles -- two CTAs per tile as one cluster, each with half of the tile's own key steps: the longest
+    // tile then sets the time, but a CTA has one piece instead of many short ones.  Costs in KV steps, measured.
     long long g = total / kMinStepsPerSplit;
     if (g > h.num_units) g = h.num_units;
     if (g < 1) g = 1;
+    const long long cost_ranges = (total + kCausalTileCostUnits * tiles_ll + g - 1) / g + kCausalRangesOverheadSteps;
+    if (ratio >= 2 && 2 * tiles_ll <= h.num_units && h.max_clusters[1] >= tiles_ll) {
+      const long long cost_pairs = ceil_div(steps, 2) + kCausalPairsOverheadSteps;
+      if (cost_pairs < cost_ranges) return (int)(2 * tiles_ll);
+    }
     return (int)g;
   }
   const int tiles = (int)tiles_ll;

@@ -235,6 +235,24 @@ def test_causal_matches_oracle(env, d, L):
     _run_and_compare(env, case, lambda a, b, c: binding.forward(a, b, c, causal=True), causal=True)
 
 
+@pytest.mark.parametrize("B,H,L,d", [(1, 8, 2048, 128), (1, 4, 1000, 128), (2, 5, 1408, 64), (1, 16, 1024, 128), (1, 3, 300, 64)])
+def test_causal_short_shapes_run_as_pair_clusters(env, B, H, L, d):
+    """Few short tiles: two CTAs per tile as one cluster, each with half of the tile's own key steps."""
+    torch, _, binding = env
+    t = binding.plan(binding.hw_desc_query(0), B, H, L, d, causal=True)
+    assert t.ctas == 2 * t.tiles
+    run = lambda a, b, c: binding.forward(a, b, c, causal=True)
+    _run_and_compare(env, _case("causal_pairs", B, H, L, d, sigma_qk=math.sqrt(3.0)), run, causal=True)
+    assert binding.last_cluster_size() == 2
+    q, k, v = (to_cuda_bf16(x) for x in synth.make_qkv(_case("causal_pairs", B, H, L, d), seed=3))
+    o1, o2 = binding.forward(q, k, v, causal=True), binding.forward(q, k, v, causal=True)
+    ranges = binding.forward_tiles(q, k, v, ctas=min(148, max(1, t.tiles)), causal=True)     # equal ranges, merged elsewhere
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))
+    assert float((o1.float() - ranges.float()).abs().max()) <= 2e-2
+
+
 @pytest.mark.parametrize("kw", [dict(ctas=1), dict(ctas=2), dict(ctas=7), dict(ctas=37), dict(ctas=101),
                                 dict(tile_kv=64), dict(n_q=1), dict(n_q=1, tile_kv=64, ctas=53), dict(kv_stages=2)])
 def test_causal_tile_variants_and_grid_sizes(env, kw):
