@@ -141,10 +141,10 @@ int attn_plan(const attn_hw_desc *desc, int B, int H, int L, int d, attn_tiles *
 /* Same derivation for causal attention (causal != 0): Q tile q needs only the key
  * steps up to its own last row, so the work per tile is unequal and the occupancy
  * step always deals the (Q tile, KV step) units out in equal ranges, one per unit.
- * Exception: with at most num_units / 2 tiles (and that many clusters of two resident), two
- * CTAs per tile as one cluster, each with half of the tile's own key steps, if
- * ceil(steps / 2) + 6 < ceil((units + 3 * tiles) / G) + 15 (short sequences: a CTA then has
- * one piece instead of many short ones).
+ * Exception: k = 2..4 CTAs per tile as one cluster, each with a share of the tile's own key
+ * steps, if tiles * k <= num_units, max_clusters[k-1] >= tiles, ceil(steps / k) >= 2, the
+ * landing areas fit and ceil(steps / k) + 6 < ceil((units + 3 * tiles) / G) + 15 (few short
+ * tiles: a CTA then has one piece instead of many short ones; ctas == k * tiles).
  * (The paper treats non-causal attention only; this applies its -inf masking rule,
  * Section "Online Softmax", to a triangular mask.) */
 int attn_plan_ex(const attn_hw_desc *desc, int B, int H, int L, int d, int causal, attn_tiles *out);

@@ -124,13 +124,21 @@ def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal
     if causal:
         total = B * H * causal_head_units(-(-L // tile_q), steps, tile_q // tile_kv)
         ctas = max(1, min(total // _MIN_STEPS_PER_SPLIT, desc["num_units"]))
-        # equal ranges (3 cost units per tile on the line, 15 steps of overhead) against two CTAs per tile as one
-        # cluster, half of the tile's own key steps each (the longest tile sets the time; 6 steps of overhead)
+        # equal ranges (3 cost units per tile on the line, 15 steps of overhead) against k = 2..4 CTAs per tile as one
+        # cluster, a share of the tile's own key steps each (the longest tile sets the time; 6 steps of overhead)
         cost_ranges = -(-(total + 3 * tiles) // ctas) + 15
         ratio = tile_q // tile_kv
-        if ratio >= 2 and 2 * tiles <= desc["num_units"] and list(desc.get("max_clusters", [0] * 8))[1] >= tiles:
-            if -(-steps // 2) + 6 < cost_ranges:
-                ctas = 2 * tiles
+        best = cost_ranges
+        clusters = list(desc.get("max_clusters", [0] * 8))
+        part = 32 * 4 * d + _LANDING_PART_EXTRA
+        for k in (2, 3, 4):
+            if ratio < 2 or k * tiles > desc["num_units"] or clusters[k - 1] < tiles or -(-steps // k) < 2:
+                continue
+            if k > 2 and -(-(4 * n_q) // k) * (k - 1) * part > stages * stage:
+                continue
+            cost = -(-steps // k) + 6
+            if cost < best:
+                best, ctas = cost, k * tiles
     elif under:
         # one CTA per tile; k CTAs per tile as one cluster; k CTAs per tile through the workspace; equal ranges.
         # The cheapest wins, ties go to the earlier candidate.

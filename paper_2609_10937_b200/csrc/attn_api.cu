@@ -220,8 +220,10 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
     kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
     return ATTN_OK;
   };
-  if (p.causal && t.ctas == 2 * t.tiles && p.ratio >= 2) {
-    // causal, two CTAs per tile as one cluster: each half of the tile's own key steps (no other way to run this grid)
+  const int ck = (t.tiles > 0 && t.ctas % t.tiles == 0) ? t.ctas / t.tiles : 0;
+  const size_t c_landing = ck > 2 ? (size_t)((4 * NQ + ck - 1) / ck) * (ck - 1) * (32 * D * 4 + 256) : 0;
+  if (p.causal && ck >= 2 && ck <= 4 && p.ratio >= 2 && c_landing <= (size_t)t.kv_stages * SM::kStageBytes) {
+    // causal, ck CTAs per tile as one cluster: each a share of the tile's own key steps (the only way to run this grid)
     auto kern = attn::attn_fwd_kernel<D, TKV, NQ, true, true, true>;
     ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     cudaLaunchConfig_t cfg = {};
@@ -231,16 +233,16 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.x = ck;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     attn::FwdParams pc = p;
-    pc.cluster_k = 2;
-    pc.seg_skip = -1;
+    pc.cluster_k = ck;
+    pc.seg_skip = -ck;
     ATTN_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, to, pc));
-    t_cluster_size = 2;
+    t_cluster_size = ck;
     rc = ATTN_OK;
   } else if (p.causal) rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, true, false>);
   else if (eager) rc = launch_eager(attn::attn_fwd_kernel<D, TKV, NQ, false, true>, attn::attn_fwd_kernel<D, TKV, NQ, false, true, true>);

@@ -177,7 +177,7 @@ struct FwdParams {
   unsigned int* counters;  // arrival counters of shared Q tiles; zero between launches
   int cluster_k;           // > 1: the k CTAs of a Q tile are one thread-block cluster (uniform key split only)
   long long seg_skip;      // > 0: (gridDim.x - 1) * n_steps -- CTA c walks the whole tiles c, c + gridDim.x, ...
-                           // < 0 (causal, clusters of two): CTA c takes half of the key steps of tile c / 2
+                           // < 0 (causal, clusters of k = -seg_skip): CTA c takes a share of the key steps of tile c / k
 };
 
 // Work decomposition.  A work unit is one KV step of one Q tile.  Q tile q of a head needs
@@ -234,17 +234,20 @@ __device__ __forceinline__ bool next_segment(long long& u, long long u_hi, int& 
     sg.n = sg.j1 - sg.j0;
     u += sg.n + skip;                                   // skip > 0: whole tiles, every gridDim.x-th one
   } else if (skip < 0) {
-    // causal, two CTAs per tile as one cluster (u = the CTA's index): each takes half of the tile's own key steps --
-    // at least one each, a tile has at least `ratio` >= 2 of them
-    const int t_lin = (int)(u >> 1), part = (int)(u & 1);
+    // causal, k = -skip CTAs per tile as one cluster (u = the CTA's index): the tile's own key steps are dealt out
+    // in equal shares to its first min(k, steps) CTAs; the others have nothing to do (a tile's first rows have
+    // fewer key steps than the cluster has CTAs)
+    const int k = (int)-skip;
+    const int t_lin = (int)(u / k), part = (int)(u % k);
     sg.bh = t_lin / q_tiles;
     sg.q = t_lin % q_tiles;
     sg.tile = t_lin;
     sg.steps_t = tile_steps(n_steps, ratio, 1, sg.q);
+    const int parts = sg.steps_t < k ? sg.steps_t : k;
+    if (part >= parts) return false;
     sg.unit0 = 0;
-    const int half = (sg.steps_t + 1) >> 1;
-    sg.j0 = part ? half : 0;
-    sg.j1 = part ? sg.steps_t : half;
+    sg.j0 = (int)((long long)part * sg.steps_t / parts);
+    sg.j1 = (int)((long long)(part + 1) * sg.steps_t / parts);
     sg.n = sg.j1 - sg.j0;
     u = u_hi;
   } else {
@@ -457,6 +460,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const long long u_lo = p.seg_skip > 0 ? (long long)cta * p.n_steps : p.seg_skip < 0 ? (long long)cta : range_begin(cta, T, G);
   const long long u_hi = p.seg_skip > 0 ? T : p.seg_skip < 0 ? (long long)cta + 1 : range_begin(cta + 1, T, G);
 
+  // CLUSTER: number of CTAs of this CTA's cluster that have key steps (all of them, except for short causal tiles)
+  int cl_parts = p.cluster_k;
+  if constexpr (CLUSTER && CAUSAL) {
+    const int st = tile_steps(p.n_steps, p.ratio, 1, (cta / p.cluster_k) % p.q_tiles);
+    if (st < cl_parts) cl_parts = st;
+  }
+  (void)cl_parts;
   ATTN_TRACE_CTA(0);
   if (threadIdx.x == 0) {
     ATTN_TRACE_MARK(0);
@@ -486,14 +496,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       {
         // Partials travel through distributed shared memory (see the end of a segment).  The merging warps of
         // this CTA -- warp w merges if w mod k is this CTA's rank -- expect the parts of the k-1 other CTAs.
-        mbar_init(smem_u32(&misc->peers_ready), p.cluster_k - 1);
+        mbar_init(smem_u32(&misc->peers_ready), cl_parts - 1);
         for (int w = 0; w < 4 * NQ; ++w) {
           mbar_init(smem_u32(&misc->data_ready[w][0]), 1);
           mbar_init(smem_u32(&misc->data_ready[w][1]), 1);
-          if (w % p.cluster_k == cta % p.cluster_k) {
+          if (w % cl_parts == cta % p.cluster_k) {
             // first the statistics and columns 0..63 of every part, then (d = 128) columns 64..127
-            mbar_arrive_expect_tx(smem_u32(&misc->data_ready[w][0]), (uint32_t)(p.cluster_k - 1) * (32 * 64 * 4 + 256));
-            if (KCH == 2) mbar_arrive_expect_tx(smem_u32(&misc->data_ready[w][1]), (uint32_t)(p.cluster_k - 1) * (32 * 64 * 4));
+            mbar_arrive_expect_tx(smem_u32(&misc->data_ready[w][0]), (uint32_t)(cl_parts - 1) * (32 * 64 * 4 + 256));
+            if (KCH == 2) mbar_arrive_expect_tx(smem_u32(&misc->data_ready[w][1]), (uint32_t)(cl_parts - 1) * (32 * 64 * 4));
           }
         }
       }
@@ -675,9 +685,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (ok) {
           cluster_wait();
           cluster_waited = true;
-          if (p.cluster_k == 2 && warp == 0) {
+          if (cl_parts == 2 && warp == 0) {
             ok = wait_bar_warp(smem_u32(&misc->q_empty), 0, abort_flag, wait_info(kRoleSoftmax, kBarQ, 0x2000));
-            if (ok && lane < 2 && lane != (cta & 1)) mbar_arrive_peer(map_to_cta(smem_u32(&misc->peers_ready), lane));
+            if (ok && lane < 2 && lane != cta % p.cluster_k) mbar_arrive_peer(map_to_cta(smem_u32(&misc->peers_ready), lane));
           }
         }
       }
@@ -750,7 +760,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             // in global memory.  Roles as below ("Who merges"): softmax warp w belongs to rank w mod k.  The
             // landing areas lie in the K/V ring, which is dead in a CTA once the last product of both its
             // sub-tiles has finished; every CTA tells its peers when that is so.
-            const int k = p.cluster_k;
+            const int k = cl_parts;
             const int owner = warp % k, ms = warp / k;
             // Two parts: what a CTA receives fits its Q buffer (O) and the idle staging chunks of its publishing
             // warps (m, delta), and the Q buffer is dead one step before the end.  More parts: the K/V ring,

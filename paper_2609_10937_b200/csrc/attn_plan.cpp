@@ -43,7 +43,7 @@ constexpr int kBalancedOverheadSteps = 12;   // equal ranges of the unit line: t
 constexpr int kLandingPartExtra = 256;       // m and delta of the 32 rows of one part
 constexpr int kCausalTileCostUnits = 3;      // cost units that precede every causal tile on the unit line (kernel constant)
 constexpr int kCausalRangesOverheadSteps = 15;   // causal, equal ranges: many short pieces per CTA, merges through the workspace
-constexpr int kCausalPairsOverheadSteps = 6;     // causal, two CTAs per tile as one cluster
+constexpr int kCausalPairsOverheadSteps = 6;     // causal, k CTAs per tile as one cluster
 
 inline int floor_to(int x, int m) { return (x / m) * m; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -85,17 +85,22 @@ int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int 
   const long long total = (long long)heads * head_units(q_tiles, steps, ratio, causal);
   if (causal) {
     // Equal ranges of the unit line (every tile preceded by kCausalTileCostUnits cost units, as in the kernel), or -- few
-    // and short tiles -- two CTAs per tile as one cluster, each with half of the tile's own key steps: the longest
-    // tile then sets the time, but a CTA has one piece instead of many short ones.  Costs in KV steps, measured.
+    // and short tiles -- k = 2..4 CTAs per tile as one cluster, each with a share of the tile's own key steps: the
+    // longest tile then sets the time, but a CTA has one piece instead of many short ones.  Costs in KV steps, measured.
     long long g = total / kMinStepsPerSplit;
     if (g > h.num_units) g = h.num_units;
     if (g < 1) g = 1;
     const long long cost_ranges = (total + kCausalTileCostUnits * tiles_ll + g - 1) / g + kCausalRangesOverheadSteps;
-    if (ratio >= 2 && 2 * tiles_ll <= h.num_units && h.max_clusters[1] >= tiles_ll) {
-      const long long cost_pairs = ceil_div(steps, 2) + kCausalPairsOverheadSteps;
-      if (cost_pairs < cost_ranges) return (int)(2 * tiles_ll);
+    long long best = cost_ranges;
+    int ctas = (int)g;
+    for (int k = 2; k <= 4 && ratio >= 2; ++k) {
+      if (k * tiles_ll > h.num_units || h.max_clusters[k - 1] < tiles_ll || ceil_div(steps, k) < 2) continue;
+      const long long landing = (long long)ceil_div(groups, k) * (k - 1) * (32LL * 4 * part_floats_per_row + kLandingPartExtra);
+      if (k > 2 && landing > ring_bytes) continue;
+      const long long cost = ceil_div(steps, k) + kCausalPairsOverheadSteps;
+      if (cost < best) { best = cost; ctas = (int)(k * tiles_ll); }
     }
-    return (int)g;
+    return ctas;
   }
   const int tiles = (int)tiles_ll;
   if (tiles_ll >= h.num_units) {

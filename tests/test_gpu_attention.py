@@ -235,18 +235,20 @@ def test_causal_matches_oracle(env, d, L):
     _run_and_compare(env, case, lambda a, b, c: binding.forward(a, b, c, causal=True), causal=True)
 
 
-@pytest.mark.parametrize("B,H,L,d", [(1, 8, 2048, 128), (1, 4, 1000, 128), (2, 5, 1408, 64), (1, 16, 1024, 128), (1, 3, 300, 64)])
-def test_causal_short_shapes_run_as_pair_clusters(env, B, H, L, d):
-    """Few short tiles: two CTAs per tile as one cluster, each with half of the tile's own key steps."""
+@pytest.mark.parametrize("B,H,L,d,k", [(1, 8, 2048, 128, 2), (1, 4, 1000, 128, 4), (2, 5, 1408, 64, 2), (1, 16, 1024, 128, 2),
+                                       (1, 3, 300, 64, 2), (1, 1, 4096, 128, 4), (1, 3, 2500, 128, 4), (1, 5, 1800, 64, 3)])
+def test_causal_short_shapes_run_as_clusters(env, B, H, L, d, k):
+    """Few short tiles: k CTAs per tile as one cluster, each with a share of the tile's own key steps (the tiles
+    at the start of a head have fewer key steps than the cluster has CTAs: some CTAs then have nothing to do)."""
     torch, _, binding = env
     t = binding.plan(binding.hw_desc_query(0), B, H, L, d, causal=True)
-    assert t.ctas == 2 * t.tiles
+    assert t.ctas == k * t.tiles
     run = lambda a, b, c: binding.forward(a, b, c, causal=True)
     _run_and_compare(env, _case("causal_pairs", B, H, L, d, sigma_qk=math.sqrt(3.0)), run, causal=True)
-    assert binding.last_cluster_size() == 2
-    q, k, v = (to_cuda_bf16(x) for x in synth.make_qkv(_case("causal_pairs", B, H, L, d), seed=3))
-    o1, o2 = binding.forward(q, k, v, causal=True), binding.forward(q, k, v, causal=True)
-    ranges = binding.forward_tiles(q, k, v, ctas=min(148, max(1, t.tiles)), causal=True)     # equal ranges, merged elsewhere
+    assert binding.last_cluster_size() == k
+    q, kk, v = (to_cuda_bf16(x) for x in synth.make_qkv(_case("causal_pairs", B, H, L, d), seed=3))
+    o1, o2 = binding.forward(q, kk, v, causal=True), binding.forward(q, kk, v, causal=True)
+    ranges = binding.forward_tiles(q, kk, v, ctas=t.tiles + 1, causal=True)                  # equal ranges, merged elsewhere
     torch.cuda.synchronize()
     assert binding.last_device_status()[0] == 0
     assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))

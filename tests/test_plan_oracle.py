@@ -119,11 +119,14 @@ def test_tmem_machine_expected_defaults_for_the_benchmark_shapes():
     assert ctas(1, 2, 8192, 128) == 128        # 64 tiles x 64: clusters of 2 (32 + 5) against ranges (28 + 12)
     assert ctas(1, 1, 16384, 128) == 148       # 64 tiles x 128: ranges (56 + 12) against clusters of 2 (64 + 5)
     assert ctas(1, 4, 8192, 128) == 128        # 128 tiles: whole tiles (64 + 2) against ranges (56 + 12)
-    # causal: equal ranges, ceil((units + 3 tiles) / G) + 15, against two CTAs per tile as a cluster, ceil(steps / 2) + 6
+    # causal: equal ranges, ceil((units + 3 tiles) / G) + 15, against k = 2..4 CTAs per tile as a cluster,
+    # ceil(steps / k) + 6 (k * tiles <= 148, that many clusters resident, the longest part at least two steps)
     cc = lambda B, H, L, d, desc=B200: po.derive_tiles_tmem_machine(desc, B, H, L, d, causal=True)["ctas"]
     assert cc(1, 8, 2048, 128) == 128          # 64 tiles x <= 16 steps: pairs (8 + 6) against ranges (6 + 15)
     assert cc(1, 4, 4096, 128) == 128          # 64 tiles x <= 32: pairs (16 + 6) against ranges (9 + 15)
-    assert cc(1, 1, 4096, 128) == 68           # 16 tiles: ranges over 68 CTAs (5 + 15) against pairs (16 + 6)
+    assert cc(1, 1, 4096, 128) == 64           # 16 tiles: clusters of 4 (8 + 6) against ranges over 68 CTAs (5 + 15)
+    assert cc(1, 1, 8192, 128) == 128          # 32 tiles x <= 64: clusters of 4 (16 + 6) against ranges (8 + 15)
+    assert cc(1, 3, 300, 64) == 12             # 3 steps: pairs (2 + 6); three parts would be one step each
     assert cc(1, 1, 16384, 128) == 148 and cc(1, 2, 8192, 128) == 148
     assert cc(1, 8, 2048, 128, dict(B200, max_clusters=[0] * 8)) == 144
     no_clusters = dict(B200, max_clusters=[0] * 8)
