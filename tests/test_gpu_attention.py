@@ -428,3 +428,34 @@ def test_persistent_grid_with_ragged_lengths(env, B, H, L, d):
     case = _case("persistent", B, H, L, d)
     _run_and_compare(env, case, binding.forward)
     _run_and_compare(env, case, lambda a, b, c: binding.forward(a, b, c, causal=True), causal=True)
+
+
+def test_random_shapes_every_grid_mode_agrees_with_an_unsplit_run(env):
+    """Seeded random shapes, causal and not: whatever grid the plan picks (one CTA per tile, clusters of 2 to 8,
+    equal ranges, persistent), the output equals that of a launch that shares no Q tile between CTAs, up to the
+    merge's rounding; the modes met are counted so that a change of the plan that stops exercising one shows."""
+    torch, _, binding = env
+    import random
+
+    rng = random.Random(2024)
+    desc = binding.hw_desc_query(0)
+    modes = {}
+    for it in range(120):
+        d = rng.choice([64, 128])
+        causal = rng.random() < 0.5
+        L = rng.choice([rng.randint(1, 300), rng.randint(300, 2500), rng.randint(2500, 7000)])
+        B = rng.randint(1, 2)
+        H = rng.randint(1, max(1, min(40, 50000 // L) // B))
+        g = torch.Generator(device="cuda").manual_seed(it)
+        q, k, v = (torch.randn(B, H, L, d, device="cuda", generator=g).mul_(1.3).to(torch.bfloat16) for _ in range(3))
+        t = binding.plan(desc, B, H, L, d, causal=causal)
+        o = binding.forward(q, k, v, causal=causal)
+        cl = binding.last_cluster_size()
+        ref = binding.forward_tiles(q, k, v, ctas=1 if causal else t.tiles, causal=causal)
+        torch.cuda.synchronize()
+        assert binding.last_device_status()[0] == 0, (B, H, L, d, causal)
+        assert bool(torch.isfinite(o.float()).all())
+        assert float((o.float() - ref.float()).abs().max()) <= 2e-2, (B, H, L, d, causal, t.ctas, t.tiles, cl)
+        mode = ("causal " if causal else "") + ("cluster" if cl else "tiles" if t.ctas == t.tiles else "ranges")
+        modes[mode] = modes.get(mode, 0) + 1
+    assert all(modes.get(m, 0) >= 3 for m in ("cluster", "tiles", "ranges", "causal cluster", "causal ranges")), modes
