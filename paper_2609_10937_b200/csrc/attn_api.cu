@@ -241,9 +241,25 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
     attn::FwdParams pc = p;
     pc.cluster_k = ck;
     pc.seg_skip = -ck;
-    ATTN_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, to, pc));
-    t_cluster_size = ck;
-    rc = ATTN_OK;
+    // all clusters resident at once, else (or if the cluster launch fails) the same grid as equal ranges
+    static int c_resident[5][kMaxDevices] = {};
+    int dev = 0, n_res = 0;
+    ATTN_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < kMaxDevices) {
+      if (c_resident[ck][dev] == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+        c_resident[ck][dev] = n + 1;
+      }
+      n_res = c_resident[ck][dev] - 1;
+    }
+    if ((long long)n_res * ck >= grid && cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, to, pc) == cudaSuccess) {
+      t_cluster_size = ck;
+      rc = ATTN_OK;
+    } else {
+      (void)cudaGetLastError();
+      rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, true, false>);
+    }
   } else if (p.causal) rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, true, false>);
   else if (eager) rc = launch_eager(attn::attn_fwd_kernel<D, TKV, NQ, false, true>, attn::attn_fwd_kernel<D, TKV, NQ, false, true, true>);
   else rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, false, false>);
