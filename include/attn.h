@@ -187,7 +187,8 @@ int attn_forward_causal(const void *q, const void *k, const void *v, void *o,
  * the closed-form value): n_q (1|2), tile_kv (64|128), kv_stages (2..plan maximum),
  * kv_splits (that many CTAs per Q tile) or ctas (the grid size itself, from 1 up
  * to the number of (Q tile, KV step) units), causal (non-zero selects causal
- * attention).  ATTN_ERR_BAD_TILES if the combination was not compiled or does not
+ * attention; a grid of 2, 3 or 4 CTAs per tile then runs as clusters that share out
+ * each tile's own key steps, any other grid as equal ranges of the unit line).  ATTN_ERR_BAD_TILES if the combination was not compiled or does not
  * fit. */
 int attn_forward_tiles(const void *q, const void *k, const void *v, void *o,
                        int B, int H, int L, int d, const attn_tiles *override_tiles,
