@@ -173,6 +173,18 @@ int attn_forward(const void *q, const void *k, const void *v, void *o,
                  int B, int H, int L, int d, void *cuda_stream);
 
 /*
+ * The same with Lq query rows and Lk keys per head (q, o: [B][H][Lq][d]; k, v: [B][H][Lk][d]):
+ * O = softmax(Q K^T / sqrt(d)) V with every query row attending to all Lk keys.  The paper's
+ * operator is the case Lq == Lk; a block of query rows of a longer sequence is the case
+ * q = Q + r0 * d, Lq = rows in the block (what attn_forward_host uses to overlap copies with
+ * compute).  attn_plan_qk is the derivation for it (tiles from Lq, key steps from Lk).
+ * Errors as attn_forward.
+ */
+int attn_plan_qk(const attn_hw_desc *desc, int B, int H, int Lq, int Lk, int d, attn_tiles *out);
+int attn_forward_qk(const void *q, const void *k, const void *v, void *o,
+                    int B, int H, int Lq, int Lk, int d, void *cuda_stream);
+
+/*
  * Causal fused attention forward: as attn_forward, but row i attends to keys 0..i
  * only -- the scores of later keys are -inf before the softmax (the paper's rule
  * that masked elements are -inf, never zero, Section "Online Softmax", applied to

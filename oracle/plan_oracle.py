@@ -80,7 +80,9 @@ def causal_head_units(q_tiles: int, steps: int, ratio: int) -> int:
     return sum(min(steps, (q + 1) * ratio) for q in range(q_tiles))
 
 
-def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal: bool = False) -> dict:
+def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal: bool = False, Lk: int = 0) -> dict:
+    """L query rows and Lk keys per head (Lk = 0: self-attention, Lk = L)."""
+    Lk = Lk or L
     sub = desc["atom_m"]
     out = dict(feasible=False, binding=BIND_SHAPE)
     if d % desc["atom_k"] or d % desc["atom_n"] or d > desc["atom_n_max"] or min(B, H, L, d) <= 0:
@@ -117,10 +119,10 @@ def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal
             return out
     tile_q = n_q * sub
     tiles = B * H * -(-L // tile_q)
-    steps = -(-L // tile_kv)
+    steps = -(-Lk // tile_kv)
     under = tiles < desc["num_units"]
     ctas = tiles
-    kv_head_bytes = 2 * L * d * desc["elem_bytes"]            # K and V of one head
+    kv_head_bytes = 2 * Lk * d * desc["elem_bytes"]           # K and V of one head
     if causal:
         total = B * H * causal_head_units(-(-L // tile_q), steps, tile_q // tile_kv)
         ctas = max(1, min(total // _MIN_STEPS_PER_SPLIT, desc["num_units"]))

@@ -22,7 +22,7 @@ BIND_NAMES = ("none", "smem", "tmem", "reg", "atom", "shape")
 
 EXPORTED_SYMBOLS = (
     "attn_hw_desc_b200", "attn_hw_desc_query", "attn_plan", "attn_plan_ex", "attn_workspace_bytes",
-    "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_static_scratch", "attn_forward_desc",
+    "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_static_scratch", "attn_forward_desc", "attn_plan_qk", "attn_forward_qk",
     "attn_last_device_status",
     "attn_last_launch_count", "attn_last_cluster_size", "attn_status_string", "attn_last_cuda_error",
     "gemm_plan", "gemm_forward", "softmax_rows_forward", "attn_forward_unfused",
@@ -87,6 +87,8 @@ def lib() -> ctypes.CDLL:
         L.attn_workspace_bytes.restype = ctypes.c_size_t
         L.attn_set_workspace.argtypes = [i32, vp, ctypes.c_size_t]
         L.attn_forward.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+        L.attn_plan_qk.argtypes = [ctypes.POINTER(AttnHwDesc), i32, i32, i32, i32, i32, ctypes.POINTER(AttnTiles)]
+        L.attn_forward_qk.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.attn_forward_tiles.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, ctypes.POINTER(AttnTiles), vp]
         L.attn_forward_simple.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
         L.attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_size_t, vp]
@@ -233,6 +235,35 @@ def forward_desc(desc: AttnHwDesc, q, k, v, o=None, causal=False):
             ensure_workspace(dev, workspace_bytes(t, B, H, L, d))
         _check(lib().attn_forward_desc(ctypes.byref(desc), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
                                        B, H, L, d, 1 if causal else 0, stream), "attn_forward_desc")
+    return o
+
+
+def plan_qk(desc: AttnHwDesc, B: int, H: int, Lq: int, Lk: int, d: int) -> AttnTiles:
+    t = AttnTiles()
+    _check(lib().attn_plan_qk(ctypes.byref(desc), B, H, Lq, Lk, d, ctypes.byref(t)), "attn_plan_qk")
+    return t
+
+
+def forward_qk(q, k, v, o=None):
+    """O = softmax(Q K^T / sqrt(d)) V for q [B, H, Lq, d] and k, v [B, H, Lk, d] (contiguous CUDA bf16)."""
+    import torch
+
+    for name, x in (("q", q), ("k", k), ("v", v)):
+        if x.dtype != torch.bfloat16 or not x.is_cuda or not x.is_contiguous() or x.dim() != 4:
+            raise ValueError(f"{name} must be a contiguous CUDA bfloat16 tensor [B, H, L, d]")
+    B, H, Lq, d = (int(x) for x in q.shape)
+    Lk = int(k.shape[2])
+    if tuple(k.shape) != (B, H, Lk, d) or tuple(v.shape) != (B, H, Lk, d):
+        raise ValueError("k and v must be [B, H, Lk, d] with q's B, H and d")
+    if o is None:
+        o = torch.empty_like(q)
+    dev = q.device.index if q.device.index is not None else torch.cuda.current_device()
+    with torch.cuda.device(dev):
+        t = plan_qk(_device_desc(dev), B, H, Lq, Lk, d)
+        ensure_workspace(dev, workspace_bytes(t, B, H, Lq, d))
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+        _check(lib().attn_forward_qk(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, Lq, Lk, d, stream),
+               "attn_forward_qk")
     return o
 
 

@@ -103,33 +103,35 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
   return a0 < b0 + nb && b0 < a0 + na;
 }
 
-int check_args(const void* q, const void* k, const void* v, const void* o, int B, int H, int L, int d) {
-  if (!q || !k || !v || !o || B <= 0 || H <= 0 || L <= 0 || d <= 0) return ATTN_ERR_INVALID_ARG;
+int check_args(const void* q, const void* k, const void* v, const void* o, int B, int H, int L, int d, int Lk = 0) {
+  if (Lk == 0) Lk = L;
+  if (!q || !k || !v || !o || B <= 0 || H <= 0 || L <= 0 || Lk <= 0 || d <= 0) return ATTN_ERR_INVALID_ARG;
   if (d != 64 && d != 128) return ATTN_ERR_UNSUPPORTED_SHAPE;
   if ((long long)B * H * ((L + 127) / 128) > 0x3FFFFFFFLL) return ATTN_ERR_UNSUPPORTED_SHAPE;  // grid index range
   if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15u) return ATTN_ERR_MISALIGNED;
-  const size_t bytes = (size_t)B * H * L * d * 2;
-  if (overlaps(o, bytes, q, bytes) || overlaps(o, bytes, k, bytes) || overlaps(o, bytes, v, bytes))
+  if ((long long)B * H * ((Lk + 127) / 128) > 0x3FFFFFFFLL) return ATTN_ERR_UNSUPPORTED_SHAPE;
+  const size_t bytes = (size_t)B * H * L * d * 2, kv_bytes = (size_t)B * H * Lk * d * 2;
+  if (overlaps(o, bytes, q, bytes) || overlaps(o, bytes, k, kv_bytes) || overlaps(o, bytes, v, kv_bytes))
     return ATTN_ERR_ALIASING;
   return ATTN_OK;
 }
 
 template <int D, int TKV, int NQ>
-int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int L, const attn_tiles& t,
+int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int Lk, const attn_tiles& t,
                float* ws, cudaStream_t stream) {
   using SM = attn::FwdSmem<D, TKV, NQ>;
   const int BH = B * H;
   CUtensorMap tq, tk, tv, to;
   int rc;
   if ((rc = make_tmap(&tq, q, BH, L, D, attn::kSub)) != ATTN_OK) return rc;
-  if ((rc = make_tmap(&tk, k, BH, L, D, TKV)) != ATTN_OK) return rc;
-  if ((rc = make_tmap(&tv, v, BH, L, D, TKV)) != ATTN_OK) return rc;
+  if ((rc = make_tmap(&tk, k, BH, Lk, D, TKV)) != ATTN_OK) return rc;
+  if ((rc = make_tmap(&tv, v, BH, Lk, D, TKV)) != ATTN_OK) return rc;
   if ((rc = make_tmap(&to, o, BH, L, D, 32)) != ATTN_OK) return rc;    // every warp stores its own 32 rows
 
   attn::FwdParams p;
-  p.L = L;
+  p.L = Lk;                                                       // keys per head (L: query rows per head)
   p.q_tiles = (L + NQ * attn::kSub - 1) / (NQ * attn::kSub);
-  p.n_steps = (L + TKV - 1) / TKV;
+  p.n_steps = (Lk + TKV - 1) / TKV;
   p.tiles = BH * p.q_tiles;
   p.stages = t.kv_stages;
   p.causal = t.causal ? 1 : 0;
@@ -270,9 +272,10 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
 }
 
 int dispatch_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
-                 const attn_tiles& t, float* ws, cudaStream_t s) {
+                 const attn_tiles& t, float* ws, cudaStream_t s, int Lk = 0) {
+  if (Lk == 0) Lk = L;
 #define ATTN_CASE(D_, TKV_, NQ_) \
-  if (d == D_ && t.tile_kv == TKV_ && t.n_q == NQ_) return launch_fwd<D_, TKV_, NQ_>(q, k, v, o, B, H, L, t, ws, s);
+  if (d == D_ && t.tile_kv == TKV_ && t.n_q == NQ_) return launch_fwd<D_, TKV_, NQ_>(q, k, v, o, B, H, L, Lk, t, ws, s);
   ATTN_CASE(128, 128, 2)
   ATTN_CASE(128, 64, 2)
   ATTN_CASE(128, 128, 1)
@@ -289,10 +292,12 @@ int dispatch_fwd(const void* q, const void* k, const void* v, void* o, int B, in
 bool plan_needs_workspace(const attn_tiles& t) { return t.causal != 0 || t.ctas != t.tiles; }
 
 int forward_impl(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d, int causal,
-                 const attn_tiles* ovr, void* cuda_stream, const attn_hw_desc* plan_desc = nullptr) {
+                 const attn_tiles* ovr, void* cuda_stream, const attn_hw_desc* plan_desc = nullptr, int Lk = 0) {
   t_launch_count = 0;
-  int rc = check_args(q, k, v, o, B, H, L, d);
+  if (Lk == 0) Lk = L;                       // keys per head; L is the number of query rows per head
+  int rc = check_args(q, k, v, o, B, H, L, d, Lk);
   if (rc != ATTN_OK) return rc;
+  if (Lk != L && (causal || (ovr && ovr->causal))) return ATTN_ERR_UNSUPPORTED_SHAPE;
   DeviceState* st = nullptr;
   if ((rc = device_state(&st)) != ATTN_OK) return rc;
   if (ovr && ovr->causal) causal = 1;
@@ -309,7 +314,7 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
   }
   const attn_hw_desc& desc = plan_desc ? *plan_desc : st->desc;
   attn_tiles t;
-  if ((rc = attn_plan_ex(&desc, B, H, L, d, causal, &t)) != ATTN_OK) return rc;
+  if ((rc = attn_internal::plan_qk(&desc, B, H, L, Lk, d, causal, &t)) != ATTN_OK) return rc;
   if (!t.feasible) return ATTN_ERR_INFEASIBLE_PLAN;
   if (ovr) {
     if (ovr->n_q > 0) t.n_q = ovr->n_q;
@@ -326,14 +331,14 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
     t.tiles = B * H * ((L + t.tile_q - 1) / t.tile_q);
     // grid: ctas if given, else kv_splits CTAs per Q tile if given, else the planner's occupancy rule
     // re-applied to the overridden tile shape
-    const int steps = (L + t.tile_kv - 1) / t.tile_kv;
+    const int steps = (Lk + t.tile_kv - 1) / t.tile_kv;
     if (ovr->ctas > 0) {
       t.ctas = ovr->ctas;
     } else if (ovr->kv_splits > 0) {
       t.ctas = t.tiles * ovr->kv_splits;
     } else {
       t.ctas = attn_internal::grid_size(desc, B * H, (L + t.tile_q - 1) / t.tile_q, steps, t.tile_q / t.tile_kv, causal,
-                                        2LL * L * d * desc.elem_bytes, 4 * t.n_q, d, (long long)t.kv_stages * stage);
+                                        2LL * Lk * d * desc.elem_bytes, 4 * t.n_q, d, (long long)t.kv_stages * stage);
     }
     t.kv_splits = (t.ctas + t.tiles - 1) / t.tiles;
     if (t.ctas < 1) return ATTN_ERR_BAD_TILES;
@@ -346,7 +351,7 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
     if (!st->ws || st->ws_bytes < need) return ATTN_ERR_NEED_WORKSPACE;
     ws = static_cast<float*>(st->ws);
   }
-  return dispatch_fwd(q, k, v, o, B, H, L, d, t, ws, static_cast<cudaStream_t>(cuda_stream));
+  return dispatch_fwd(q, k, v, o, B, H, L, d, t, ws, static_cast<cudaStream_t>(cuda_stream), Lk);
 }
 
 template <int D, int TKV>
@@ -441,6 +446,12 @@ extern "C" int attn_set_workspace(int device, void* dev_ptr, size_t bytes) {
 extern "C" int attn_forward(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
                             void* cuda_stream) {
   return forward_impl(q, k, v, o, B, H, L, d, 0, nullptr, cuda_stream);
+}
+
+extern "C" int attn_forward_qk(const void* q, const void* k, const void* v, void* o, int B, int H, int Lq, int Lk, int d,
+                               void* cuda_stream) {
+  if (Lk <= 0) return ATTN_ERR_INVALID_ARG;
+  return forward_impl(q, k, v, o, B, H, Lq, d, 0, nullptr, cuda_stream, nullptr, Lk);
 }
 
 extern "C" int attn_forward_causal(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,

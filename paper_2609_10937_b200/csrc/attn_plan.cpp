@@ -183,7 +183,8 @@ void plan_register_machine(const attn_hw_desc& h, int B, int H, int L, int d, at
   t->under_occupied = t->tiles < h.num_units;
 }
 
-void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, int causal, attn_tiles* t) {
+// L query rows and Lk keys per head (Lk == L for self-attention)
+void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int Lk, int d, int causal, attn_tiles* t) {
   const int sub = h.atom_m;  // one tensor-memory lane per Q row
   t->binding_constraint = ATTN_BIND_SHAPE;
   if (d % h.atom_k || d % h.atom_n || d > h.atom_n_max) return;
@@ -232,11 +233,11 @@ void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int d, int ca
   //    Q tiles shared by several CTAs are merged with the merge operator of the online softmax.
   const int tile_q = n_q * sub;
   const int tiles = B * H * ceil_div(L, tile_q);
-  const int steps = ceil_div(L, tile_kv);
+  const int steps = ceil_div(Lk, tile_kv);
   const int under = tiles < h.num_units;
   // (4 n_q groups of 32 rows per tile; a part of one group is 32 rows of d fp32 values plus statistics)
   const int ctas = attn_internal::grid_size(h, B * H, ceil_div(L, tile_q), steps, tile_q / tile_kv, causal,
-                                             2LL * L * d * h.elem_bytes, 4 * n_q, d, (long long)stages * stage);
+                                             2LL * Lk * d * h.elem_bytes, 4 * n_q, d, (long long)stages * stage);
   const int kv_splits = ceil_div(ctas, tiles);
 
   t->feasible = 1;
@@ -296,16 +297,25 @@ extern "C" int attn_plan(const attn_hw_desc* desc, int B, int H, int L, int d, a
 }
 
 extern "C" int attn_plan_ex(const attn_hw_desc* desc, int B, int H, int L, int d, int causal, attn_tiles* out) {
+  return attn_internal::plan_qk(desc, B, H, L, L, d, causal, out);
+}
+
+extern "C" int attn_plan_qk(const attn_hw_desc* desc, int B, int H, int Lq, int Lk, int d, attn_tiles* out) {
+  if (Lk <= 0) return ATTN_ERR_INVALID_ARG;
+  return attn_internal::plan_qk(desc, B, H, Lq, Lk, d, 0, out);
+}
+
+int attn_internal::plan_qk(const attn_hw_desc* desc, int B, int H, int L, int Lk, int d, int causal, attn_tiles* out) {
   if (!desc || !out) return ATTN_ERR_INVALID_ARG;
   if (desc->struct_bytes != (int32_t)sizeof(attn_hw_desc)) return ATTN_ERR_INVALID_ARG;
   std::memset(out, 0, sizeof(*out));
   out->binding_constraint = ATTN_BIND_SHAPE;
-  if (B <= 0 || H <= 0 || L <= 0 || d <= 0) return ATTN_OK;
+  if (B <= 0 || H <= 0 || L <= 0 || Lk <= 0 || d <= 0) return ATTN_OK;
   if (desc->num_units <= 0 || desc->local_mem_bytes <= 0 || desc->atom_m <= 0 || desc->atom_n <= 0 ||
       desc->atom_k <= 0 || desc->elem_bytes <= 0 || desc->simd_width <= 0 || desc->max_regs_per_thread <= 16)
     return ATTN_ERR_INVALID_ARG;
   if (desc->acc_mem_columns > 0)
-    plan_tmem_machine(*desc, B, H, L, d, causal, out);
+    plan_tmem_machine(*desc, B, H, L, Lk, d, causal, out);
   else
     plan_register_machine(*desc, B, H, L, d, out);
   return ATTN_OK;

@@ -15,6 +15,8 @@ namespace attn_internal {
 // Causal (tiles need unequal numbers of steps): always equal ranges of the unit line, one per unit.
 int grid_size(const attn_hw_desc& h, int heads, int q_tiles, int steps, int ratio, int causal,
               long long kv_bytes_per_head, int groups, int part_floats_per_row, long long ring_bytes);
+// The derivation for Lq query rows and Lk keys per head (attn_plan_ex is the case Lq == Lk).
+int plan_qk(const attn_hw_desc* desc, int B, int H, int Lq, int Lk, int d, int causal, attn_tiles* out);
 // Work units (KV steps summed over Q tiles) of one head.
 long long head_units(int q_tiles, int steps, int ratio, int causal);
 }  // namespace attn_internal

@@ -479,3 +479,33 @@ def test_random_shapes_every_grid_mode_agrees_with_an_unsplit_run(env):
         mode = ("causal " if causal else "") + ("cluster" if cl else "tiles" if t.ctas == t.tiles else "ranges")
         modes[mode] = modes.get(mode, 0) + 1
     assert all(modes.get(m, 0) >= 3 for m in ("cluster", "tiles", "ranges", "causal cluster", "causal ranges")), modes
+
+
+@pytest.mark.parametrize("B,H,Lq,Lk,d", [(1, 2, 300, 1408, 128), (2, 3, 1000, 2500, 64), (1, 1, 4096, 16384, 128),
+                                          (1, 2, 1500, 700, 128), (1, 5, 1, 333, 64), (1, 1, 2048, 8192, 128)])
+def test_separate_query_and_key_lengths(env, B, H, Lq, Lk, d):
+    """attn_forward_qk: Lq query rows against Lk keys.  The oracle is the self-attention oracle of length Lk whose
+    first query rows are a block of the Lq rows (every query row attends to all keys, so blocks are independent)."""
+    torch, orc, binding = env
+    rng = np.random.default_rng([B, H, Lq, Lk, d])
+    bits = lambda *shape: synth.f32_to_bf16_bits((rng.standard_normal(shape) * 1.2).astype(np.float32))
+    q, k, v = bits(B * H, Lq, d), bits(B * H, Lk, d), bits(B * H, Lk, d)
+    out = binding.forward_qk(to_cuda_bf16(q).view(B, H, Lq, d), to_cuda_bf16(k).view(B, H, Lk, d),
+                             to_cuda_bf16(v).view(B, H, Lk, d))
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0
+    got = to_host_f64(out).reshape(B * H, Lq, d)
+    blocks = [(r0, min(Lq, r0 + Lk)) for r0 in range(0, Lq, Lk)]
+    if Lq > 2048:                                            # sampled rows of the large case
+        blocks = [(r0, r0 + 32) for r0 in (0, 1000, Lq - 32)]
+    for r0, r1 in blocks:
+        q_pad = np.zeros((B * H, Lk, d), dtype=q.dtype)
+        q_pad[:, : r1 - r0] = q[:, r0:r1]
+        ref = orc.attention_rows(q_pad.reshape(-1), k.reshape(-1), v.reshape(-1), B, H, Lk, d,
+                                 np.arange(r1 - r0, dtype=np.int32))
+        assert_close(got[:, r0:r1], ref, f"qk rows {r0}:{r1}")
+    # the same through the self-attention entry point when the lengths agree
+    if Lq <= 2048:
+        o_self = binding.forward(to_cuda_bf16(k).view(B, H, Lk, d), to_cuda_bf16(k).view(B, H, Lk, d), to_cuda_bf16(v).view(B, H, Lk, d))
+        o_qk = binding.forward_qk(to_cuda_bf16(k).view(B, H, Lk, d), to_cuda_bf16(k).view(B, H, Lk, d), to_cuda_bf16(v).view(B, H, Lk, d))
+        assert torch.equal(o_self.view(torch.int16), o_qk.view(torch.int16))

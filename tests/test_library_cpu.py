@@ -63,6 +63,22 @@ def test_gemm_plan_closed_form(binding):
     assert t.feasible == 0 or t.stages >= 2
 
 
+def test_plan_for_separate_query_and_key_lengths(binding):
+    """attn_plan_qk: Q tiles from the query rows, key steps from the keys; equal to the oracle's restatement, and to
+    attn_plan when the two lengths agree."""
+    desc = binding.hw_desc_b200()
+    dd = _desc_dict(desc)
+    for B, H, Lq, Lk, d in [(1, 1, 4096, 16384, 128), (1, 1, 8192, 16384, 128), (2, 3, 300, 5000, 64), (1, 4, 5000, 300, 128),
+                            (1, 1, 100, 4096, 128), (1, 200, 1000, 2000, 64)]:
+        got = binding.plan_qk(desc, B, H, Lq, Lk, d)
+        ref = po.derive_tiles_tmem_machine(dd, B, H, Lq, d, Lk=Lk)
+        assert got.feasible and (got.tile_q, got.tile_kv, got.n_q, got.kv_stages, got.tiles, got.ctas) == \
+            (ref["tile_q"], ref["tile_kv"], ref["n_q"], ref["kv_stages"], ref["tiles"], ref["ctas"])
+        assert got.tiles == B * H * -(-Lq // got.tile_q)
+    a, b = binding.plan_qk(desc, 1, 8, 2048, 2048, 128), binding.plan(desc, 1, 8, 2048, 128)
+    assert a.as_dict() == b.as_dict()
+
+
 def test_struct_sizes_match_the_header(binding):
     d = binding.hw_desc_b200()
     assert d.struct_bytes == ctypes.sizeof(binding.AttnHwDesc) == 112
