@@ -264,7 +264,7 @@ def run_ours(args):
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes,
                 "ms_per_step": e2e_ms, "steps": e2e_steps,
-                "path": "attn_forward_host: pinned host q,k,v -> device, forward, o -> pinned host, all in the timed region"},
+                "path": "attn_forward_host: pinned host q,k,v -> device, forward (two blocks of query rows, copies overlapped with the kernels), o -> pinned host, all in the timed region"},
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {
             "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": UNIT,

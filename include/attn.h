@@ -243,8 +243,22 @@ int attn_forward_desc(const attn_hw_desc *desc, const void *q, const void *k, co
  * at least 4 * B*H*L*d*2 bytes, 256-byte aligned, that receives the device
  * copies of q, k, v and o.  Queues three host-to-device copies, the forward
  * pass and one device-to-host copy on cuda_stream; does not synchronise.
+ *
+ * One long head (B * H == 1 and L >= 8192) is pipelined: the query rows go as two
+ * blocks, ceil(L / 2) rows rounded up to 256 and the rest, each an independent
+ * attn_forward_qk problem against all L keys, so that the second block's copy in
+ * runs under the first block's kernel and the first block's result leaves under
+ * the second block's kernel.  Those copies are queued on two streams the library
+ * creates on the device's first such call; cuda_stream waits for them before the
+ * call's work counts as done on it, so to the caller the call is still one unit
+ * of work on cuda_stream.  Calls of this form are serialised by a lock while
+ * they queue their work.
+ *
+ * Workspace: attn_forward_host_workspace_bytes (it covers the blocks' plans
+ * as well as the unsplit one; 0 if the shape has no feasible plan).
  * Errors: as attn_forward, plus ATTN_ERR_INVALID_ARG if the scratch is small.
  */
+size_t attn_forward_host_workspace_bytes(const attn_hw_desc *desc, int B, int H, int L, int d);
 int attn_forward_host(const void *q_host, const void *k_host, const void *v_host, void *o_host,
                       int B, int H, int L, int d, void *dev_scratch, size_t dev_scratch_bytes,
                       void *cuda_stream);

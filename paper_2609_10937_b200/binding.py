@@ -22,7 +22,7 @@ BIND_NAMES = ("none", "smem", "tmem", "reg", "atom", "shape")
 
 EXPORTED_SYMBOLS = (
     "attn_hw_desc_b200", "attn_hw_desc_query", "attn_plan", "attn_plan_ex", "attn_workspace_bytes",
-    "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_static_scratch", "attn_forward_desc", "attn_plan_qk", "attn_forward_qk",
+    "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_host_workspace_bytes", "attn_forward_static_scratch", "attn_forward_desc", "attn_plan_qk", "attn_forward_qk",
     "attn_last_device_status",
     "attn_last_launch_count", "attn_last_cluster_size", "attn_status_string", "attn_last_cuda_error",
     "gemm_plan", "gemm_forward", "softmax_rows_forward", "attn_forward_unfused",
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
         L.attn_forward_qk.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.attn_forward_tiles.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, ctypes.POINTER(AttnTiles), vp]
         L.attn_forward_simple.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
+        L.attn_forward_host_workspace_bytes.argtypes = [ctypes.POINTER(AttnHwDesc), i32, i32, i32, i32]
+        L.attn_forward_host_workspace_bytes.restype = ctypes.c_size_t
         L.attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_size_t, vp]
         L.attn_forward_static_scratch.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
         L.attn_forward_desc.argtypes = [ctypes.POINTER(AttnHwDesc), vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
@@ -320,9 +322,8 @@ def forward_host(q_host, k_host, v_host, o_host, dev_scratch):
     dev = dev_scratch.device.index
     stream = torch.cuda.current_stream(dev_scratch.device).cuda_stream
     with torch.cuda.device(dev):
-        t = plan(_device_desc(dev), B, H, L, d)
-        if t.feasible:
-            ensure_workspace(dev, workspace_bytes(t, B, H, L, d))
+        desc = _device_desc(dev)
+        ensure_workspace(dev, int(lib().attn_forward_host_workspace_bytes(ctypes.byref(desc), B, H, L, d)))
         _check(lib().attn_forward_host(q_host.data_ptr(), k_host.data_ptr(), v_host.data_ptr(), o_host.data_ptr(),
                                        B, H, L, d, dev_scratch.data_ptr(), dev_scratch.numel(), stream),
                "attn_forward_host")

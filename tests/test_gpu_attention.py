@@ -393,6 +393,32 @@ def test_host_buffer_entry_point(env):
     assert_close(got.reshape(2, 512, 128), ref, "host entry")
 
 
+@pytest.mark.parametrize("L,d", [(8192, 128), (8192 + 72, 64), (16384 + 8, 128)])
+def test_host_buffer_entry_point_pipelined_long_head(env, L, d):
+    """One long head goes through the host entry point as blocks of query rows whose copies overlap the kernels:
+    the result must match the oracle on sampled rows of every block and on the rows either side of each block
+    boundary, on two calls in a row (the streams and events are reused)."""
+    torch, orc, binding = env
+    case = _case("hostpipe", 1, 1, L, d)
+    q, k, v = synth.make_qkv(case, seed=5)
+    hq, hk, hv = (torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory() for x in (q, k, v))
+    scratch = torch.empty(4 * hq.numel() * 2, dtype=torch.uint8, device="cuda")
+    blocks = 2
+    per = (-(-L // blocks) + 255) // 256 * 256
+    edges = [e for i in range(1, blocks) for e in (i * per - 1, i * per) if e < L]
+    rows = np.unique(np.concatenate([synth.sample_rows(L)[::max(1, L // 2048)], edges, [0, L - 1]])).astype(np.int32)
+    ref = orc.attention_rows(q, k, v, 1, 1, L, d, rows)
+    for _ in range(2):
+        ho = torch.full_like(hq, float("nan")).pin_memory()
+        binding.forward_host(hq, hk, hv, ho, scratch)
+        torch.cuda.synchronize()
+        assert binding.last_device_status()[0] == 0
+        got = (ho.view(torch.int16).numpy().view(np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+        assert np.isfinite(got).all()
+        assert_close(got.reshape(1, L, d)[:, rows], ref, "pipelined host entry")
+        scratch.zero_()
+
+
 def test_shared_tile_counters_bound_the_grid(env):
     """Grids whose CTAs share Q tiles keep two counters per warp of every (CTA, sub-tile) in the 64 KB counter block:
     more than 1024 such CTAs are refused, not run."""

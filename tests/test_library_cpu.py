@@ -188,6 +188,25 @@ def test_forward_argument_errors_come_before_any_cuda_call(binding):
     assert binding.status_string(12345) == "unknown status"
 
 
+def test_host_entry_workspace_covers_both_query_blocks(binding):
+    """One long head runs through the host entry point as blocks of query rows: its workspace figure is the
+    largest of the unsplit plan's and the blocks' plans; other shapes need what attn_forward needs."""
+    L = binding.lib()
+    desc = binding.hw_desc_b200()
+    need = lambda B, H, n, d: int(L.attn_forward_host_workspace_bytes(ctypes.byref(desc), B, H, n, d))
+    for (B, H, n, d) in [(1, 1, 16384, 128), (1, 1, 8192 + 72, 64), (1, 1, 8192, 128), (1, 1, 32768 + 8, 128)]:
+        blocks = 2
+        per = (-(-n // blocks) + 255) // 256 * 256
+        sizes = {min(per, n - i * per) for i in range(blocks) if n - i * per > 0}
+        want = binding.workspace_bytes(binding.plan(desc, B, H, n, d), B, H, n, d)
+        for r in sizes:
+            want = max(want, binding.workspace_bytes(binding.plan_qk(desc, B, H, r, n, d), B, H, r, d))
+        assert need(B, H, n, d) == want > 0
+    for (B, H, n, d) in [(1, 2, 16384, 128), (1, 1, 4096, 128), (4, 32, 4096, 128)]:
+        assert need(B, H, n, d) == binding.workspace_bytes(binding.plan(desc, B, H, n, d), B, H, n, d)
+    assert need(1, 1, 128, 96) == 0
+
+
 def test_product_does_not_reach_the_oracle():
     """The product package must not import, read or execute anything under oracle/."""
     pkg = os.path.join(ROOT, "paper_2609_10937_b200")
