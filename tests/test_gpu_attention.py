@@ -535,3 +535,48 @@ def test_separate_query_and_key_lengths(env, B, H, Lq, Lk, d):
         o_self = binding.forward(to_cuda_bf16(k).view(B, H, Lk, d), to_cuda_bf16(k).view(B, H, Lk, d), to_cuda_bf16(v).view(B, H, Lk, d))
         o_qk = binding.forward_qk(to_cuda_bf16(k).view(B, H, Lk, d), to_cuda_bf16(k).view(B, H, Lk, d), to_cuda_bf16(v).view(B, H, Lk, d))
         assert torch.equal(o_self.view(torch.int16), o_qk.view(torch.int16))
+
+
+@pytest.mark.parametrize("L,d,heads", [(512, 128, 33024), (520, 64, 64640)])
+def test_tensors_beyond_two_to_the_31_elements(env, L, d, heads):
+    """Each of Q, K, V, O holds more than 2^31 elements (4.3 GB): byte offsets and element indices past the 32-bit range.
+    64 seeded heads are laid out `heads / 64` times one after the other (a device-side copy of the same host data).
+    Every element of every group is compared with the oracle's result for those 64 heads (on the device, max-abs bar),
+    the first and the last group -- the one past the 2^31st element -- with both bars on the host, and all but the few
+    heads whose tiles straddle a boundary between two CTAs' ranges (computed in two pieces and merged) must reproduce the
+    first group's bits exactly."""
+    torch, orc, binding = env
+    base = 64
+    assert heads % base == 0 and heads * L * d > 2 ** 31
+    free, _ = torch.cuda.mem_get_info()
+    if free < 5 * heads * L * d * 2:
+        pytest.skip("not enough free device memory for four 4.3 GB tensors")
+    case = _case("big", 1, base, L, d)
+    q, k, v = synth.make_qkv(case, seed=6)
+    groups = heads // base
+    tq, tk, tv = (to_cuda_bf16(x).reshape(1, base, L, d).repeat(1, groups, 1, 1).contiguous() for x in (q, k, v))
+    assert tq.numel() > 2 ** 31
+    out = torch.full_like(tq, float("nan"))
+    binding.forward(tq, tk, tv, out)
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0
+    rows = np.arange(L, dtype=np.int32)
+    ref = orc.attention_rows(q, k, v, 1, base, L, d, rows)
+    ref_dev = torch.from_numpy(ref.reshape(base, L, d)).cuda()
+    bits = out.view(torch.int16).reshape(groups, base, L, d)
+    grouped = out.reshape(groups, base, L, d)
+    differing_heads, worst = 0, 0.0
+    for g0 in range(0, groups, 16):
+        blk = grouped[g0:g0 + 16]
+        assert bool(torch.isfinite(blk).all()), f"non-finite output in groups {g0}.."
+        worst = max(worst, float((blk.double() - ref_dev).abs().max()))
+        differing_heads += int((bits[g0:g0 + 16] != bits[:1]).flatten(2).any(dim=2).sum())
+    print(f"L={L} d={d} heads={heads}: max_abs over all groups {worst:.3e}, heads differing bitwise {differing_heads}")
+    assert worst <= 1e-2, f"max_abs {worst:.3e} over all groups"
+    plan = binding.plan(binding.hw_desc_query(torch.cuda.current_device()), 1, heads, L, d)
+    assert differing_heads <= plan.ctas, f"{differing_heads} heads differ from their copy in the first group"
+    for g in (0, groups - 1):
+        got = to_host_f64(out.reshape(groups, base, L, d)[g]).reshape(base, L, d)
+        assert_close(got, ref, f"head group {g}")
+    del tq, tk, tv, out, bits
+    torch.cuda.empty_cache()
