@@ -397,7 +397,8 @@ def test_host_buffer_entry_point(env):
 def test_host_buffer_entry_point_pipelined_long_head(env, L, d):
     """One long head goes through the host entry point as blocks of query rows whose copies overlap the kernels:
     the result must match the oracle on sampled rows of every block and on the rows either side of each block
-    boundary, on two calls in a row (the streams and events are reused)."""
+    boundary, on three calls in a row (the streams and events are reused), two of them on a stream of the caller's
+    that alone is waited for."""
     torch, orc, binding = env
     case = _case("hostpipe", 1, 1, L, d)
     q, k, v = synth.make_qkv(case, seed=5)
@@ -408,10 +409,18 @@ def test_host_buffer_entry_point_pipelined_long_head(env, L, d):
     edges = [e for i in range(1, blocks) for e in (i * per - 1, i * per) if e < L]
     rows = np.unique(np.concatenate([synth.sample_rows(L)[::max(1, L // 2048)], edges, [0, L - 1]])).astype(np.int32)
     ref = orc.attention_rows(q, k, v, 1, 1, L, d, rows)
-    for _ in range(2):
+    side = torch.cuda.Stream()
+    for it in range(3):
         ho = torch.full_like(hq, float("nan")).pin_memory()
-        binding.forward_host(hq, hk, hv, ho, scratch)
-        torch.cuda.synchronize()
+        if it == 0:
+            binding.forward_host(hq, hk, hv, ho, scratch)
+            torch.cuda.synchronize()
+        else:
+            # the caller waits for its own stream only: the library's copy streams must have been joined into it
+            torch.cuda.synchronize()
+            with torch.cuda.stream(side):
+                binding.forward_host(hq, hk, hv, ho, scratch)
+            side.synchronize()
         assert binding.last_device_status()[0] == 0
         got = (ho.view(torch.int16).numpy().view(np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
         assert np.isfinite(got).all()
