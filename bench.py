@@ -32,6 +32,8 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 
 WORKLOAD = "cfg3"
+WORKLOAD_TEXT = ("cfg3: attention fwd B=1,H=1,L=16384,d=128, non-causal, bf16 N(0,1), seed 0, scale 1/sqrt(d), "
+            "fp32 accumulate (one such problem per GPU)")
 METRIC = "fused_attention_fwd_tflops_L16384_d128"
 UNIT = "TFLOP/s"
 L2_FLUSH_BYTES = 256 << 20
@@ -160,7 +162,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "cfg3: attention fwd B=1,H=1,L=16384,d=128, non-causal, bf16 inputs N(0,1), seed 0"},
+        "config": {"workload": WORKLOAD_TEXT, "arithmetic": "the oracle's: fp64 over the same bf16 inputs"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -253,8 +255,7 @@ def run_ours(args):
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {
-            "workload": "cfg3: attention fwd B=1,H=1,L=16384,d=128, non-causal, bf16 N(0,1), scale 1/sqrt(d), "
-                        "fp32 accumulate (one such problem per GPU)",
+            "workload": WORKLOAD_TEXT,
             "tiles": {"tile_q": plan.tile_q, "tile_kv": plan.tile_kv, "kv_stages": plan.kv_stages,
                       "kv_splits": plan.kv_splits, "ctas": plan.ctas, "closed_form_default": True},
             "l2": f"{L2_FLUSH_BYTES >> 20} MiB device write between timed steps (outside the step's events)",
