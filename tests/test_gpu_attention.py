@@ -589,3 +589,16 @@ def test_tensors_beyond_two_to_the_31_elements(env, L, d, heads):
         assert_close(got, ref, f"head group {g}")
     del tq, tk, tv, out, bits
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("L,d", [(131072 + 40, 128), (262144, 64)])
+def test_very_long_single_head(env, L, d):
+    """One head of 131,112 (ragged) and 262,144 keys: 1025 and 2048 key steps per Q tile, row sums of that many terms
+    carried through as many rescales; a stratified sample of rows against the oracle plus the whole-output properties."""
+    torch, orc, binding = env
+    case = _case("long", 1, 1, L, d)
+    rows = synth.sample_rows(L)[:: max(1, L // 16384)]
+    rows = np.unique(np.concatenate([rows, [0, 127, 128, L - 129, L - 1]])).astype(np.int32)
+    assert len(rows) >= 256
+    _run_and_compare(env, case, binding.forward, rows=rows)
+    _run_and_compare(env, case, lambda q, k, v: binding.forward(q, k, v, causal=True), rows=rows[::4], causal=True)
