@@ -428,6 +428,41 @@ def test_host_buffer_entry_point_pipelined_long_head(env, L, d):
         scratch.zero_()
 
 
+def test_missing_or_small_workspace_is_reported_and_nothing_runs(env):
+    """A plan that shares Q tiles between CTAs needs the caller's workspace: with none registered, or one smaller than
+    attn_workspace_bytes, the call returns NEED_WORKSPACE before any launch and the output is untouched."""
+    import ctypes
+
+    torch, _, binding = env
+    lib = binding.lib()
+    dev = torch.cuda.current_device()
+    B, H, L, d = 1, 1, 4096, 128
+    case = _case("needws", B, H, L, d)
+    tq, tk, tv = (to_cuda_bf16(x) for x in synth.make_qkv(case, seed=7))
+    o = torch.full_like(tq, float("nan"))
+    need = binding.workspace_bytes(binding.plan(binding.hw_desc_query(dev), B, H, L, d), B, H, L, d)
+    assert need > 65536
+    binding.ensure_workspace(dev, need)                  # the buffer the binding keeps registered; restored below
+    kept = binding._workspaces[dev]
+    stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    call = lambda: lib.attn_forward(tq.data_ptr(), tk.data_ptr(), tv.data_ptr(), o.data_ptr(), B, H, L, d, stream)
+    small = torch.empty(need - 16, dtype=torch.uint8, device="cuda")
+    try:
+        assert lib.attn_set_workspace(dev, None, 0) == 0
+        assert call() == binding.ERR_NEED_WORKSPACE
+        assert lib.attn_set_workspace(dev, small.data_ptr(), small.numel()) == 0
+        assert call() == binding.ERR_NEED_WORKSPACE
+        assert binding.lib().attn_last_launch_count() == 0
+        torch.cuda.synchronize()
+        assert bool(torch.isnan(o).all())
+    finally:
+        assert lib.attn_set_workspace(dev, kept.data_ptr(), kept.numel()) == 0
+    assert call() == 0
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0 and bool(torch.isfinite(o).all())
+    assert "workspace" in binding.status_string(binding.ERR_NEED_WORKSPACE)
+
+
 def test_shared_tile_counters_bound_the_grid(env):
     """Grids whose CTAs share Q tiles keep two counters per warp of every (CTA, sub-tile) in the 64 KB counter block:
     more than 1024 such CTAs are refused, not run."""
