@@ -302,6 +302,20 @@ int attn_forward_static_scratch(const void *q, const void *k, const void *v, voi
  * a spare word -- or ATTN_OK.  Clears the record. */
 int attn_last_device_status(void *cuda_stream, uint32_t *detail);
 
+/*
+ * Self-test of the bounded device-side waits (no counterpart in the paper: part of the error
+ * behaviour of this boundary).  Every wait inside the kernels -- on a barrier, a flag, a peer CTA --
+ * gives up after a fixed cycle count (about half a second), records where, and lets the kernel
+ * return, so that a lost signal shows as ATTN_ERR_DEVICE_TIMEOUT from attn_last_device_status
+ * instead of a hung GPU.  This call queues, on cuda_stream, one warp that waits with that same
+ * routine on a barrier nothing ever arrives at; it ends by itself when the limit runs out.
+ * Afterwards attn_last_device_status reports ATTN_ERR_DEVICE_TIMEOUT with detail[1] =
+ * role 5 << 24 | barrier 10 << 16 | ATTN_SELFTEST_STEP, and the context stays usable.
+ * Errors: WRONG_ARCH, CUDA.
+ */
+#define ATTN_SELFTEST_STEP 0x7E57
+int attn_selftest_wait_expiry(void *cuda_stream);
+
 /* Number of kernels the last attn_forward* call on this thread launched. */
 int attn_last_launch_count(void);
 

@@ -23,7 +23,7 @@ BIND_NAMES = ("none", "smem", "tmem", "reg", "atom", "shape")
 EXPORTED_SYMBOLS = (
     "attn_hw_desc_b200", "attn_hw_desc_query", "attn_plan", "attn_plan_ex", "attn_workspace_bytes",
     "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_host_workspace_bytes", "attn_forward_static_scratch", "attn_forward_desc", "attn_plan_qk", "attn_forward_qk",
-    "attn_last_device_status",
+    "attn_last_device_status", "attn_selftest_wait_expiry",
     "attn_last_launch_count", "attn_last_cluster_size", "attn_status_string", "attn_last_cuda_error",
     "gemm_plan", "gemm_forward", "softmax_rows_forward", "attn_forward_unfused",
 )
@@ -97,6 +97,7 @@ def lib() -> ctypes.CDLL:
         L.attn_forward_static_scratch.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
         L.attn_forward_desc.argtypes = [ctypes.POINTER(AttnHwDesc), vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.attn_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+        L.attn_selftest_wait_expiry.argtypes = [vp]
         L.attn_last_launch_count.argtypes = []
         L.attn_last_cluster_size.argtypes = []
         L.attn_status_string.argtypes = [i32]

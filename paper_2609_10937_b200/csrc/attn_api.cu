@@ -662,6 +662,32 @@ extern "C" int attn_forward_static_scratch(const void* q, const void* k, const v
   return dispatch_fwd(q, k, v, o, B, H, L, d, t, static_cast<float*>(scratch), stream);
 }
 
+namespace {
+// One warp waits, with the kernels' bounded wait, on a barrier that nothing arrives at: the wait runs out
+// after its cycle limit (about half a second), records the expiry and the kernel returns by itself.
+__global__ void wait_expiry_selftest_kernel() {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    sm100::mbar_init(sm100::smem_u32(&bar), 1);
+    sm100::fence_mbar_init();
+  }
+  __syncthreads();
+  (void)attn::wait_bar_warp(sm100::smem_u32(&bar), 0, &abort_flag,
+                            attn::wait_info(attn::kRoleSimple, attn::kBarSync, ATTN_SELFTEST_STEP));
+}
+}  // namespace
+
+extern "C" int attn_selftest_wait_expiry(void* cuda_stream) {
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);
+  if (rc != ATTN_OK) return rc;
+  wait_expiry_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>();
+  ATTN_CUDA_TRY(cudaGetLastError());
+  return ATTN_OK;
+}
+
 extern "C" int attn_last_device_status(void* cuda_stream, uint32_t* detail) {
   ATTN_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
   unsigned int h[4] = {0, 0, 0, 0};

@@ -463,6 +463,29 @@ def test_missing_or_small_workspace_is_reported_and_nothing_runs(env):
     assert "workspace" in binding.status_string(binding.ERR_NEED_WORKSPACE)
 
 
+def test_bounded_wait_expiry_is_reported_and_the_context_survives(env):
+    """The library's self-test queues one warp that waits, with the kernels' bounded wait, on a barrier nothing arrives
+    at.  The wait must run out by itself (about half a second), the expiry must be reported once with the place that
+    gave up, and the device must go on computing correct results afterwards."""
+    import ctypes
+    import time
+
+    torch, _, binding = env
+    lib = binding.lib()
+    assert binding.last_device_status()[0] == 0
+    stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    t0 = time.perf_counter()
+    assert lib.attn_selftest_wait_expiry(stream) == 0
+    code, detail = binding.last_device_status()              # synchronises the stream
+    waited = time.perf_counter() - t0
+    assert code == binding.ERR_DEVICE_TIMEOUT
+    assert detail[0] == 1 and detail[1] == (5 << 24) | (10 << 16) | 0x7E57 and detail[2] == 0
+    assert 0.2 < waited < 5.0, f"the wait took {waited:.2f} s"
+    assert binding.last_device_status()[0] == 0              # reported once, then cleared
+    _run_and_compare(env, _case("after_expiry", 1, 2, 512, 128), binding.forward)
+    _run_and_compare(env, _case("after_expiry_split", 1, 1, 4096, 128), binding.forward, rows=synth.sample_rows(4096))
+
+
 def test_shared_tile_counters_bound_the_grid(env):
     """Grids whose CTAs share Q tiles keep two counters per warp of every (CTA, sub-tile) in the 64 KB counter block:
     more than 1024 such CTAs are refused, not run."""
