@@ -12,8 +12,9 @@
  *   - Plain C types only; no exceptions cross the boundary; every function
  *     returns an attn_status (0 = success, negative = error) unless noted.
  *   - q, k, v, o are DEVICE pointers to contiguous [B][H][L][d] bf16 arrays
- *     (d fastest), 16-byte aligned.  Non-causal, no mask, scale 1/sqrt(d),
- *     fp32 accumulation, bf16 (round-to-nearest-even) output.
+ *     (d fastest), 16-byte aligned.  Scale 1/sqrt(d), fp32 accumulation, bf16
+ *     (round-to-nearest-even) output.  attn_forward is non-causal (the paper's
+ *     operator); attn_forward_causal applies a triangular -inf mask.
  *   - The caller owns every buffer, including the workspace.  The library
  *     allocates no device memory and keeps no reference to q/k/v/o after a
  *     call returns.  attn_forward* are asynchronous on `cuda_stream`
@@ -43,7 +44,7 @@ typedef enum attn_status {
   ATTN_ERR_ALIASING = -4,          /* o overlaps q, k or v                                */
   ATTN_ERR_INFEASIBLE_PLAN = -5,   /* no tile choice fits; see binding_constraint         */
   ATTN_ERR_WRONG_ARCH = -6,        /* current device is not compute capability 10.x       */
-  ATTN_ERR_NEED_WORKSPACE = -7,    /* plan splits the keys but no workspace was supplied  */
+  ATTN_ERR_NEED_WORKSPACE = -7,    /* CTAs share Q tiles but no (large enough) workspace  */
   ATTN_ERR_CUDA = -8,              /* a CUDA runtime/driver call failed                   */
   ATTN_ERR_DEVICE_TIMEOUT = -9,    /* a bounded device-side wait expired                  */
   ATTN_ERR_BAD_TILES = -10,        /* tile override not among the compiled variants       */
@@ -67,6 +68,14 @@ typedef enum attn_binding {
  * acc_mem_columns == 0 describes a machine whose accumulators live in vector
  * registers (the paper's CDNA targets); > 0 describes tensor memory (B200).
  * Caller-owned plain data; set struct_bytes = sizeof(attn_hw_desc).
+ *
+ * The ovh_* fields are hardware facts in the same sense as the capacities: what
+ * the start and the end of a CTA's work cost on this machine under each way of
+ * sharing out the key axis, measured once per target, in units of one KV step of
+ * the kernel (the occupancy step of the derivation compares critical paths in
+ * KV steps).  Changing them re-runs the occupancy step like changing a capacity
+ * re-runs the tile step.  hbm_gbps and peak_tflops feed the predicted time and
+ * bound that attn_plan reports (attn_tiles.predicted_us, .bound).
  */
 typedef struct attn_hw_desc {
   int32_t struct_bytes;
@@ -85,9 +94,17 @@ typedef struct attn_hw_desc {
   int32_t cache_bytes;         /* last-level cache shared by all units (L2); 0 if not modelled */
   int32_t max_clusters[8];     /* [k-1]: clusters of k CTAs (one CTA per unit, distributed shared    */
                                /* memory between them) that can be resident at once; 0: none        */
-  double hbm_gbps;             /* sustained HBM bandwidth, GB/s                       */
-  double peak_tflops;          /* dense tensor peak for the operand type, TFLOP/s     */
-  double sm_clock_mhz;         /* maximum SM clock                                    */
+  /* cost of a CTA's start and end, in KV steps (B200 values in attn_hw_desc_b200) */
+  int32_t ovh_whole_tile;      /* one CTA per whole Q tile, nothing to merge                         */
+  int32_t ovh_cluster;         /* k CTAs per tile as one cluster, partials through distributed SMEM  */
+  int32_t ovh_workspace;       /* k CTAs per tile, partials through the workspace (plus k / 2)       */
+  int32_t ovh_ranges;          /* equal ranges of the (tile, step) line, fewer tiles than units      */
+  int32_t ovh_persistent;      /* one persistent CTA per unit on an equal range, more tiles than units */
+  int32_t ovh_tile_change;     /* a persistent CTA moving on to its next Q tile                      */
+  int32_t ovh_causal_ranges;   /* causal, equal ranges: many short pieces per CTA                    */
+  int32_t ovh_causal_cluster;  /* causal, k CTAs per tile as one cluster                             */
+  double hbm_gbps;             /* HBM bandwidth, GB/s (nominal, or measured by the caller)           */
+  double peak_tflops;          /* dense tensor peak for the operand type, TFLOP/s                    */
 } attn_hw_desc;
 
 /* Result of the closed-form derivation.  Caller-owned plain data. */
@@ -111,10 +128,16 @@ typedef struct attn_tiles {
   int32_t binding_constraint; /* attn_binding                                           */
   int32_t under_occupied; /* 1 if tiles < num_units (occupancy check of the derivation) */
   int32_t causal;         /* 1 if planned for causal attention (row i sees keys 0..i)   */
+  int32_t cost_steps;     /* what the occupancy step minimised: KV steps on the longest CTA's path plus the
+                             ovh_* cost of the chosen way of sharing out the key axis                      */
+  int32_t bound;          /* 0: tensor time exceeds HBM time (predicted), 1: the reverse                   */
+  float predicted_us;     /* max(cost_steps * FLOPs of one KV step / (peak_tflops / num_units),
+                             compulsory bytes / hbm_gbps); 0 if the descriptor gives no peaks            */
 } attn_tiles;
 
 /* Built-in descriptor of one B200 (148 SMs, 227 KB SMEM opt-in, 64 K registers,
- * 128 x 512 tensor memory, tcgen05 kind::f16 atom 128 x N x 16).  Host only. */
+ * 128 x 512 tensor memory, tcgen05 kind::f16 atom 128 x N x 16; ovh_* = 2, 5, 8, 12,
+ * 6, 1, 15, 6 KV steps as measured on B200; 7.7 TB/s and 2250 TFLOP/s nominal).  Host only. */
 int attn_hw_desc_b200(attn_hw_desc *out);
 
 /* Descriptor of CUDA device `device`, from cudaDeviceGetAttribute plus the
@@ -129,12 +152,18 @@ int attn_hw_desc_query(int device, attn_hw_desc *out);
  * is infeasible (out->feasible == 0 and out->binding_constraint says why);
  * returns ATTN_ERR_INVALID_ARG for null pointers or a bad struct_bytes.
  * Occupancy step with fewer Q tiles than units (costs in KV steps per CTA, the
- * cheapest wins, ties to the earlier): one CTA per tile, steps + 2; k CTAs per
- * tile along the keys as one thread-block cluster, ceil(steps / k) + 5 (2 <= k <= 8,
- * tiles * k <= num_units, steps / k >= 2, max_clusters[k-1] >= tiles, landing areas
- * fit); k CTAs per tile through the workspace, ceil(steps / k) + 8 + k / 2 with
+ * cheapest wins, ties to the earlier; the result is attn_tiles.cost_steps): one CTA
+ * per tile, steps + ovh_whole_tile; k CTAs per tile along the keys as one
+ * thread-block cluster, ceil(steps / k) + ovh_cluster (2 <= k <= 8, tiles * k <=
+ * num_units, steps / k >= 2, max_clusters[k-1] >= tiles, landing areas fit); k CTAs
+ * per tile through the workspace, ceil(steps / k) + ovh_workspace + k / 2 with
  * k = min(num_units / tiles, steps / 4); equal ranges of the (tile, step) line for
- * G = min(num_units, tiles * steps / 4) CTAs, ceil(tiles * steps / G) + 12.
+ * G = min(num_units, tiles * steps / 4) CTAs, ceil(tiles * steps / G) + ovh_ranges.
+ * With at least as many tiles as units: one CTA per tile in whole waves,
+ * ceil(tiles / units) * (steps + ovh_whole_tile), or -- only if the K and V of the
+ * heads then in flight fit two thirds of cache_bytes -- one persistent CTA per unit
+ * on an equal range, ceil(tiles * steps / units) + ovh_persistent +
+ * ceil(tiles / units) * ovh_tile_change.
  */
 int attn_plan(const attn_hw_desc *desc, int B, int H, int L, int d, attn_tiles *out);
 
@@ -143,8 +172,9 @@ int attn_plan(const attn_hw_desc *desc, int B, int H, int L, int d, attn_tiles *
  * step always deals the (Q tile, KV step) units out in equal ranges, one per unit.
  * Exception: k = 2..4 CTAs per tile as one cluster, each with a share of the tile's own key
  * steps, if tiles * k <= num_units, max_clusters[k-1] >= tiles, ceil(steps / k) >= 2, the
- * landing areas fit and ceil(steps / k) + 6 < ceil((units + 3 * tiles) / G) + 15 (few short
- * tiles: a CTA then has one piece instead of many short ones; ctas == k * tiles).
+ * landing areas fit and ceil(steps / k) + ovh_causal_cluster < ceil((units + 3 * tiles) / G) +
+ * ovh_causal_ranges (few short tiles: a CTA then has one piece instead of many short ones;
+ * ctas == k * tiles).
  * (The paper treats non-causal attention only; this applies its -inf masking rule,
  * Section "Online Softmax", to a triangular mask.) */
 int attn_plan_ex(const attn_hw_desc *desc, int B, int H, int L, int d, int causal, attn_tiles *out);
@@ -159,18 +189,49 @@ size_t attn_workspace_bytes(const attn_tiles *tiles, int B, int H, int L, int d)
  * NULL, 0 to clear) and zeroes its first 64 KB (the arrival counters) with a
  * synchronous cudaMemset on the current device, which must be `device`.  The
  * buffer must stay valid until replaced; concurrent attn_forward calls on
- * different streams of one device must not share it. */
+ * different streams of one device must not share it (use attn_forward_ws with a
+ * workspace per stream for that).  After ATTN_ERR_DEVICE_TIMEOUT the counters may
+ * be non-zero: attn_last_device_status clears them when it reports the timeout, so
+ * poll it before the workspace is used again. */
 int attn_set_workspace(int device, void *dev_ptr, size_t bytes);
 
 /*
  * Fused attention forward (Algorithm 1) with the closed-form default tiles for
  * the current device.  Asynchronous on cuda_stream.  Errors: INVALID_ARG,
  * UNSUPPORTED_SHAPE, MISALIGNED, ALIASING, WRONG_ARCH, INFEASIBLE_PLAN,
- * NEED_WORKSPACE (plan has kv_splits > 1 and the registered workspace is
- * smaller than attn_workspace_bytes), CUDA.
+ * NEED_WORKSPACE (the plan's CTAs share Q tiles -- ctas != tiles, e.g. a key split
+ * or equal ranges of the (tile, step) line; kv_splits may still be 1 -- and the
+ * registered workspace is smaller than attn_workspace_bytes), CUDA.
  */
 int attn_forward(const void *q, const void *k, const void *v, void *o,
                  int B, int H, int L, int d, void *cuda_stream);
+
+/*
+ * attn_forward (causal == 0) or attn_forward_causal (causal != 0) with the workspace and the status words of
+ * THIS call instead of the device-wide ones: what two streams of one device need to run plans that share Q
+ * tiles at the same time, and what attributes an expired device-side wait to the launch it happened in.
+ *   workspace        DEVICE buffer, 16-byte aligned, at least attn_workspace_bytes for the plan (may be NULL
+ *                    with workspace_bytes 0 when that is 0); caller-owned; must not be used by another call
+ *                    that may run at the same time.  Its first 64 KB (arrival counters) must be zero before
+ *                    the first launch that uses it -- attn_workspace_init queues that clearing on a stream --
+ *                    and every launch that ends normally leaves them zero.
+ *   status_dev       four DEVICE words, 16-byte aligned, zero before first use (attn_workspace_init clears
+ *                    them too), or NULL: then an expired wait is recorded in the device-wide record that
+ *                    attn_last_device_status reads.  attn_status_read(status_dev, workspace, stream, detail)
+ *                    synchronises the stream, returns ATTN_ERR_DEVICE_TIMEOUT with the four words in detail
+ *                    (as attn_last_device_status) if a wait expired, clears the words and -- an aborted
+ *                    launch may leave counters non-zero -- the workspace's counters; ATTN_OK otherwise.
+ * A uniform key split that cannot run as thread-block clusters is merged here by the last CTA of a tile to finish
+ * (never by fixed roles, whose merging warps wait for CTAs that a second kernel on the device could keep from
+ * starting); the output bits are the same.
+ * The paper's operator and merge (Sections "Fused Attention", "Online Softmax") are unchanged; this is the
+ * ownership rule of the boundary made explicit per call.  Errors as attn_forward; NEED_WORKSPACE if the
+ * buffer is too small.
+ */
+int attn_workspace_init(void *workspace, size_t workspace_bytes, uint32_t *status_dev, void *cuda_stream);
+int attn_forward_ws(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int d, int causal,
+                    void *workspace, size_t workspace_bytes, uint32_t *status_dev, void *cuda_stream);
+int attn_status_read(uint32_t *status_dev, void *workspace, void *cuda_stream, uint32_t *detail);
 
 /*
  * The same with Lq query rows and Lk keys per head (q, o: [B][H][Lq][d]; k, v: [B][H][Lk][d]):
@@ -198,7 +259,8 @@ int attn_forward_causal(const void *q, const void *k, const void *v, void *o,
 /* Same, with tile fields overridden (tile sweep only).  Honoured fields (0 keeps
  * the closed-form value): n_q (1|2), tile_kv (64|128), kv_stages (2..plan maximum),
  * kv_splits (that many CTAs per Q tile) or ctas (the grid size itself, from 1 up
- * to the number of (Q tile, KV step) units), causal (non-zero selects causal
+ * to the number of (Q tile, KV step) units; a uniform split whose grid exceeds the SM count
+ * is merged by the last CTA of a tile to finish, since fixed merge roles need every CTA resident), causal (non-zero selects causal
  * attention; a grid of 2, 3 or 4 CTAs per tile then runs as clusters that share out
  * each tile's own key steps, any other grid as equal ranges of the unit line).  ATTN_ERR_BAD_TILES if the combination was not compiled or does not
  * fit. */
@@ -315,6 +377,9 @@ int attn_last_device_status(void *cuda_stream, uint32_t *detail);
  */
 #define ATTN_SELFTEST_STEP 0x7E57
 int attn_selftest_wait_expiry(void *cuda_stream);
+/* The same with the record going to four caller-owned DEVICE words (as attn_forward_ws's status_dev; NULL: the
+ * device-wide record): shows that an expiry is attributed to the launch whose status words were given. */
+int attn_selftest_wait_expiry_to(uint32_t *status_dev, void *cuda_stream);
 
 /* Number of kernels the last attn_forward* call on this thread launched. */
 int attn_last_launch_count(void);

@@ -69,7 +69,9 @@ int gemm_forward(const void *a, const void *b, void *c, int batch, int M, int N,
  * p[r][:] = softmax(scale * s[r][:]) for `rows` rows of `cols` bf16 values
  * (cols a multiple of 8, at most 32768); p may be s (in place).  One read and
  * one write of the matrix: the row is held in registers, or staged in shared
- * memory when it has more than 16384 columns.
+ * memory when it has more than 16384 columns.  scale must be positive and finite
+ * (the row maximum is taken on the unscaled scores, which a positive scale keeps
+ * in order): ATTN_ERR_INVALID_ARG otherwise.
  * Errors: ATTN_ERR_INVALID_ARG, ATTN_ERR_UNSUPPORTED_SHAPE, ATTN_ERR_MISALIGNED, ATTN_ERR_CUDA.
  */
 int softmax_rows_forward(const void *s, void *p, long long rows, int cols, float scale, void *cuda_stream);

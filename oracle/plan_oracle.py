@@ -15,8 +15,12 @@ Nothing here is imported by the product; nothing here imports the product.
   Pinned by Table 2 (tests/golden/paper_table2_tiles.txt).
 * ``derive_tiles_tmem_machine`` -- the same fixed-order derivation restated for
   a machine whose accumulators live in tensor memory (B200).  No paper numbers
-  exist for it: parity unpinned against the paper; pinned by capacity
-  invariants only.
+  exist for it: parity unpinned against the paper.  Its capacity part is pinned
+  by capacity invariants; its occupancy part (``grid_candidates`` /
+  ``choose_grid``: every way of sharing out the key axis listed with its
+  eligibility and cost, the first cheapest taken) is pinned by the properties
+  the arithmetic fixes (tests/test_plan_oracle.py) and, for the B200 cost
+  constants, by a measured sweep of grid sizes kept under profiles/.
 * ``traffic_fused`` / ``traffic_unfused`` -- the paper's HBM accounting
   (savings equation and the "HBM traffic" paragraph of Section "Results").
   Pinned by the printed 34 MB / 1,074 MB / 4,329 MB / 129x / 17 GB figures.
@@ -63,21 +67,90 @@ _OUT_ROW_BYTES = 128       # output staging: per softmax warpgroup 64 bf16 colum
 _MAX_STAGES = 8
 _MIN_STAGES = 4
 _MIN_TILE_KV = 32
-_MIN_STEPS_PER_SPLIT = 4
-_SEGMENT_OVERHEAD_STEPS = 3
-_CTA_OVERHEAD_STEPS = 2     # start and end of a CTA that handles one whole Q tile
-_TRANSITION_STEPS = 1       # a persistent CTA moving on to its next Q tile
-# fewer Q tiles than units: cost of the end of a CTA's work, in KV steps
-_MIN_STEPS_PER_CLUSTER_SPLIT = 2
-_CLUSTER_OVERHEAD_STEPS = 5      # k CTAs per tile as one cluster (partials through distributed shared memory)
-_WORKSPACE_OVERHEAD_STEPS = 8    # k CTAs per tile, partials through the workspace (plus k // 2)
-_BALANCED_OVERHEAD_STEPS = 12    # equal ranges of the unit line
-_LANDING_PART_EXTRA = 256        # m and delta of the 32 rows of one part
 
 
 def causal_head_units(q_tiles: int, steps: int, ratio: int) -> int:
     """KV steps summed over the Q tiles of one head when tile q needs min(steps, (q+1)*ratio) of them."""
     return sum(min(steps, (q + 1) * ratio) for q in range(q_tiles))
+
+
+def _cdiv(a: int, b: int) -> int:
+    return -(-a // b)
+
+
+def grid_candidates(desc: dict, heads: int, q_tiles: int, steps: int, ratio: int, causal: bool, n_q: int, d: int,
+                    ring_bytes: int, kv_head_bytes: int) -> list:
+    """Occupancy step (Section "Tile Derivation": block count against compute units) as a table.
+
+    Every way of sharing the (Q tile, KV step) units out to CTAs is one row: its name, the CTAs per tile k (0 if
+    not a per-tile split), the grid size, whether the machine can run it (with the reason if not), the KV steps on
+    the longest CTA's path, and that path plus the descriptor's measured start/end cost for this way (`ovh_*`,
+    in KV steps).  The derivation takes the first row of least cost among the eligible ones; nothing is searched
+    beyond this fixed list.  A part that travels between CTAs of a cluster is 32 rows of d fp32 values plus 256
+    bytes of row statistics; what a CTA receives lands in its Q buffer (two parts) or in its K/V ring.
+    """
+    units = desc["num_units"]
+    clusters = list(desc.get("max_clusters", [0] * 8))
+    tiles = heads * q_tiles
+    part_bytes = 32 * 4 * d + 256
+    groups = 4 * n_q                                  # 32-row groups of one Q tile
+    rows = []
+
+    def row(mode, k, ctas, path, ovh, reasons):
+        rows.append(dict(mode=mode, k=k, ctas=ctas, path=path, cost=path + ovh, eligible=not reasons,
+                         why_not=reasons))
+
+    def cluster_reasons(k, min_share):
+        why = []
+        if tiles * k > units:
+            why.append("more CTAs than units")
+        if clusters[k - 1] < tiles:
+            why.append("clusters not all resident")
+        if min_share < 2:
+            why.append("fewer than 2 steps per CTA")
+        if k > 2 and _cdiv(groups, k) * (k - 1) * part_bytes > ring_bytes:
+            why.append("landing areas exceed the ring")
+        return why
+
+    if causal:
+        total = heads * causal_head_units(q_tiles, steps, ratio)
+        g = max(1, min(units, total // 4))
+        row("ranges", 0, g, _cdiv(total + 3 * tiles, g), desc["ovh_causal_ranges"], [])
+        for k in (2, 3, 4):
+            why = cluster_reasons(k, _cdiv(steps, k))
+            if ratio < 2:
+                why.append("Q tile no longer than the KV tile")
+            row("cluster", k, tiles * k, _cdiv(steps, k), desc["ovh_causal_cluster"], why)
+        return rows
+
+    total = tiles * steps
+    if tiles >= units:
+        waves = _cdiv(tiles, units)
+        rows.append(dict(mode="whole_tiles", k=1, ctas=tiles, path=waves * steps,
+                         cost=waves * (steps + desc["ovh_whole_tile"]), eligible=True, why_not=[]))
+        in_flight = min(heads, units)
+        cached = desc.get("cache_bytes", 0) > 0 and 3 * in_flight * kv_head_bytes <= 2 * desc["cache_bytes"]
+        row("persistent", 0, units, _cdiv(total, units), desc["ovh_persistent"] + waves * desc["ovh_tile_change"],
+            [] if cached else ["K/V of the heads in flight exceed two thirds of the cache"])
+        return rows
+
+    row("whole_tiles", 1, tiles, steps, desc["ovh_whole_tile"], [])
+    for k in range(2, 9):
+        row("cluster", k, tiles * k, _cdiv(steps, k), desc["ovh_cluster"], cluster_reasons(k, steps // k))
+    k = min(units // tiles, steps // 4)
+    row("workspace", k, tiles * max(k, 1), _cdiv(steps, max(k, 1)), desc["ovh_workspace"] + k // 2,
+        [] if k >= 2 else ["fewer than two parts of 4 steps"])
+    g = min(units, total // 4)
+    row("ranges", 0, max(g, 1), _cdiv(total, max(g, 1)), desc["ovh_ranges"],
+        [] if g > tiles else ["no more CTAs than tiles"])
+    return rows
+
+
+def choose_grid(rows: list) -> dict:
+    """First row of least cost among the eligible ones (ties go to the earlier row)."""
+    ok = [r for r in rows if r["eligible"]]
+    least = min(r["cost"] for r in ok)
+    return next(r for r in ok if r["cost"] == least)
 
 
 def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal: bool = False, Lk: int = 0) -> dict:
@@ -118,77 +191,24 @@ def derive_tiles_tmem_machine(desc: dict, B: int, H: int, L: int, d: int, causal
             out["binding"] = BIND_SMEM
             return out
     tile_q = n_q * sub
-    tiles = B * H * -(-L // tile_q)
-    steps = -(-Lk // tile_kv)
+    q_tiles = _cdiv(L, tile_q)
+    tiles = B * H * q_tiles
+    steps = _cdiv(Lk, tile_kv)
     under = tiles < desc["num_units"]
-    ctas = tiles
-    kv_head_bytes = 2 * Lk * d * desc["elem_bytes"]           # K and V of one head
-    if causal:
-        total = B * H * causal_head_units(-(-L // tile_q), steps, tile_q // tile_kv)
-        ctas = max(1, min(total // _MIN_STEPS_PER_SPLIT, desc["num_units"]))
-        # equal ranges (3 cost units per tile on the line, 15 steps of overhead) against k = 2..4 CTAs per tile as one
-        # cluster, a share of the tile's own key steps each (the longest tile sets the time; 6 steps of overhead)
-        cost_ranges = -(-(total + 3 * tiles) // ctas) + 15
-        ratio = tile_q // tile_kv
-        best = cost_ranges
-        clusters = list(desc.get("max_clusters", [0] * 8))
-        part = 32 * 4 * d + _LANDING_PART_EXTRA
-        for k in (2, 3, 4):
-            if ratio < 2 or k * tiles > desc["num_units"] or clusters[k - 1] < tiles or -(-steps // k) < 2:
-                continue
-            if k > 2 and -(-(4 * n_q) // k) * (k - 1) * part > stages * stage:
-                continue
-            cost = -(-steps // k) + 6
-            if cost < best:
-                best, ctas = cost, k * tiles
-    elif under:
-        # one CTA per tile; k CTAs per tile as one cluster; k CTAs per tile through the workspace; equal ranges.
-        # The cheapest wins, ties go to the earlier candidate.
-        units = desc["num_units"]
-        total = tiles * steps
-        best = steps + _CTA_OVERHEAD_STEPS
-        clusters = list(desc.get("max_clusters", [0] * 8))
-        groups = 4 * n_q
-        part = 32 * 4 * d + _LANDING_PART_EXTRA
-        for k in range(2, 9):
-            if tiles * k > units or steps // k < _MIN_STEPS_PER_CLUSTER_SPLIT or clusters[k - 1] < tiles:
-                continue
-            if k > 2 and -(-groups // k) * (k - 1) * part > stages * stage:
-                continue
-            cost = -(-steps // k) + _CLUSTER_OVERHEAD_STEPS
-            if cost < best:
-                best, ctas = cost, tiles * k
-        k = min(units // tiles, steps // _MIN_STEPS_PER_SPLIT)
-        if k >= 2:
-            cost = -(-steps // k) + _WORKSPACE_OVERHEAD_STEPS + k // 2
-            if cost < best:
-                best, ctas = cost, tiles * k
-        g = min(total // _MIN_STEPS_PER_SPLIT, units)
-        if g > tiles:
-            cost = -(-total // g) + _BALANCED_OVERHEAD_STEPS
-            if cost < best:
-                best, ctas = cost, g
-    else:
-        # enough tiles for every unit: one CTA per tile (whole waves, each CTA its own start and end), or one
-        # persistent CTA per unit on an equal range of the (tile, step) line -- only if the K/V of the heads
-        # then in flight stay inside two thirds of the last-level cache
-        units = desc["num_units"]
-        total = tiles * steps
-        cost_tiles = -(-tiles // units) * (steps + _CTA_OVERHEAD_STEPS)
-        cost_balanced = -(-total // units) + 2 * _SEGMENT_OVERHEAD_STEPS + -(-tiles // units) * _TRANSITION_STEPS
-        in_flight = min(B * H, units)
-        cached = desc.get("cache_bytes", 0) > 0 and 3 * in_flight * kv_head_bytes <= 2 * desc["cache_bytes"]
-        if cached and cost_balanced < cost_tiles:
-            ctas = units
-    kv_splits = -(-ctas // tiles)
+    rows = grid_candidates(desc, B * H, q_tiles, steps, tile_q // tile_kv, causal, n_q, d, stages * stage,
+                           2 * Lk * d * desc["elem_bytes"])
+    pick = choose_grid(rows)
+    ctas = pick["ctas"]
     per_unit = ctas / desc["num_units"]
     cols = n_q * (tile_kv + d)
     return dict(feasible=True, binding=binding, tile_q=tile_q, tile_kv=tile_kv, n_q=n_q, n_s=1,
-                kv_stages=stages, kv_splits=kv_splits,
+                kv_stages=stages, kv_splits=_cdiv(ctas, tiles),
                 smem_bytes=q_bytes + stages * stage + reserve,
                 tmem_columns=max(32, 1 << (cols - 1).bit_length()), regs_softmax=regs_soft,
                 threads=threads, tiles=tiles, ctas=ctas, ctas_per_unit=per_unit,
-                wave_efficiency=per_unit / math.ceil(per_unit), under_occupied=under)
+                wave_efficiency=per_unit / math.ceil(per_unit), under_occupied=under,
+                cost_steps=pick["cost"], mode=pick["mode"], k=pick["k"], candidates=rows, steps=steps,
+                ring_bytes=stages * stage)
 
 
 def traffic_fused(B, H, L, d, elem_bytes):

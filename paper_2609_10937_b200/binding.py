@@ -22,8 +22,8 @@ BIND_NAMES = ("none", "smem", "tmem", "reg", "atom", "shape")
 
 EXPORTED_SYMBOLS = (
     "attn_hw_desc_b200", "attn_hw_desc_query", "attn_plan", "attn_plan_ex", "attn_workspace_bytes",
-    "attn_set_workspace", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_host_workspace_bytes", "attn_forward_static_scratch", "attn_forward_desc", "attn_plan_qk", "attn_forward_qk",
-    "attn_last_device_status", "attn_selftest_wait_expiry",
+    "attn_set_workspace", "attn_workspace_init", "attn_forward_ws", "attn_status_read", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_host_workspace_bytes", "attn_forward_static_scratch", "attn_forward_desc", "attn_plan_qk", "attn_forward_qk",
+    "attn_last_device_status", "attn_selftest_wait_expiry", "attn_selftest_wait_expiry_to",
     "attn_last_launch_count", "attn_last_cluster_size", "attn_status_string", "attn_last_cuda_error",
     "gemm_plan", "gemm_forward", "softmax_rows_forward", "attn_forward_unfused",
 )
@@ -33,7 +33,10 @@ class AttnHwDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "struct_bytes", "num_units", "local_mem_bytes", "regs_per_unit", "max_regs_per_thread", "simd_width",
         "acc_mem_lanes", "acc_mem_columns", "atom_m", "atom_n", "atom_k", "atom_n_max", "elem_bytes", "cache_bytes",
-    )] + [("max_clusters", ctypes.c_int32 * 8)] + [("hbm_gbps", ctypes.c_double), ("peak_tflops", ctypes.c_double), ("sm_clock_mhz", ctypes.c_double)]
+    )] + [("max_clusters", ctypes.c_int32 * 8)] + [(n, ctypes.c_int32) for n in (
+        "ovh_whole_tile", "ovh_cluster", "ovh_workspace", "ovh_ranges", "ovh_persistent", "ovh_tile_change",
+        "ovh_causal_ranges", "ovh_causal_cluster",
+    )] + [("hbm_gbps", ctypes.c_double), ("peak_tflops", ctypes.c_double)]
 
 
 class AttnTiles(ctypes.Structure):
@@ -41,7 +44,8 @@ class AttnTiles(ctypes.Structure):
         "tile_q", "tile_kv", "n_q", "n_s", "kv_stages", "kv_splits", "smem_bytes", "tmem_columns", "regs_softmax",
         "threads", "tiles", "ctas",
     )] + [("ctas_per_unit", ctypes.c_float), ("wave_efficiency", ctypes.c_float)] + [
-        (n, ctypes.c_int32) for n in ("feasible", "binding_constraint", "under_occupied", "causal")]
+        (n, ctypes.c_int32) for n in ("feasible", "binding_constraint", "under_occupied", "causal", "cost_steps",
+                                      "bound")] + [("predicted_us", ctypes.c_float)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -87,6 +91,9 @@ def lib() -> ctypes.CDLL:
         L.attn_workspace_bytes.restype = ctypes.c_size_t
         L.attn_set_workspace.argtypes = [i32, vp, ctypes.c_size_t]
         L.attn_forward.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+        L.attn_workspace_init.argtypes = [vp, ctypes.c_size_t, vp, vp]
+        L.attn_forward_ws.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, ctypes.c_size_t, vp, vp]
+        L.attn_status_read.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_uint32)]
         L.attn_plan_qk.argtypes = [ctypes.POINTER(AttnHwDesc), i32, i32, i32, i32, i32, ctypes.POINTER(AttnTiles)]
         L.attn_forward_qk.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.attn_forward_tiles.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, ctypes.POINTER(AttnTiles), vp]
@@ -98,6 +105,7 @@ def lib() -> ctypes.CDLL:
         L.attn_forward_desc.argtypes = [ctypes.POINTER(AttnHwDesc), vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.attn_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.attn_selftest_wait_expiry.argtypes = [vp]
+        L.attn_selftest_wait_expiry_to.argtypes = [vp, vp]
         L.attn_last_launch_count.argtypes = []
         L.attn_last_cluster_size.argtypes = []
         L.attn_status_string.argtypes = [i32]
@@ -211,6 +219,46 @@ def forward(q, k, v, o=None, causal=False):
         _check(fn(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d, stream),
                "attn_forward_causal" if causal else "attn_forward")
     return o
+
+
+def workspace_init(workspace, status=None):
+    """Queues, on the current stream, the clearing of a workspace's arrival counters (its first 64 KB) and of a
+    four-word status tensor; both are caller-owned CUDA tensors (uint8 / int32)."""
+    import torch
+
+    dev = workspace.device if workspace is not None else status.device
+    with torch.cuda.device(dev):
+        stream = torch.cuda.current_stream(dev).cuda_stream
+        _check(lib().attn_workspace_init(workspace.data_ptr() if workspace is not None else None,
+                                         workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                         status.data_ptr() if status is not None else None, stream),
+               "attn_workspace_init")
+
+
+def forward_ws(q, k, v, o=None, *, workspace=None, status=None, causal=False):
+    """forward() with this call's own workspace (a CUDA uint8 tensor, counters cleared by workspace_init) and
+    status words (a CUDA int32 tensor of four elements, or None for the device-wide record)."""
+    o, B, H, L, d, dev, stream = _prep(q, k, v, o)
+    import torch
+
+    with torch.cuda.device(dev):
+        _check(lib().attn_forward_ws(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, L, d,
+                                     1 if causal else 0, workspace.data_ptr() if workspace is not None else None,
+                                     workspace.numel() if workspace is not None else 0,
+                                     status.data_ptr() if status is not None else None, stream), "attn_forward_ws")
+    return o
+
+
+def status_read(status, workspace=None):
+    """Synchronises the current stream; returns (code, detail words) of a call's own status words."""
+    import torch
+
+    detail = (ctypes.c_uint32 * 4)()
+    with torch.cuda.device(status.device):
+        stream = torch.cuda.current_stream(status.device).cuda_stream
+        code = lib().attn_status_read(status.data_ptr(), workspace.data_ptr() if workspace is not None else None,
+                                      stream, detail)
+    return int(code), [int(x) for x in detail]
 
 
 def forward_static_scratch(q, k, v, o):

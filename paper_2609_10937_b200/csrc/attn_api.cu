@@ -79,6 +79,7 @@ struct DeviceState {
   bool arch_checked = false;
   bool arch_ok = false;
   attn_hw_desc desc;
+  int resident[2][9] = {};     // [causal][k]: clusters of k CTAs that fit at once, + 1 (0 = not asked yet); guarded by g_mu
 };
 DeviceState g_dev[kMaxDevices];
 std::mutex g_mu;
@@ -119,7 +120,7 @@ int check_args(const void* q, const void* k, const void* v, const void* o, int B
 
 template <int D, int TKV, int NQ>
 int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int Lk, const attn_tiles& t,
-               float* ws, cudaStream_t stream) {
+               float* ws, unsigned int* status, DeviceState* st, cudaStream_t stream, bool may_overlap) {
   using SM = attn::FwdSmem<D, TKV, NQ>;
   const int BH = B * H;
   CUtensorMap tq, tk, tv, to;
@@ -140,34 +141,33 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   p.head_units = attn::tile_prefix(p.n_steps, p.ratio, p.causal, p.q_tiles);
   p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
   p.o = reinterpret_cast<__nv_bfloat16*>(o);
+  p.status = status;
   p.counters = reinterpret_cast<unsigned int*>(ws);                   // head of the workspace
   p.ws = ws ? ws + attn::kCounterBytes / sizeof(float) : nullptr;    // partial results follow
   int grid = t.ctas;
   p.seg_skip = 0;
-#ifndef ATTN_NO_STRIDED
   // One CTA per tile with more tiles than SMs: a persistent grid of one CTA per SM runs them in the same order.
+  const int sms = st->desc.num_units;                      // of the device itself (the plan may be for a smaller machine)
   if (!p.causal && t.ctas == t.tiles) {
-    int dev = 0, sms = 0;
-    ATTN_CUDA_TRY(cudaGetDevice(&dev));
-    static int sm_count[kMaxDevices] = {};
-    if (dev >= 0 && dev < kMaxDevices) {
-      if (sm_count[dev] == 0) ATTN_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
-      sms = sm_count[dev];
-    }
     if (sms > 0 && t.tiles > sms) {
       grid = sms;
       p.seg_skip = (long long)(grid - 1) * p.n_steps;
     }
   }
-#endif
   const long long total_units = p.head_units * BH;
   // at least one KV step per CTA; when Q tiles are shared, the counters of every (CTA, sub-tile, warp) --
   // two each -- must fit the counter block
   if (grid < 1 || (long long)grid > total_units) return ATTN_ERR_BAD_TILES;
   if (ws && (size_t)grid * NQ * 8 > attn::kCounterBytes / sizeof(unsigned int)) return ATTN_ERR_BAD_TILES;
   const int smem = SM::total(t.kv_stages);
-  // uniform key split (k CTAs per tile, all parts of a tile finish together): the instantiation with fixed merge roles
-  const bool eager = !p.causal && t.ctas > t.tiles && t.ctas % t.tiles == 0;
+  // uniform key split (k CTAs per tile, all parts of a tile finish together): the instantiation with fixed merge roles.
+  // Its merging warps wait for the other CTAs of their tile, so every CTA of the grid must be resident at once (one
+  // CTA per SM); a larger grid takes the instantiation in which the last CTA to finish merges and nobody waits for a
+  // CTA that has not started.  The same holds for a launch that may run beside another one of its kind on the same
+  // device (attn_forward_ws: two such kernels could each hold part of the SMs and wait for CTAs that cannot start);
+  // thread-block clusters are scheduled as a whole and stay in use there.
+  const bool eager = !p.causal && t.ctas > t.tiles && t.ctas % t.tiles == 0 && grid <= sms;
+  const bool wait_roles_ok = !may_overlap;
   auto launch = [&](auto kern) -> int {
     ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
@@ -182,7 +182,6 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
   t_cluster_size = 0;
   auto launch_eager = [&](auto kern, auto kern_cluster) -> int {
     ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-#ifndef ATTN_NO_CLUSTER
     ATTN_CUDA_TRY(cudaFuncSetAttribute(kern_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int kk = t.ctas / t.tiles;
     const size_t landing = (size_t)((4 * NQ + kk - 1) / kk) * (kk - 1) * (32 * D * 4 + 256);
@@ -199,27 +198,27 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
       attr[0].val.clusterDim.z = 1;
       cfg.attrs = attr;
       cfg.numAttrs = 1;
-      static int resident[9][kMaxDevices] = {};          // clusters of kk CTAs that fit at once (+1; 0 = not asked yet)
-      int dev = 0;
-      ATTN_CUDA_TRY(cudaGetDevice(&dev));
-      if (dev >= 0 && dev < kMaxDevices) {
-        if (resident[kk][dev] == 0) {
+      int n_res;
+      {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (st->resident[0][kk] == 0) {
           int n = 0;
           if (cudaOccupancyMaxActiveClusters(&n, kern_cluster, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
-          resident[kk][dev] = n + 1;
+          st->resident[0][kk] = n + 1;
         }
-        if ((long long)(resident[kk][dev] - 1) * kk >= grid) {
-          attn::FwdParams pc = p;
-          pc.cluster_k = kk;
-          if (cudaLaunchKernelEx(&cfg, kern_cluster, tq, tk, tv, to, pc) == cudaSuccess) {
-            t_cluster_size = kk;
-            return ATTN_OK;
-          }
-          (void)cudaGetLastError();                       // fall through to the plain launch
+        n_res = st->resident[0][kk] - 1;
+      }
+      if ((long long)n_res * kk >= grid) {
+        attn::FwdParams pc = p;
+        pc.cluster_k = kk;
+        if (cudaLaunchKernelEx(&cfg, kern_cluster, tq, tk, tv, to, pc) == cudaSuccess) {
+          t_cluster_size = kk;
+          return ATTN_OK;
         }
+        (void)cudaGetLastError();                         // fall through to the plain launch
       }
     }
-#endif
+    if (!wait_roles_ok) return ATTN_ERR_BAD_TILES;        // (marker: the caller launches the last-finisher instantiation)
     kern<<<grid, 512, smem, stream>>>(tq, tk, tv, to, p);
     return ATTN_OK;
   };
@@ -245,16 +244,15 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
     pc.cluster_k = ck;
     pc.seg_skip = -ck;
     // all clusters resident at once, else (or if the cluster launch fails) the same grid as equal ranges
-    static int c_resident[5][kMaxDevices] = {};
-    int dev = 0, n_res = 0;
-    ATTN_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev >= 0 && dev < kMaxDevices) {
-      if (c_resident[ck][dev] == 0) {
+    int n_res = 0;
+    {
+      std::lock_guard<std::mutex> lk(g_mu);
+      if (st->resident[1][ck] == 0) {
         int n = 0;
         if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
-        c_resident[ck][dev] = n + 1;
+        st->resident[1][ck] = n + 1;
       }
-      n_res = c_resident[ck][dev] - 1;
+      n_res = st->resident[1][ck] - 1;
     }
     if ((long long)n_res * ck >= grid && cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, to, pc) == cudaSuccess) {
       t_cluster_size = ck;
@@ -264,8 +262,10 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
       rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, true, false>);
     }
   } else if (p.causal) rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, true, false>);
-  else if (eager) rc = launch_eager(attn::attn_fwd_kernel<D, TKV, NQ, false, true>, attn::attn_fwd_kernel<D, TKV, NQ, false, true, true>);
-  else rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, false, false>);
+  else if (eager) {
+    rc = launch_eager(attn::attn_fwd_kernel<D, TKV, NQ, false, true>, attn::attn_fwd_kernel<D, TKV, NQ, false, true, true>);
+    if (rc == ATTN_ERR_BAD_TILES && !wait_roles_ok) rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, false, false>);
+  } else rc = launch(attn::attn_fwd_kernel<D, TKV, NQ, false, false>);
   if (rc != ATTN_OK) return rc;
   ATTN_CUDA_TRY(cudaGetLastError());
   t_launch_count = 1;
@@ -273,10 +273,12 @@ int launch_fwd(const void* q, const void* k, const void* v, void* o, int B, int 
 }
 
 int dispatch_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
-                 const attn_tiles& t, float* ws, cudaStream_t s, int Lk = 0) {
+                 const attn_tiles& t, float* ws, unsigned int* status, DeviceState* st, cudaStream_t s, int Lk = 0,
+                 bool may_overlap = false) {
   if (Lk == 0) Lk = L;
 #define ATTN_CASE(D_, TKV_, NQ_) \
-  if (d == D_ && t.tile_kv == TKV_ && t.n_q == NQ_) return launch_fwd<D_, TKV_, NQ_>(q, k, v, o, B, H, L, Lk, t, ws, s);
+  if (d == D_ && t.tile_kv == TKV_ && t.n_q == NQ_) \
+    return launch_fwd<D_, TKV_, NQ_>(q, k, v, o, B, H, L, Lk, t, ws, status, st, s, may_overlap);
   ATTN_CASE(128, 128, 2)
   ATTN_CASE(128, 64, 2)
   ATTN_CASE(128, 128, 1)
@@ -292,8 +294,16 @@ int dispatch_fwd(const void* q, const void* k, const void* v, void* o, int B, in
 // A plan needs the workspace unless every CTA owns exactly one whole Q tile.
 bool plan_needs_workspace(const attn_tiles& t) { return t.causal != 0 || t.ctas != t.tiles; }
 
+// A workspace handed to one call (attn_forward_ws) instead of the one registered for the device.
+struct CallWorkspace {
+  void* ws;
+  size_t bytes;
+  unsigned int* status;
+};
+
 int forward_impl(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d, int causal,
-                 const attn_tiles* ovr, void* cuda_stream, const attn_hw_desc* plan_desc = nullptr, int Lk = 0) {
+                 const attn_tiles* ovr, void* cuda_stream, const attn_hw_desc* plan_desc = nullptr, int Lk = 0,
+                 const CallWorkspace* call_ws = nullptr) {
   t_launch_count = 0;
   if (Lk == 0) Lk = L;                       // keys per head; L is the number of query rows per head
   int rc = check_args(q, k, v, o, B, H, L, d, Lk);
@@ -339,7 +349,7 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
       t.ctas = t.tiles * ovr->kv_splits;
     } else {
       t.ctas = attn_internal::grid_size(desc, B * H, (L + t.tile_q - 1) / t.tile_q, steps, t.tile_q / t.tile_kv, causal,
-                                        2LL * Lk * d * desc.elem_bytes, 4 * t.n_q, d, (long long)t.kv_stages * stage);
+                                        2LL * Lk * d * desc.elem_bytes, 4 * t.n_q, d, (long long)t.kv_stages * stage).ctas;
     }
     t.kv_splits = (t.ctas + t.tiles - 1) / t.tiles;
     if (t.ctas < 1) return ATTN_ERR_BAD_TILES;
@@ -348,11 +358,17 @@ int forward_impl(const void* q, const void* k, const void* v, void* o, int B, in
   float* ws = nullptr;
   if (plan_needs_workspace(t)) {
     const size_t need = attn_workspace_bytes(&t, B, H, L, d);
-    std::lock_guard<std::mutex> lk(g_mu);
-    if (!st->ws || st->ws_bytes < need) return ATTN_ERR_NEED_WORKSPACE;
-    ws = static_cast<float*>(st->ws);
+    if (call_ws) {
+      if (!call_ws->ws || call_ws->bytes < need) return ATTN_ERR_NEED_WORKSPACE;
+      ws = static_cast<float*>(call_ws->ws);
+    } else {
+      std::lock_guard<std::mutex> lk(g_mu);
+      if (!st->ws || st->ws_bytes < need) return ATTN_ERR_NEED_WORKSPACE;
+      ws = static_cast<float*>(st->ws);
+    }
   }
-  return dispatch_fwd(q, k, v, o, B, H, L, d, t, ws, static_cast<cudaStream_t>(cuda_stream), Lk);
+  return dispatch_fwd(q, k, v, o, B, H, L, d, t, ws, call_ws ? call_ws->status : nullptr, st,
+                      static_cast<cudaStream_t>(cuda_stream), Lk, call_ws != nullptr);
 }
 
 template <int D, int TKV>
@@ -367,11 +383,9 @@ int launch_simple(const void* q, const void* k, const void* v, void* o, int B, i
   const int smem = attn::kSub * D * 2 + 2 * TKV * D * 2 + 1024;
   auto kern = attn::attn_fwd_simple_kernel<D, TKV>;
   ATTN_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  const char* dbg = std::getenv("ATTN_SIMPLE_DEBUG_FLAGS");
-  const int flags = dbg ? std::atoi(dbg) : 0;
   const float scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
   dim3 grid((L + attn::kSub - 1) / attn::kSub, BH);
-  kern<<<grid, 128, smem, stream>>>(tq, tk, tv, reinterpret_cast<__nv_bfloat16*>(o), L, scale_log2, scores_out, flags);
+  kern<<<grid, 128, smem, stream>>>(tq, tk, tv, reinterpret_cast<__nv_bfloat16*>(o), L, scale_log2, scores_out);
   ATTN_CUDA_TRY(cudaGetLastError());
   t_launch_count = 1;
   return ATTN_OK;
@@ -396,8 +410,7 @@ extern "C" int attn_hw_desc_query(int device, attn_hw_desc* out) {
   out->num_units = sms;
   out->local_mem_bytes = smem_optin;
   out->regs_per_unit = regs;
-  out->sm_clock_mhz = clock_khz / 1000.0;
-  // dense bf16: 8192 FLOP per clock per SM
+  // dense bf16: 8192 FLOP per clock per SM at the device's maximum SM clock
   out->peak_tflops = 8192.0 * sms * (clock_khz * 1e3) / 1e12;
   // Resident clusters of k CTAs, asked for the kernel that uses them at its largest shared-memory footprint.
   {
@@ -447,6 +460,39 @@ extern "C" int attn_set_workspace(int device, void* dev_ptr, size_t bytes) {
 extern "C" int attn_forward(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d,
                             void* cuda_stream) {
   return forward_impl(q, k, v, o, B, H, L, d, 0, nullptr, cuda_stream);
+}
+
+extern "C" int attn_workspace_init(void* workspace, size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream) {
+  if (!workspace && !status_dev) return ATTN_ERR_INVALID_ARG;
+  if (workspace && (((uintptr_t)workspace & 15u) || workspace_bytes < (size_t)attn::kCounterBytes)) return ATTN_ERR_INVALID_ARG;
+  if (status_dev && ((uintptr_t)status_dev & 15u)) return ATTN_ERR_MISALIGNED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (workspace) ATTN_CUDA_TRY(cudaMemsetAsync(workspace, 0, attn::kCounterBytes, s));
+  if (status_dev) ATTN_CUDA_TRY(cudaMemsetAsync(status_dev, 0, 4 * sizeof(uint32_t), s));
+  return ATTN_OK;
+}
+
+extern "C" int attn_forward_ws(const void* q, const void* k, const void* v, void* o, int B, int H, int L, int d, int causal,
+                               void* workspace, size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream) {
+  if (workspace && ((uintptr_t)workspace & 15u)) return ATTN_ERR_MISALIGNED;
+  if (status_dev && ((uintptr_t)status_dev & 15u)) return ATTN_ERR_MISALIGNED;
+  const CallWorkspace cw = {workspace, workspace ? workspace_bytes : 0, status_dev};
+  return forward_impl(q, k, v, o, B, H, L, d, causal ? 1 : 0, nullptr, cuda_stream, nullptr, 0, &cw);
+}
+
+extern "C" int attn_status_read(uint32_t* status_dev, void* workspace, void* cuda_stream, uint32_t* detail) {
+  if (!status_dev) return ATTN_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  ATTN_CUDA_TRY(cudaStreamSynchronize(s));
+  unsigned int h[4] = {0, 0, 0, 0};
+  ATTN_CUDA_TRY(cudaMemcpy(h, status_dev, sizeof h, cudaMemcpyDeviceToHost));
+  if (detail)
+    for (int i = 0; i < 4; ++i) detail[i] = h[i];
+  if (h[0] == 0) return ATTN_OK;
+  // the aborted launch may have left arrival counters non-zero
+  ATTN_CUDA_TRY(cudaMemset(status_dev, 0, sizeof h));
+  if (workspace) ATTN_CUDA_TRY(cudaMemset(workspace, 0, attn::kCounterBytes));
+  return ATTN_ERR_DEVICE_TIMEOUT;
 }
 
 extern "C" int attn_forward_qk(const void* q, const void* k, const void* v, void* o, int B, int H, int Lq, int Lk, int d,
@@ -520,17 +566,12 @@ HostPipe* host_pipe() {
 // (Measured at L = 16384, d = 128: unsplit 0.450 ms, two blocks 0.398 ms, four blocks 0.475 ms -- a 4096-row
 // launch against 16384 keys fills the machine worse than the copies it hides.)
 int host_split(int B, int H, int L, int rows[kHostBlocksMax]) {
-#ifdef ATTN_NO_HOST_PIPELINE
-  (void)B; (void)H; (void)L; (void)rows;
-  return 0;
-#else
   if ((long long)B * H != 1 || L < 8192) return 0;
   const int n = std::min(kHostBlocksMax, L / 4096);
   const int per = ((L + n - 1) / n + 255) / 256 * 256;
   int left = L, c = 0;
   for (; c < n && left > 0; ++c) { rows[c] = std::min(per, left); left -= rows[c]; }
   return c;
-#endif
 }
 }  // namespace
 
@@ -659,34 +700,37 @@ extern "C" int attn_forward_static_scratch(const void* q, const void* k, const v
     // the array keeps the previous call's contents: the arrival counters must start at zero
     ATTN_CUDA_TRY(cudaMemsetAsync(scratch, 0, attn::kCounterBytes, stream));
   }
-  return dispatch_fwd(q, k, v, o, B, H, L, d, t, static_cast<float*>(scratch), stream);
+  return dispatch_fwd(q, k, v, o, B, H, L, d, t, static_cast<float*>(scratch), nullptr, st, stream);
 }
 
 namespace {
 // One warp waits, with the kernels' bounded wait, on a barrier that nothing arrives at: the wait runs out
 // after its cycle limit (about half a second), records the expiry and the kernel returns by itself.
-__global__ void wait_expiry_selftest_kernel() {
+__global__ void wait_expiry_selftest_kernel(unsigned int* status) {
   __shared__ uint64_t bar;
-  __shared__ int abort_flag;
+  __shared__ attn::AbortCell abort_cell;
   if (threadIdx.x == 0) {
-    abort_flag = 0;
+    attn::abort_cell_init(&abort_cell, status);
     sm100::mbar_init(sm100::smem_u32(&bar), 1);
     sm100::fence_mbar_init();
   }
   __syncthreads();
-  (void)attn::wait_bar_warp(sm100::smem_u32(&bar), 0, &abort_flag,
+  (void)attn::wait_bar_warp(sm100::smem_u32(&bar), 0, &abort_cell.flag,
                             attn::wait_info(attn::kRoleSimple, attn::kBarSync, ATTN_SELFTEST_STEP));
 }
 }  // namespace
 
-extern "C" int attn_selftest_wait_expiry(void* cuda_stream) {
+extern "C" int attn_selftest_wait_expiry_to(uint32_t* status_dev, void* cuda_stream) {
+  if (status_dev && ((uintptr_t)status_dev & 15u)) return ATTN_ERR_MISALIGNED;
   DeviceState* st = nullptr;
   int rc = device_state(&st);
   if (rc != ATTN_OK) return rc;
-  wait_expiry_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>();
+  wait_expiry_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(status_dev);
   ATTN_CUDA_TRY(cudaGetLastError());
   return ATTN_OK;
 }
+
+extern "C" int attn_selftest_wait_expiry(void* cuda_stream) { return attn_selftest_wait_expiry_to(nullptr, cuda_stream); }
 
 extern "C" int attn_last_device_status(void* cuda_stream, uint32_t* detail) {
   ATTN_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
@@ -708,23 +752,6 @@ extern "C" int attn_last_device_status(void* cuda_stream, uint32_t* detail) {
   return ATTN_ERR_DEVICE_TIMEOUT;
 }
 
-#ifdef ATTN_TRACE
-// Debug builds only: copies the timeline of CTA 0 (5 roles x 16 steps x 8 events, clock64 values).
-extern "C" int attn_debug_read_trace(long long* out) {
-  ATTN_CUDA_TRY(cudaDeviceSynchronize());
-  ATTN_CUDA_TRY(cudaMemcpyFromSymbol(out, attn::g_attn_trace, sizeof(long long) * 5 * 16 * 8));
-  return ATTN_OK;
-}
-#endif
-
-#ifdef ATTN_TRACE
-extern "C" int attn_debug_read_cta_times(unsigned long long* out, int n) {
-  ATTN_CUDA_TRY(cudaDeviceSynchronize());
-  ATTN_CUDA_TRY(cudaMemcpyFromSymbol(out, attn::g_attn_cta_times, sizeof(unsigned long long) * 2 * n));
-  return ATTN_OK;
-}
-#endif
-
 extern "C" int attn_last_launch_count(void) { return t_launch_count; }
 extern "C" int attn_last_cluster_size(void) { return t_cluster_size; }
 
@@ -739,7 +766,7 @@ extern "C" const char* attn_status_string(int status) {
     case ATTN_ERR_ALIASING: return "output overlaps an input";
     case ATTN_ERR_INFEASIBLE_PLAN: return "no feasible tile plan";
     case ATTN_ERR_WRONG_ARCH: return "device is not compute capability 10.x";
-    case ATTN_ERR_NEED_WORKSPACE: return "plan splits the key axis: register a workspace with attn_set_workspace";
+    case ATTN_ERR_NEED_WORKSPACE: return "CTAs share Q tiles: register a workspace with attn_set_workspace (or pass one to attn_forward_ws)";
     case ATTN_ERR_CUDA: return "CUDA error (see attn_last_cuda_error)";
     case ATTN_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
     case ATTN_ERR_BAD_TILES: return "tile override not available";
@@ -803,7 +830,8 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
 }
 
 int softmax_launch(const void* s, void* pout, long long rows, int cols, float scale, cudaStream_t stream) {
-  if (!s || !pout || rows <= 0 || cols <= 0) return ATTN_ERR_INVALID_ARG;
+  // the kernels take the row maximum on the raw scores and scale it afterwards: the scale must keep the order
+  if (!s || !pout || rows <= 0 || cols <= 0 || !(scale > 0.0f) || !std::isfinite(scale)) return ATTN_ERR_INVALID_ARG;
   if ((cols & 7) || cols > 32768 || rows > 0x7FFFFFFFLL) return ATTN_ERR_UNSUPPORTED_SHAPE;
   if (((uintptr_t)s | (uintptr_t)pout) & 15u) return ATTN_ERR_MISALIGNED;
   const float scale_log2 = scale * 1.4426950408889634f;

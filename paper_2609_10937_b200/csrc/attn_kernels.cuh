@@ -45,44 +45,23 @@ enum Role : uint32_t { kRoleLoad = 1, kRoleMma = 2, kRoleSoftmax = 3, kRoleCorre
 enum BarId : uint32_t { kBarQ = 1, kBarKvFull = 2, kBarKvEmpty = 3, kBarSFull = 4, kBarPFull = 5, kBarOFull = 6,
                         kBarAlpha = 7, kBarLoad = 8, kBarMma = 9, kBarSync = 10 };
 
-// Optional timeline instrumentation (debug builds only, -DATTN_TRACE): CTA 0 records clock64()
-// at fixed points of each role for KV steps [kTraceStep0, kTraceStep0 + 16).
-#ifdef ATTN_TRACE
-#ifndef ATTN_TRACE_STEP0
-#define ATTN_TRACE_STEP0 8
-#endif
-constexpr int kTraceStep0 = ATTN_TRACE_STEP0;
-__device__ long long g_attn_trace[5][16][8];
-#define ATTN_TRACE_EVENT(role_slot, step, ev)                                                   \
-  do {                                                                                          \
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (step) >= kTraceStep0 && (step) < kTraceStep0 + 16) \
-      g_attn_trace[role_slot][(step) - kTraceStep0][ev] = clock64();                            \
-  } while (0)
-__device__ unsigned long long g_attn_cta_times[4096][2];
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
+// A CTA's abort flag (shared memory) and, beside it, where this launch reports an expired wait: four words of the
+// caller's (attn_forward_ws) or g_attn_dev_status.  Every `abort_flag` pointer in the kernels points at `flag` of
+// such a cell.
+struct AbortCell {
+  int flag;
+  int pad;
+  unsigned int* status;
+};
+__device__ __forceinline__ void abort_cell_init(AbortCell* c, unsigned int* status) {
+  c->flag = 0;
+  c->status = status ? status : g_attn_dev_status;
 }
-#define ATTN_TRACE_CTA(which)                                                  \
-  do {                                                                         \
-    if (threadIdx.x == 0 && blockIdx.x < 4096) g_attn_cta_times[blockIdx.x][which] = global_timer_ns(); \
-  } while (0)
-#define ATTN_TRACE_MARK(ev)                                                    \
-  do {                                                                         \
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) g_attn_trace[4][ev >> 3][ev & 7] = clock64(); \
-  } while (0)
-#else
-constexpr int kTraceStep0 = 0;
-#define ATTN_TRACE_EVENT(role_slot, step, ev) do {} while (0)
-#define ATTN_TRACE_MARK(ev) do {} while (0)
-#define ATTN_TRACE_CTA(which) do {} while (0)
-#endif
-
-__device__ __noinline__ void report_timeout(uint32_t info) {
-  if (atomicCAS(&g_attn_dev_status[0], 0u, 1u) == 0u) {
-    g_attn_dev_status[1] = info;
-    g_attn_dev_status[2] = blockIdx.x + gridDim.x * blockIdx.y;
+__device__ __noinline__ void report_timeout(uint32_t info, volatile int* abort_flag) {
+  unsigned int* st = reinterpret_cast<const AbortCell*>(const_cast<const int*>(abort_flag))->status;
+  if (atomicCAS(&st[0], 0u, 1u) == 0u) {
+    st[1] = info;
+    st[2] = blockIdx.x + gridDim.x * blockIdx.y;
     __threadfence();
   }
 }
@@ -97,7 +76,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     if ((++it & 127u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) {
-        report_timeout(info);
+        report_timeout(info, abort_flag);
         *abort_flag = 1;
         return false;
       }
@@ -175,6 +154,7 @@ struct FwdParams {
   __nv_bfloat16* o;        // output, written directly when a result cannot go through the Q buffer
   float* ws;               // partial results of Q tiles shared by several CTAs
   unsigned int* counters;  // arrival counters of shared Q tiles; zero between launches
+  unsigned int* status;    // four words that receive the record of an expired wait (nullptr: g_attn_dev_status)
   int cluster_k;           // > 1: the k CTAs of a Q tile are one thread-block cluster (uniform key split only)
   long long seg_skip;      // > 0: (gridDim.x - 1) * n_steps -- CTA c walks the whole tiles c, c + gridDim.x, ...
                            // < 0 (causal, clusters of k = -seg_skip): CTA c takes a share of the key steps of tile c / k
@@ -194,10 +174,7 @@ __host__ __device__ __forceinline__ int tile_steps(int n_steps, int ratio, int c
 // about as much as a few KV steps.  So that equal ranges of the line mean equal time, every causal tile is
 // preceded on the line by kCausalTileCost units that stand for that cost: a CTA whose range covers them
 // simply has fewer real steps.  (Non-causal tiles all have the same length: nothing to even out.)
-#ifndef ATTN_CAUSAL_TILE_COST
-#define ATTN_CAUSAL_TILE_COST 3
-#endif
-constexpr int kCausalTileCost = ATTN_CAUSAL_TILE_COST;
+constexpr int kCausalTileCost = 3;
 // Units of Q tiles 0..q-1 of one head (closed form: a triangular number until the step count saturates;
 // causal: plus the cost units of those tiles).
 __host__ __device__ __forceinline__ long long tile_prefix(int n_steps, int ratio, int causal, int q) {
@@ -313,9 +290,8 @@ struct FwdMisc {               // lives in the last 3072 bytes of dynamic shared
   uint64_t s_free[2];          // d = 64: the softmax warpgroup holds the step's scores in registers
   uint64_t peers_ready;        // cluster: every other CTA of the tile has finished with its K/V ring
   uint64_t data_ready[8][2];   // cluster: the other CTAs' parts of softmax warp w's rows have landed ([1]: columns 64..)
-  uint64_t dbg_bar[2];         // trace builds only: completion of the first half of P V
+  AbortCell abort;
   uint32_t tmem_slot;
-  int abort_flag;
 };
 static_assert(sizeof(FwdMisc) <= 3072, "misc region too large");
 
@@ -376,20 +352,15 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, const ExpConsts& k, 
 // by MUFU ex2, which balances the two pipes (MUFU alone would take as long as the matrix products).
 // Two of eight measured best on B200: more polynomial work costs issue slots that the other warps
 // of the scheduler partition (and the MMA-issuing warp) need.
-#ifndef ATTN_POLY_PAIRS_D128
-#define ATTN_POLY_PAIRS_D128 2
-#endif
-#ifndef ATTN_POLY_PAIRS_D64
-#define ATTN_POLY_PAIRS_D64 2
-#endif
-template <int kPolyPairsPer8>
+constexpr int kPolyPairsPer8 = 2;
+template <int kPolyPairs>
 __device__ __forceinline__ void exp_chunk(const uint32_t* s, const ExpConsts& k, uint64_t neg_m2, uint64_t& sum2,
                                           uint32_t (&pk)[16]) {
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
     const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[2 * j]), __uint_as_float(s[2 * j + 1])), k.scale2, neg_m2);
     float e0, e1;
-    if ((j & 7) < kPolyPairsPer8) {
+    if ((j & 7) < kPolyPairs) {
       exp2_poly_pair(x2, k, e0, e1);
     } else {
       float x0, x1;
@@ -426,7 +397,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   constexpr int S_COLS = TKV;                         // fp32 score columns per sub-tile
   constexpr int O_COL0 = NQ * S_COLS;                 // O accumulators follow the score buffers
   constexpr int NCH = TKV / 32;                       // 32-column chunks of one score row
-  constexpr int kPoly = (D == 128) ? ATTN_POLY_PAIRS_D128 : ATTN_POLY_PAIRS_D64;   // polynomial pairs per 8
+  constexpr int kPoly = kPolyPairsPer8;             // polynomial pairs per 8
   // d = 64 leaves tensor memory for P next to S and O.  The score buffer is then free as soon as the softmax
   // warpgroup has read it into registers, and the next step's Q K^T runs during this step's exponentials instead
   // of after this step's P V.  (d = 128 fills tensor memory: P overwrites the front of the score buffer.)
@@ -444,7 +415,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const uint32_t ring_smem = smem_base + SM::kQBytes;
   const uint32_t out_smem = ring_smem + p.stages * SM::kStageBytes;   // output staging of segments that are not the CTA's last
   FwdMisc* misc = reinterpret_cast<FwdMisc*>(smem_raw + SM::kQBytes + p.stages * SM::kStageBytes + SM::kOutBytes);
-  volatile int* abort_flag = &misc->abort_flag;
+  volatile int* abort_flag = &misc->abort.flag;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -467,13 +438,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (st < cl_parts) cl_parts = st;
   }
   (void)cl_parts;
-  ATTN_TRACE_CTA(0);
   if (threadIdx.x == 0) {
-    ATTN_TRACE_MARK(0);
-    misc->abort_flag = 0;
+    abort_cell_init(&misc->abort, p.status);
     if (smem_base & 1023u) {                 // swizzled tiles need 1024-byte alignment
-      report_timeout(wait_info(kRoleLoad, 0, 0xFFFF));
-      misc->abort_flag = 1;
+      report_timeout(wait_info(kRoleLoad, 0, 0xFFFF), abort_flag);
+      misc->abort.flag = 1;
     }
     mbar_init(smem_u32(&misc->q_full[0]), 1);
     mbar_init(smem_u32(&misc->q_full[1]), 1);
@@ -487,7 +456,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(smem_u32(&misc->p_half[i]), kSub);
       mbar_init(smem_u32(&misc->o_full[i]), 1);
       mbar_init(smem_u32(&misc->alpha_full[i]), kSub);
-      mbar_init(smem_u32(&misc->dbg_bar[i]), 1);
       mbar_init(smem_u32(&misc->o_free[i]), kSub);
       mbar_init(smem_u32(&misc->s_free[i]), kSub);
     }
@@ -527,7 +495,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   if constexpr (CLUSTER) cluster_arrive();
   const uint32_t tmem_base = misc->tmem_slot;
   const bool run = (*abort_flag == 0) && u_hi > u_lo;
-  if (threadIdx.x == 0) ATTN_TRACE_MARK(1);
 
   // Every role walks the same list of segments (see next_segment); `g` counts KV steps over all
   // segments of this CTA and gives the parity of the per-step barriers.
@@ -567,8 +534,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         constexpr bool kMasked = decltype(mask_tag)::value;
         if (!wait_bar_warp(bar_s, g & 1, abort_flag, wait_info(kRoleSoftmax, kBarSFull, g))) return false;
         tc_fence_after();
-        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 0);
-        if (warp == 0 && g == 0) ATTN_TRACE_MARK(2);
         uint32_t s[TKV];
         // load the row in two halves: the maximum of the first half is taken while the second is in flight
 #pragma unroll
@@ -588,7 +553,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                                  fmaxf(chain_max<TKV / 4, 3 * TKV / 8>(s), chain_max<3 * TKV / 8, TKV / 2>(s)));
 #pragma unroll
         for (int c = NCH / 2; c < NCH; ++c) tmem_ld_fence(*reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 1);
         if constexpr (kSplitP) {
           tc_fence_before();
           mbar_arrive(smem_u32(&misc->s_free[i]));         // the scores are in registers: the buffer may be overwritten
@@ -617,19 +581,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const bool move = (gap > kRescaleThreshold) || (gap > 0.f && kDominanceFactor > delta * shrink);
         const float m_new = move ? m_cand : m_run;
         const float alpha = move ? shrink : 1.0f;
-        misc->alpha[i][g & 1][row] = alpha;
-        mbar_arrive(bar_a);
-        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 2);
-        const uint64_t neg_m2 = pack_f32x2(-m_new, -m_new);
-        uint64_t sum_a = 0ull, sum_b = 0ull;               // packed (0.f, 0.f)
-        uint32_t pk[16];
         if constexpr (kSplitP) {
-          // P has its own columns: the previous step's P V must have read them (it finished long ago as a rule)
+          // P has its own columns: the previous step's P V must have read them before they are overwritten (it
+          // finished long ago as a rule).  The wait stands BEFORE this step's arrivals on purpose.  With P in its
+          // own columns the next scores are produced before this step's P V is issued, so without it a fast warp
+          // (softmax or, through alpha_full, correction) could make its arrival of step g+1 on alpha_full / p_full
+          // while a slow warp has not made that of step g; arrivals are anonymous, so the barrier's phase g would
+          // complete on the wrong 128 / 256 arrivals.  Here every arrival of step g comes after P V(g-1) has
+          // finished, hence after every thread's arrivals of step g-1.  (The segment's first step is covered by
+          // the wait for the last P V at the end of the previous segment.)
           if (g != g_seg0) {
             if (!wait_bar_warp(smem_u32(&misc->o_full[i]), (g - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, 0x4000 | g))) return false;
             tc_fence_after();
           }
         }
+        misc->alpha[i][g & 1][row] = alpha;
+        mbar_arrive(bar_a);
+        const uint64_t neg_m2 = pack_f32x2(-m_new, -m_new);
+        uint64_t sum_a = 0ull, sum_b = 0ull;               // packed (0.f, 0.f)
+        uint32_t pk[16];
         // first half of the row: the second product may start on it while the rest is computed
 #pragma unroll
         for (int c = 0; c < NCH / 2; ++c) {
@@ -638,11 +608,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         uint32_t pk2[16];
         exp_chunk<kPoly>(&s[(NCH / 2) * 32], ek, neg_m2, sum_b, pk2);
-        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 3);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar_p);
-        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 4);
         tmem_st16(p_tmem + (NCH / 2) * 16, pk2);
 #pragma unroll
         for (int c = NCH / 2 + 1; c < NCH; ++c) {
@@ -654,11 +622,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         unpack_f32x2(sum_b, sb0, sb1);
         delta = delta * alpha + ((sa0 + sa1) + (sb0 + sb1));
         m_run = m_new;
-        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 5);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar_h);
-        if ((warp & 3) == 0) ATTN_TRACE_EVENT(i, (int)g, 6);
               return true;
       };
       for (int jj = 0; ok && jj < n; ++jj, ++g) {
@@ -678,7 +644,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       // ----------------------------------------------------- end of segment
       // Each warp finishes its own 32 rows without meeting the other warps of its warpgroup.
-      if (warp == 0) ATTN_TRACE_MARK(3);
       if constexpr (CLUSTER) {
         // The peers' barriers exist (arrival at kernel start).  Two parts: what a CTA receives lands in its Q
         // buffer, which is dead one step before the end -- its peers may be told so right away.
@@ -694,7 +659,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (ok) ok = wait_bar_warp(smem_u32(&misc->o_full[i]), (g - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, g));
       if (!ok) break;
       tc_fence_after();
-      if (warp == 0) ATTN_TRACE_MARK(4);
       const int wq = warp & 3;                               // which 32 rows of the sub-tile
       // This warp's staging: [32 rows][64 columns] bf16 chunks.  Before the CTA's last segment there is one
       // (the next Q tile may already be arriving in the Q buffer) and the two halves of a 128-wide row take
@@ -771,7 +735,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                   !wait_bar_warp(smem_u32(&misc->o_full[1 - i]), (g - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, 0x2000 | g))) { ok = false; break; }
               if (warp == 0 && lane < k && lane != mine) mbar_arrive_peer(map_to_cta(smem_u32(&misc->peers_ready), lane));
             }
-            if (warp == 0) ATTN_TRACE_MARK(5);
             // landing area of part `src` (index among the k-1 other parts) of this warp's rows, as local addresses
             auto o_land = [&](int src) -> uint32_t {
               return q_land ? q_smem + (uint32_t)ms * (32 * D * 4) : ring_smem + (uint32_t)(ms * (k - 1) + src) * kPartBytes;
@@ -803,7 +766,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               mbar_arrive(smem_u32(&misc->o_free[i]));
             } else {
               if (!wait_bar_warp(smem_u32(&misc->data_ready[warp][0]), 0, abort_flag, wait_info(kRoleSoftmax, kBarSync, 0x5000 | (uint32_t)warp))) { ok = false; break; }
-              if (warp == 0) ATTN_TRACE_MARK(6);
               // part q (ascending key order) of this warp's rows: own part in tensor memory, the others landed
               auto part = [&](int q) -> const float* {           // O of part q: [column / 4][lane] float4
                 return reinterpret_cast<const float*>(smem_raw + (o_land(q < mine ? q : q - 1) - smem_base));
@@ -902,7 +864,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           order = __shfl_sync(0xffffffffu, order, 0);
           merges = (order == (uint32_t)(parts - 1));
         }
-        if (warp == 0) ATTN_TRACE_MARK(5);
         if (!merges) {
           write_partial();
           tc_fence_before();
@@ -920,7 +881,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               __nanosleep(100);                              // the publishers update this cache line: poll gently
             }
             if (!seen && !*abort_flag) {
-              report_timeout(wait_info(kRoleSoftmax, kBarSync, 0x7000 | (uint32_t)wq));
+              report_timeout(wait_info(kRoleSoftmax, kBarSync, 0x7000 | (uint32_t)wq), abort_flag);
               *abort_flag = 1;
             }
           }
@@ -928,7 +889,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (!seen) { ok = false; break; }
           __threadfence();
           if (lane == 0) { ctr[0] = 0u; ctr[1] = 0u; }       // ready for the next launch
-          if (warp == 0) ATTN_TRACE_MARK(6);
           // part sp comes from CTA c_first + sp: its first piece if its range starts inside this tile
           auto part_ptr = [&](int sp) -> const float* {
             const int c = c_first + sp;
@@ -1247,18 +1207,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (!wait_bar_warp(smem_u32(&misc->o_free[i]), (seg - 1) & 1, abort_flag, wait_info(kRoleMma, kBarOFull, 0x8000 | seg))) { ok = false; break; }
           }
           tc_fence_after();
-          ATTN_TRACE_EVENT(3, (int)g, i * 4 + 0);
           if (elect_one()) {
             issue_pv<D, TKV>(o_acc, s_acc, v_smem, jj > 0, TKV * 128, 1024, 0, TKV / 32);
-#ifdef ATTN_TRACE
-            umma_commit(smem_u32(&misc->dbg_bar[i]));
-#endif
           }
           __syncwarp();
-          ATTN_TRACE_EVENT(3, (int)g, i * 4 + 1);
           if (!wait_bar_warp(smem_u32(&misc->p_half[i]), g & 1, abort_flag, wait_info(kRoleMma, kBarPFull, 0x8000 | g))) { ok = false; break; }
           tc_fence_after();
-          ATTN_TRACE_EVENT(3, (int)g, i * 4 + 2);
           if (more && i == 0) {
             if (!wait_bar_warp(smem_u32(&misc->kv_full[k_stage]), k_phase, abort_flag, wait_info(kRoleMma, kBarKvFull, g))) { ok = false; break; }
             tc_fence_after();
@@ -1279,7 +1233,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
           }
           __syncwarp();
-          ATTN_TRACE_EVENT(3, (int)g, i * 4 + 3);
         }
       }
       if (!ok) break;
@@ -1351,7 +1304,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   } else {
     setmaxnreg_dec<64>();
   }
-  if (warp == 0) ATTN_TRACE_MARK(7);
   tc_fence_before();
   __syncthreads();
   if constexpr (CLUSTER) {
@@ -1363,28 +1315,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
   }
-  if (threadIdx.x == 0) ATTN_TRACE_MARK(8);
-  ATTN_TRACE_CTA(1);
 }
 
 // ---------------------------------------------------------------------------
 // Non-pipelined kernel: one 128-row Q tile per CTA, 128 threads, one K/V stage,
-// every phase separated by a barrier.  dbg_flags bit 0 swaps the two byte
-// offsets of the V descriptor (layout diagnosis only).
+// every phase separated by a barrier.
 // ---------------------------------------------------------------------------
 struct SimpleMisc {
   uint64_t load_bar;
   uint64_t mma_bar;
   uint64_t sync_bar;   // bounded replacement for a CTA-wide barrier inside the loop
+  AbortCell abort;
   uint32_t tmem_slot;
-  int abort_flag;
 };
 
 template <int D, int TKV>
 __global__ void __launch_bounds__(128, 1)
 attn_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, int L,
-                       float scale_log2, float* __restrict__ scores_out, int dbg_flags) {
+                       float scale_log2, float* __restrict__ scores_out) {
   constexpr int KCH = D / 64;
   constexpr int TMEM_COLS = (TKV + D <= 128) ? 128 : 256;
   constexpr int Q_BYTES = kSub * D * 2;
@@ -1393,7 +1342,7 @@ attn_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t smem_base = smem_u32(smem_raw);
   const uint32_t q_smem = smem_base, k_smem = smem_base + Q_BYTES, v_smem = k_smem + KV_BYTES;
   SimpleMisc* misc = reinterpret_cast<SimpleMisc*>(smem_raw + Q_BYTES + 2 * KV_BYTES);
-  volatile int* abort_flag = &misc->abort_flag;
+  volatile int* abort_flag = &misc->abort.flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = threadIdx.x;
   const int q_row0 = blockIdx.x * kSub;
@@ -1404,8 +1353,11 @@ attn_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t bar_sync = smem_u32(&misc->sync_bar);
 
   if (threadIdx.x == 0) {
-    misc->abort_flag = (smem_base & 1023u) ? 1 : 0;
-    if (smem_base & 1023u) report_timeout(wait_info(kRoleSimple, 0, 0xFFFF));
+    abort_cell_init(&misc->abort, nullptr);
+    if (smem_base & 1023u) {
+      report_timeout(wait_info(kRoleSimple, 0, 0xFFFF), abort_flag);
+      misc->abort.flag = 1;
+    }
     mbar_init(bar_load, 1);
     mbar_init(bar_mma, 1);
     mbar_init(bar_sync, kSub);
@@ -1421,8 +1373,7 @@ attn_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t tmem_base = misc->tmem_slot;
   const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
   const uint32_t s_tmem = lane_base, o_tmem = lane_base + TKV;
-  const uint32_t lbo = (dbg_flags & 1) ? 1024u : (uint32_t)(TKV * 128);
-  const uint32_t sbo = (dbg_flags & 1) ? (uint32_t)(TKV * 128) : 1024u;
+  const uint32_t lbo = (uint32_t)(TKV * 128), sbo = 1024u;   // V as MN-major B: next 64-column chunk, next 8 key rows
 
   float m_run = -INFINITY, delta = 0.f;
   uint32_t ph_load = 0, ph_mma = 0;

@@ -31,19 +31,10 @@ constexpr int kOutRowBytes = 128;     // output staging: per softmax warpgroup o
 constexpr int kMaxStages = 8;
 constexpr int kMinStages = 4;         // K_j, V_j and one of each in flight
 constexpr int kMinTileKv = 32;
-constexpr int kMinStepsPerSplit = 4;
-constexpr int kSegmentOverheadSteps = 3;  // Q load + first product + partial write/merge, in units of one KV step
-constexpr int kCtaOverheadSteps = 2;      // start and end of a CTA that handles one whole Q tile
-constexpr int kTransitionSteps = 1;       // a persistent CTA moving on to its next Q tile
-// Under-occupied grids (fewer Q tiles than units): cost of the end of a CTA's work in KV steps, measured on B200 --
+constexpr int kMinStepsPerSplit = 4;          // least KV steps of a CTA whose partial goes through the workspace
 constexpr int kMinStepsPerClusterSplit = 2;
-constexpr int kClusterOverheadSteps = 5;     // k CTAs per tile as one cluster: partials through distributed shared memory
-constexpr int kWorkspaceOverheadSteps = 8;   // k CTAs per tile, partials through the workspace (plus k / 2: parts to merge)
-constexpr int kBalancedOverheadSteps = 12;   // equal ranges of the unit line: two partial pieces per CTA, staggered merges
 constexpr int kLandingPartExtra = 256;       // m and delta of the 32 rows of one part
 constexpr int kCausalTileCostUnits = 3;      // cost units that precede every causal tile on the unit line (kernel constant)
-constexpr int kCausalRangesOverheadSteps = 15;   // causal, equal ranges: many short pieces per CTA, merges through the workspace
-constexpr int kCausalPairsOverheadSteps = 6;     // causal, k CTAs per tile as one cluster
 
 inline int floor_to(int x, int m) { return (x / m) * m; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -78,29 +69,29 @@ long long attn_internal::head_units(int q_tiles, int steps, int ratio, int causa
   return (long long)ratio * qc * (qc + 1) / 2 + (long long)(q_tiles - qc) * steps;
 }
 
-// Occupancy step of the derivation (shared with the tile-override path of the launcher).
-int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int steps, int ratio, int causal,
-                             long long kv_bytes_per_head, int groups, int part_floats_per_row, long long ring_bytes) {
+// Occupancy step of the derivation (shared with the tile-override path of the launcher).  Every candidate's cost is
+// KV steps on the longest CTA's path plus the descriptor's measured cost of that candidate's start and end.
+attn_internal::Grid attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int steps, int ratio, int causal,
+                                             long long kv_bytes_per_head, int groups, int part_floats_per_row,
+                                             long long ring_bytes) {
   const long long tiles_ll = (long long)heads * q_tiles;
   const long long total = (long long)heads * head_units(q_tiles, steps, ratio, causal);
+  const long long part_bytes = 32LL * 4 * part_floats_per_row + kLandingPartExtra;
   if (causal) {
     // Equal ranges of the unit line (every tile preceded by kCausalTileCostUnits cost units, as in the kernel), or -- few
     // and short tiles -- k = 2..4 CTAs per tile as one cluster, each with a share of the tile's own key steps: the
-    // longest tile then sets the time, but a CTA has one piece instead of many short ones.  Costs in KV steps, measured.
+    // longest tile then sets the time, but a CTA has one piece instead of many short ones.
     long long g = total / kMinStepsPerSplit;
     if (g > h.num_units) g = h.num_units;
     if (g < 1) g = 1;
-    const long long cost_ranges = (total + kCausalTileCostUnits * tiles_ll + g - 1) / g + kCausalRangesOverheadSteps;
-    long long best = cost_ranges;
-    int ctas = (int)g;
+    Grid best = {(int)g, (total + kCausalTileCostUnits * tiles_ll + g - 1) / g + h.ovh_causal_ranges};
     for (int k = 2; k <= 4 && ratio >= 2; ++k) {
       if (k * tiles_ll > h.num_units || h.max_clusters[k - 1] < tiles_ll || ceil_div(steps, k) < 2) continue;
-      const long long landing = (long long)ceil_div(groups, k) * (k - 1) * (32LL * 4 * part_floats_per_row + kLandingPartExtra);
-      if (k > 2 && landing > ring_bytes) continue;
-      const long long cost = ceil_div(steps, k) + kCausalPairsOverheadSteps;
-      if (cost < best) { best = cost; ctas = (int)(k * tiles_ll); }
+      if (k > 2 && (long long)ceil_div(groups, k) * (k - 1) * part_bytes > ring_bytes) continue;
+      const long long cost = ceil_div(steps, k) + h.ovh_causal_cluster;
+      if (cost < best.cost) best = {(int)(k * tiles_ll), cost};
     }
-    return ctas;
+    return best;
   }
   const int tiles = (int)tiles_ll;
   if (tiles_ll >= h.num_units) {
@@ -108,28 +99,26 @@ int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int 
     // empty, and every CTA pays its own start and end.  One persistent CTA per unit with an equal range
     // of the unit line has neither cost but works on `units` different places at once: it is taken only
     // when the K and V of the heads then in flight stay in two thirds of the cache.
-    const long long waves = (tiles_ll + h.num_units - 1) / h.num_units;
-    const long long cost_tiles = waves * (steps + kCtaOverheadSteps);
     const long long g = h.num_units;
-    const long long cost_balanced = (total + g - 1) / g + 2 * kSegmentOverheadSteps + ((tiles_ll + g - 1) / g) * kTransitionSteps;
+    const long long waves = (tiles_ll + g - 1) / g;
+    const long long cost_tiles = waves * (steps + h.ovh_whole_tile);
+    const long long cost_balanced = (total + g - 1) / g + h.ovh_persistent + waves * h.ovh_tile_change;
     const long long heads_in_flight = heads < g ? heads : g;
     const bool cached = h.cache_bytes > 0 && 3 * heads_in_flight * kv_bytes_per_head <= 2 * (long long)h.cache_bytes;
-    if (cached && cost_balanced < cost_tiles) return (int)g;
-    return (int)tiles_ll;
+    if (cached && cost_balanced < cost_tiles) return {(int)g, cost_balanced};
+    return {tiles, cost_tiles};
   }
-  // Fewer tiles than units: k CTAs per tile along the key axis, or equal ranges of the unit line.  Costs in KV steps
-  // per CTA; the cheapest wins, ties go to the earlier candidate.
-  int ctas = tiles;                                          // one CTA per tile, nothing to merge
-  long long best = steps + kCtaOverheadSteps;
+  // Fewer tiles than units: k CTAs per tile along the key axis, or equal ranges of the unit line.  The cheapest wins,
+  // ties go to the earlier candidate.
+  Grid best = {tiles, steps + h.ovh_whole_tile};             // one CTA per tile, nothing to merge
   // (1) k CTAs per tile as one cluster: the tile's clusters must all be resident, every CTA needs a few steps, and
   // what a CTA receives must fit its landing area -- for two parts the Q buffer, else the K/V ring: the 32-row
   // groups one CTA merges, times the k-1 parts of each.
   for (int k = 2; k <= 8; ++k) {
     if ((long long)tiles * k > h.num_units || steps / k < kMinStepsPerClusterSplit || h.max_clusters[k - 1] < tiles) continue;
-    const long long landing = (long long)ceil_div(groups, k) * (k - 1) * (32LL * 4 * part_floats_per_row + kLandingPartExtra);
-    if (k > 2 && landing > ring_bytes) continue;
-    const long long cost = ceil_div(steps, k) + kClusterOverheadSteps;
-    if (cost < best) { best = cost; ctas = tiles * k; }
+    if (k > 2 && (long long)ceil_div(groups, k) * (k - 1) * part_bytes > ring_bytes) continue;
+    const long long cost = ceil_div(steps, k) + h.ovh_cluster;
+    if (cost < best.cost) best = {tiles * k, cost};
   }
   // (2) k CTAs per tile, partials through the workspace
   {
@@ -137,8 +126,8 @@ int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int 
     const int k_max = steps / kMinStepsPerSplit;
     if (k > k_max) k = k_max;
     if (k >= 2) {
-      const long long cost = ceil_div(steps, k) + kWorkspaceOverheadSteps + k / 2;
-      if (cost < best) { best = cost; ctas = tiles * k; }
+      const long long cost = ceil_div(steps, k) + h.ovh_workspace + k / 2;
+      if (cost < best.cost) best = {tiles * k, cost};
     }
   }
   // (3) equal ranges
@@ -146,11 +135,11 @@ int attn_internal::grid_size(const attn_hw_desc& h, int heads, int q_tiles, int 
     long long g = total / kMinStepsPerSplit;
     if (g > h.num_units) g = h.num_units;
     if (g > tiles) {
-      const long long cost = (total + g - 1) / g + kBalancedOverheadSteps;
-      if (cost < best) { best = cost; ctas = (int)g; }
+      const long long cost = (total + g - 1) / g + h.ovh_ranges;
+      if (cost < best.cost) best = {(int)g, cost};
     }
   }
-  return ctas;
+  return best;
 }
 
 namespace {
@@ -225,19 +214,17 @@ void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int Lk, int d
   }
 
   // 3. Occupancy: blocks against compute units.  With fewer Q tiles than units the key axis is shared
-  //    out in one of two ways, whichever has the shorter critical path (counted in KV steps, a segment
-  //    start/finish costing kSegmentOverheadSteps):
-  //      uniform   k = floor(units / tiles) CTAs per Q tile, each one contiguous piece of its tile;
-  //      balanced  min(units, tiles*steps/kMinStepsPerSplit) CTAs with equal ranges of the
-  //                tiles*steps line, which may straddle one tile boundary (two pieces).
+  //    out in whichever way has the shortest critical path, counted in KV steps plus the descriptor's
+  //    measured cost of the start and end of a CTA's work under that way (see grid_size).
   //    Q tiles shared by several CTAs are merged with the merge operator of the online softmax.
   const int tile_q = n_q * sub;
   const int tiles = B * H * ceil_div(L, tile_q);
   const int steps = ceil_div(Lk, tile_kv);
   const int under = tiles < h.num_units;
   // (4 n_q groups of 32 rows per tile; a part of one group is 32 rows of d fp32 values plus statistics)
-  const int ctas = attn_internal::grid_size(h, B * H, ceil_div(L, tile_q), steps, tile_q / tile_kv, causal,
-                                             2LL * Lk * d * h.elem_bytes, 4 * n_q, d, (long long)stages * stage);
+  const attn_internal::Grid grid = attn_internal::grid_size(h, B * H, ceil_div(L, tile_q), steps, tile_q / tile_kv, causal,
+                                                            2LL * Lk * d * h.elem_bytes, 4 * n_q, d, (long long)stages * stage);
+  const int ctas = grid.ctas;
   const int kv_splits = ceil_div(ctas, tiles);
 
   t->feasible = 1;
@@ -260,6 +247,17 @@ void plan_tmem_machine(const attn_hw_desc& h, int B, int H, int L, int Lk, int d
   t->wave_efficiency = (float)((double)t->ctas / ((double)waves * h.num_units));
   t->under_occupied = under;
   t->causal = causal ? 1 : 0;
+  t->cost_steps = (int32_t)(grid.cost > 0x7FFFFFFFLL ? 0x7FFFFFFFLL : grid.cost);
+  // Predicted time: the longest CTA's path at the per-unit share of the tensor peak against the compulsory HBM
+  // traffic (Q, K, V read once, O written once) at the HBM bandwidth.
+  if (h.peak_tflops > 0.0 && h.hbm_gbps > 0.0) {
+    const double step_flops = 4.0 * tile_q * tile_kv * d;     // both products of one KV step
+    const double t_tensor_us = (double)grid.cost * step_flops / (h.peak_tflops / h.num_units * 1e6);
+    const double bytes = 2.0 * B * H * ((double)L + Lk) * d * h.elem_bytes;
+    const double t_hbm_us = bytes / (h.hbm_gbps * 1e3);
+    t->bound = t_hbm_us > t_tensor_us ? 1 : 0;
+    t->predicted_us = (float)(t_hbm_us > t_tensor_us ? t_hbm_us : t_tensor_us);
+  }
 }
 
 }  // namespace
@@ -286,9 +284,18 @@ extern "C" int attn_hw_desc_b200(attn_hw_desc* out) {
   }
   out->elem_bytes = 2;
   out->cache_bytes = 126 << 20;   // L2
-  out->hbm_gbps = 7700.0;
-  out->peak_tflops = 2250.0;
-  out->sm_clock_mhz = 1965.0;
+  // start and end of a CTA's work under each way of sharing out the key axis, in KV steps (measured on B200;
+  // a KV step of 256 query rows x 128 keys x 128 takes about 1.7 us)
+  out->ovh_whole_tile = 2;
+  out->ovh_cluster = 5;
+  out->ovh_workspace = 8;
+  out->ovh_ranges = 12;
+  out->ovh_persistent = 6;
+  out->ovh_tile_change = 1;
+  out->ovh_causal_ranges = 15;
+  out->ovh_causal_cluster = 6;
+  out->hbm_gbps = 7700.0;      // nominal (HGX B200)
+  out->peak_tflops = 2250.0;   // nominal dense bf16: 8192 FLOP per clock per SM at 1.86 GHz
   return ATTN_OK;
 }
 

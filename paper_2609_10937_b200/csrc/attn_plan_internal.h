@@ -12,8 +12,10 @@ namespace attn_internal {
 // that many clusters can be resident; else through the workspace) and equal ranges of the unit line.
 // Non-causal, more tiles than units: one CTA per tile, or one persistent CTA per unit walking an
 // equal range of the (tile, step) line when that is cheaper and the K/V of the heads in flight fit the cache.
-// Causal (tiles need unequal numbers of steps): always equal ranges of the unit line, one per unit.
-int grid_size(const attn_hw_desc& h, int heads, int q_tiles, int steps, int ratio, int causal,
+// Causal (tiles need unequal numbers of steps): equal ranges of the unit line, or k = 2..4 CTAs per tile as one cluster.
+// Returns the grid and its cost: KV steps on the longest CTA's path plus the descriptor's ovh_* term of the winner.
+struct Grid { int ctas; long long cost; };
+Grid grid_size(const attn_hw_desc& h, int heads, int q_tiles, int steps, int ratio, int causal,
               long long kv_bytes_per_head, int groups, int part_floats_per_row, long long ring_bytes);
 // The derivation for Lq query rows and Lk keys per head (attn_plan_ex is the case Lq == Lk).
 int plan_qk(const attn_hw_desc* desc, int B, int H, int Lq, int Lk, int d, int causal, attn_tiles* out);

@@ -47,8 +47,8 @@ struct GemmMisc {
   uint64_t acc_full;      // all products of a tile have finished
   uint64_t acc_empty;     // the epilogue has read the accumulators of a tile
   uint64_t epi_sync[2];   // rendezvous of the four epilogue warps of a sub-tile
+  attn::AbortCell abort;
   uint32_t tmem_slot;
-  int abort_flag;
 };
 static_assert(sizeof(GemmMisc) <= kMiscBytes, "misc region too large");
 
@@ -64,15 +64,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
   const uint32_t smem_base = smem_u32(smem_raw);
   const uint32_t out_smem = smem_base + p.stages * kStageBytes;
   GemmMisc* misc = reinterpret_cast<GemmMisc*>(smem_raw + p.stages * kStageBytes + kOutBytes);
-  volatile int* abort_flag = &misc->abort_flag;
+  volatile int* abort_flag = &misc->abort.flag;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    misc->abort_flag = 0;
+    attn::abort_cell_init(&misc->abort, nullptr);
     if (smem_base & 1023u) {
-      attn::report_timeout(attn::wait_info(kRoleGemmLoad, 0, 0xFFFF));
-      misc->abort_flag = 1;
+      attn::report_timeout(attn::wait_info(kRoleGemmLoad, 0, 0xFFFF), abort_flag);
+      misc->abort.flag = 1;
     }
     for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(smem_u32(&misc->full[s]), 1);

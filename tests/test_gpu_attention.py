@@ -521,6 +521,117 @@ def test_other_descriptors_run_with_no_code_change(env, field, value, expect):
                      rows=synth.sample_rows(case.L), causal=True)
 
 
+def test_changed_cost_constants_change_the_grid_and_the_launch_follows(env):
+    """The occupancy step reads its cost constants from the descriptor: with the two ways of splitting a tile made
+    expensive and equal ranges made cheap, eight heads of 2048 keys no longer run as 64 clusters of two but as one
+    range per SM through the workspace -- same kernels, same result within tolerance."""
+    torch, _, binding = env
+    case = _case("ovh", 1, 8, 2048, 128)
+    desc = binding.hw_desc_query(0)
+    base = binding.plan(desc, case.B, case.H, case.L, case.d)
+    assert base.ctas == 2 * base.tiles == 128
+    _run_and_compare(env, case, lambda a, b, c: binding.forward_desc(desc, a, b, c), rows=synth.sample_rows(case.L))
+    assert binding.last_cluster_size() == 2
+    desc.ovh_cluster, desc.ovh_workspace, desc.ovh_ranges = 40, 40, 10
+    plan = binding.plan(desc, case.B, case.H, case.L, case.d)
+    assert plan.ctas == desc.num_units and plan.cost_steps == -(-64 * 16 // desc.num_units) + 10
+    _run_and_compare(env, case, lambda a, b, c: binding.forward_desc(desc, a, b, c), rows=synth.sample_rows(case.L))
+    assert binding.last_cluster_size() == 0
+
+
+def test_uniform_split_larger_than_the_machine_is_merged_by_the_last_finisher(env):
+    """Fixed merge roles make a merging warp wait for the other CTAs of its tile, so they need every CTA resident.  A
+    uniform split with more CTAs than SMs (an override; the closed form never asks for one) runs the instantiation in
+    which the last CTA of a tile to finish merges: correct, and no wait runs out."""
+    torch, _, binding = env
+    case = _case("big_uniform", 1, 8, 2048, 128)                 # 64 Q tiles
+    for k in (3, 4):                                             # 192 and 256 CTAs on 148 SMs
+        _run_and_compare(env, case, lambda a, b, c: binding.forward_tiles(a, b, c, kv_splits=k),
+                         rows=synth.sample_rows(case.L), what=f"{k} CTAs per tile")
+        assert binding.last_cluster_size() == 0
+
+
+def test_per_call_workspaces_let_two_streams_run_split_plans_at_once(env):
+    """attn_forward_ws: two streams of one device, each with its own workspace and status words, run plans that share
+    Q tiles at the same time; results equal the ordinary entry point bit for bit and the oracle within tolerance."""
+    torch, orc, binding = env
+    desc = binding.hw_desc_query(0)
+    # one range per SM (the last CTA of a tile to finish merges) and three CTAs per tile that cannot run as clusters
+    cases = [_case("ws_a", 1, 1, 16384, 128, cfg_id=81), _case("ws_b", 1, 3, 4096, 128, cfg_id=82)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    work = []
+    for case, st in zip(cases, streams):
+        plan = binding.plan(desc, case.B, case.H, case.L, case.d)
+        need = binding.workspace_bytes(plan, case.B, case.H, case.L, case.d)
+        assert need > 65536
+        q, k, v = synth.make_qkv(case, seed=3)
+        t = [to_cuda_bf16(x) for x in (q, k, v)]
+        ws = torch.empty(need, dtype=torch.uint8, device="cuda").fill_(0xAB)       # dirty: the init call must clear it
+        status = torch.full((4,), 7, dtype=torch.int32, device="cuda")
+        work.append(dict(case=case, host=(q, k, v), dev=t, ws=ws, status=status, stream=st,
+                         out=torch.full_like(t[0], float("nan"))))
+    torch.cuda.synchronize()
+    for w in work:
+        with torch.cuda.stream(w["stream"]):
+            binding.workspace_init(w["ws"], w["status"])
+    for rep in range(3):                                         # interleaved launches on the two streams
+        for w in work:
+            with torch.cuda.stream(w["stream"]):
+                binding.forward_ws(*w["dev"], w["out"], workspace=w["ws"], status=w["status"])
+                assert binding.last_cluster_size() == 0
+    for w in work:
+        with torch.cuda.stream(w["stream"]):
+            code, detail = binding.status_read(w["status"], w["ws"])
+        assert code == 0 and detail == [0, 0, 0, 0]
+    torch.cuda.synchronize()
+    for w in work:
+        case = w["case"]
+        want = binding.forward(*w["dev"])
+        torch.cuda.synchronize()
+        assert torch.equal(w["out"].view(torch.int16), want.view(torch.int16))
+        rows = synth.sample_rows(case.L)
+        ref = orc.attention_rows(*w["host"], case.B, case.H, case.L, case.d, rows)
+        got = to_host_f64(w["out"]).reshape(case.B * case.H, case.L, case.d)
+        assert_close(got[:, rows], ref, case.name)
+    # too small a buffer is refused before any launch; no workspace is fine for a plan that needs none
+    w = work[0]
+    with pytest.raises(binding.AttnError) as err:
+        binding.forward_ws(*w["dev"], w["out"], workspace=w["ws"][:70000], status=w["status"])
+    assert err.value.code == binding.ERR_NEED_WORKSPACE and binding.last_launch_count() == 0
+    small = _case("ws_none", 4, 40, 512, 64)
+    tq, tk, tv = (to_cuda_bf16(x) for x in synth.make_qkv(small, 0))
+    a = binding.forward_ws(tq, tk, tv)
+    b = binding.forward(tq, tk, tv)
+    torch.cuda.synchronize()
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+def test_bounded_wait_expiry_is_recorded_in_the_callers_status_words(env):
+    """A launch given its own status words reports an expired wait there, not in the device-wide record.  The wait that
+    runs out is the self-test's (one warp on a barrier nothing arrives at; it ends by itself at the cycle limit)."""
+    torch, _, binding = env
+    assert binding.last_device_status()[0] == 0
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    other = torch.zeros(4, dtype=torch.int32, device="cuda")
+    case = _case("ws_status", 1, 1, 4096, 128)
+    plan = binding.plan(binding.hw_desc_query(0), case.B, case.H, case.L, case.d)
+    ws = torch.zeros(binding.workspace_bytes(plan, case.B, case.H, case.L, case.d), dtype=torch.uint8, device="cuda")
+    tq, tk, tv = (to_cuda_bf16(x) for x in synth.make_qkv(case, 0))
+    stream = torch.cuda.current_stream().cuda_stream
+    rc = binding.lib().attn_selftest_wait_expiry_to(status.data_ptr(), stream)
+    assert rc == 0
+    out = binding.forward_ws(tq, tk, tv, workspace=ws, status=other)        # a normal launch with other status words
+    code, detail = binding.status_read(status, None)
+    assert code == binding.ERR_DEVICE_TIMEOUT
+    assert detail[0] == 1 and detail[1] == (5 << 24) | (10 << 16) | 0x7E57 and detail[2] == 0
+    assert binding.status_read(status, None) == (0, [0, 0, 0, 0])            # reported once, then cleared
+    assert binding.status_read(other, ws) == (0, [0, 0, 0, 0])               # the other launch saw nothing
+    assert binding.last_device_status()[0] == 0                              # nor did the device-wide record
+    want = binding.forward(tq, tk, tv)
+    torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.int16), want.view(torch.int16))
+
+
 def test_descriptor_of_a_larger_machine_is_refused(env):
     torch, _, binding = env
     desc = binding.hw_desc_query(0)

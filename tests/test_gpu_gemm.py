@@ -145,6 +145,11 @@ def test_unfused_entry_points_refuse_bad_arguments(env):
     with pytest.raises(binding.AttnError) as err:
         binding.softmax_rows(s, 1.0)
     assert err.value.code == -2
+    ok = torch.zeros(4, 128, dtype=torch.bfloat16, device="cuda")
+    for bad_scale in (0.0, -0.5, float("inf"), float("nan")):           # the row maximum is taken before scaling
+        with pytest.raises(binding.AttnError) as err:
+            binding.softmax_rows(ok, bad_scale)
+        assert err.value.code == -1
     q = torch.zeros(1, 1, 256, 64, dtype=torch.bfloat16, device="cuda")
     small = torch.empty(10, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(binding.AttnError) as err:                       # score buffer too small

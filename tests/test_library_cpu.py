@@ -81,9 +81,10 @@ def test_plan_for_separate_query_and_key_lengths(binding):
 
 def test_struct_sizes_match_the_header(binding):
     d = binding.hw_desc_b200()
-    assert d.struct_bytes == ctypes.sizeof(binding.AttnHwDesc) == 112
-    assert ctypes.sizeof(binding.AttnTiles) == 72
-    assert binding.AttnTiles.causal.offset == 68
+    assert d.struct_bytes == ctypes.sizeof(binding.AttnHwDesc) == 136
+    assert ctypes.sizeof(binding.AttnTiles) == 84
+    assert binding.AttnTiles.causal.offset == 68 and binding.AttnTiles.predicted_us.offset == 80
+    assert binding.AttnHwDesc.hbm_gbps.offset == 120
 
 
 def _desc_dict(d):
@@ -102,15 +103,65 @@ def test_b200_plan_equals_oracle_restatement(binding):
         if not ref["feasible"]:
             continue
         for key in ("tile_q", "tile_kv", "n_q", "n_s", "kv_stages", "kv_splits", "smem_bytes", "tmem_columns",
-                    "regs_softmax", "threads", "tiles", "ctas"):
+                    "regs_softmax", "threads", "tiles", "ctas", "cost_steps"):
             assert getattr(got, key) == ref[key], (key, B, H, L, d)
         assert bool(got.under_occupied) == ref["under_occupied"]
         assert got.wave_efficiency == pytest.approx(ref["wave_efficiency"], rel=1e-6)
         assert got.ctas_per_unit == pytest.approx(ref["ctas_per_unit"], rel=1e-6)
         gc = binding.plan(desc, B, H, L, d, causal=True)
         rc = po.derive_tiles_tmem_machine(dd, B, H, L, d, causal=True)
-        assert (gc.feasible, gc.causal, gc.tile_q, gc.tile_kv, gc.kv_stages, gc.ctas) == (
-            1, 1, rc["tile_q"], rc["tile_kv"], rc["kv_stages"], rc["ctas"]), (B, H, L, d)
+        assert (gc.feasible, gc.causal, gc.tile_q, gc.tile_kv, gc.kv_stages, gc.ctas, gc.cost_steps) == (
+            1, 1, rc["tile_q"], rc["tile_kv"], rc["kv_stages"], rc["ctas"], rc["cost_steps"]), (B, H, L, d)
+
+
+def test_occupancy_step_follows_the_descriptor_cost_constants(binding):
+    """The occupancy step of the C planner against the oracle's candidate table for descriptors whose cost constants,
+    unit counts and resident-cluster counts are drawn at random: the grid and its cost must be the first cheapest
+    eligible candidate whatever the constants are -- the rule, not the B200 values, is what is compared here."""
+    import numpy as np
+
+    rng = np.random.default_rng(11)
+    ovh = ("ovh_whole_tile", "ovh_cluster", "ovh_workspace", "ovh_ranges", "ovh_persistent", "ovh_tile_change",
+           "ovh_causal_ranges", "ovh_causal_cluster")
+    for _ in range(40):
+        desc = binding.hw_desc_b200()
+        desc.num_units = int(rng.integers(8, 200))
+        for k in range(8):
+            desc.max_clusters[k] = max(0, desc.num_units // (k + 1) - int(rng.integers(0, 3)))
+        desc.cache_bytes = int(rng.integers(0, 3)) * (63 << 20)
+        for name in ovh:
+            setattr(desc, name, int(rng.integers(0, 24)))
+        dd = _desc_dict(desc)
+        for B, H, L, d in [(1, 1, 1024, 128), (1, 8, 2048, 128), (1, 1, 16384, 128), (2, 3, 1500, 64), (1, 40, 4096, 128),
+                           (4, 32, 4096, 64), (1, 2, 8192, 128), (1, 5, 640, 64), (1, 3, 3000, 128)]:
+            for causal in (False, True):
+                got = binding.plan(desc, B, H, L, d, causal=causal)
+                ref = po.derive_tiles_tmem_machine(dd, B, H, L, d, causal=causal)
+                assert (got.ctas, got.cost_steps, got.kv_splits) == (ref["ctas"], ref["cost_steps"], ref["kv_splits"]), \
+                    (B, H, L, d, causal, dd)
+    # a constant changed in the descriptor changes the grid: the B200 pick for eight heads of 2048 keys is 64 clusters of 2
+    desc = binding.hw_desc_b200()
+    assert binding.plan(desc, 1, 8, 2048, 128).ctas == 128
+    desc.ovh_cluster = desc.ovh_workspace = 40          # both ways of splitting a tile made expensive:
+    assert binding.plan(desc, 1, 8, 2048, 128).ctas == 64      # whole tiles (16 + 2) beat equal ranges (7 + 12)
+    desc.ovh_ranges = 10
+    assert binding.plan(desc, 1, 8, 2048, 128).ctas == 148     # ... until equal ranges get cheaper (7 + 10)
+
+
+def test_predicted_time_and_bound(binding):
+    """attn_plan's predicted time: the longest CTA's path at the per-unit share of the descriptor's tensor peak against
+    the compulsory HBM traffic at its bandwidth (the roofline the derivation's hardware model implies)."""
+    desc = binding.hw_desc_b200()
+    t = binding.plan(desc, 1, 1, 16384, 128)
+    step_flops = 4.0 * t.tile_q * t.tile_kv * 128
+    want = t.cost_steps * step_flops / (desc.peak_tflops / desc.num_units * 1e6)
+    assert t.bound == 0 and t.predicted_us == pytest.approx(want, rel=1e-5)
+    assert t.predicted_us >= 4.0 * 16384 ** 2 * 128 / (desc.peak_tflops * 1e6)      # never below the whole-machine roofline
+    desc.hbm_gbps = 1.0                                                             # a machine with almost no bandwidth
+    t = binding.plan(desc, 1, 1, 16384, 128)
+    assert t.bound == 1 and t.predicted_us == pytest.approx(4 * 16384 * 128 * 2 / 1e3, rel=1e-5)
+    desc.peak_tflops = 0.0
+    assert binding.plan(desc, 1, 1, 16384, 128).predicted_us == 0.0
 
 
 def test_other_descriptors_rerun_the_same_derivation(binding):
@@ -219,8 +270,8 @@ def test_product_does_not_reach_the_oracle():
 
 
 def test_traffic_model_matches_the_paper_figures():
-    """The product-side traffic calculator against the figures the paper prints."""
-    from paper_2609_10937_b200 import traffic
+    """The benchmark's traffic calculator against the figures the paper prints."""
+    import bench as traffic
 
     g = {row[0]: (int(row[1]), float(row[2])) for row in read_golden("paper_hbm_traffic.txt")}
     L = g["fused_mb"][0]
@@ -228,5 +279,4 @@ def test_traffic_model_matches_the_paper_figures():
     assert round(traffic.unfused_bytes(1, 1, L, 128, 4, 4) / 1e6) == g["unfused_mb"][1]
     assert round(traffic.unfused_bytes(1, 1, L, 128, 4, 4) / traffic.fused_bytes(1, 1, L, 128, 4)) == g["ratio"][1]
     assert round(traffic.unfused_bytes(1, 1, g["unfused_gb"][0], 128, 4, 4) / 1e9) == g["unfused_gb"][1]
-    assert traffic.savings(L, 128) == g["savings"][1]
     assert traffic.unfused_bytes(1, 1, L, 128, 4, 4) == po.traffic_unfused(1, 1, L, 128, 4, 4)

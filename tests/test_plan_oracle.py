@@ -1,10 +1,18 @@
 """Pins for the tile-derivation and traffic restatements under oracle/.
 
 The register-machine derivation is pinned by the numbers the paper prints
-(Table 2, the descriptor listing, the HBM-traffic paragraph); the tensor-memory
-derivation has no printed numbers and is pinned by capacity invariants.
+(Table 2, the descriptor listing, the HBM-traffic paragraph).  The tensor-memory
+derivation has no printed numbers: its capacity part is pinned by capacity
+invariants, its occupancy part by what the arithmetic fixes -- brute-force
+enumeration of the CTAs' shares on small grids, optimality and first-minimum of
+the choice over the candidate table, floors on the steps per CTA, landing areas
+inside the ring -- for the built-in descriptor and for descriptors with random
+cost constants.
 """
+import itertools
 import math
+
+import numpy as np
 
 import pytest
 
@@ -16,7 +24,10 @@ CDNA = dict(lds_bytes=64 * 1024, regs_per_thread=256, wavefront=64, atom_m=16, a
 B200 = dict(num_units=148, local_mem_bytes=232448, regs_per_unit=65536, max_regs_per_thread=255,
             simd_width=32, acc_mem_lanes=128, acc_mem_columns=512, atom_m=128, atom_n=16, atom_k=16,
             atom_n_max=256, elem_bytes=2, cache_bytes=126 << 20,
-            max_clusters=[148, 74, 45, 33, 26, 22, 15, 15])
+            max_clusters=[148, 74, 45, 33, 26, 22, 15, 15],
+            # start and end of a CTA's work under each way of sharing out the key axis, in KV steps
+            ovh_whole_tile=2, ovh_cluster=5, ovh_workspace=8, ovh_ranges=12, ovh_persistent=6, ovh_tile_change=1,
+            ovh_causal_ranges=15, ovh_causal_cluster=6)
 
 
 def test_table2_register_use_and_feasibility():
@@ -134,3 +145,105 @@ def test_tmem_machine_expected_defaults_for_the_benchmark_shapes():
     assert ctas(1, 1, 4096, 128, no_clusters) == 128   # 16 tiles x 32: eight parts through the workspace (4 + 8 + 4) = ranges (4 + 12): tie
     assert not po.derive_tiles_tmem_machine(B200, 1, 1, 1024, 72)["feasible"]          # d not a multiple of 16
     assert not po.derive_tiles_tmem_machine(B200, 1, 1, 1024, 512)["feasible"]         # d beyond the atom's N
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Occupancy step: the candidate table and the choice (Section "Tile Derivation", blocks against compute units)
+# ---------------------------------------------------------------------------------------------------------
+def _random_descriptors(n, seed=7):
+    """The B200 capacities with other cost constants, unit counts and resident-cluster counts."""
+    rng = np.random.default_rng(seed)
+    out = [B200, dict(B200, max_clusters=[0] * 8), dict(B200, num_units=74, max_clusters=[74, 37, 22, 16, 13, 11, 7, 7])]
+    for _ in range(n):
+        units = int(rng.integers(8, 200))
+        d = dict(B200, num_units=units, max_clusters=[units // k - int(rng.integers(0, 3)) for k in range(1, 9)],
+                 cache_bytes=int(rng.integers(0, 3)) * (63 << 20))
+        for key in ("ovh_whole_tile", "ovh_cluster", "ovh_workspace", "ovh_ranges", "ovh_persistent", "ovh_tile_change",
+                    "ovh_causal_ranges", "ovh_causal_cluster"):
+            d[key] = int(rng.integers(0, 24))
+        out.append(d)
+    return out
+
+
+_SHAPES = [(B, H, L, d) for B, H, L, d in itertools.product([1, 2], [1, 3, 8, 40], [128, 300, 1024, 2048, 4096, 16384],
+                                                            [64, 128])]
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_occupancy_choice_is_the_first_cheapest_eligible_candidate(causal):
+    for desc in _random_descriptors(12):
+        units = desc["num_units"]
+        for B, H, L, d in _SHAPES:
+            t = po.derive_tiles_tmem_machine(desc, B, H, L, d, causal=causal)
+            rows = t["candidates"]
+            ok = [r for r in rows if r["eligible"]]
+            assert ok, "some way of running the problem is always eligible"
+            pick = next(r for r in ok if r["ctas"] == t["ctas"] and r["cost"] == t["cost_steps"] and r["mode"] == t["mode"])
+            assert all(pick["cost"] <= r["cost"] for r in ok)                        # cheapest
+            assert not any(r["cost"] == pick["cost"] for r in ok[:ok.index(pick)])   # and the first of the cheapest
+            tiles, steps = t["tiles"], t["steps"]
+            total = tiles * steps if not causal else B * H * po.causal_head_units(-(-L // t["tile_q"]), steps,
+                                                                                  t["tile_q"] // t["tile_kv"])
+            assert 1 <= t["ctas"] <= max(tiles, units) and t["kv_splits"] == -(-t["ctas"] // tiles)
+            if t["under_occupied"] or causal:
+                assert t["ctas"] <= units or (causal and t["mode"] == "cluster")
+            # nobody's path is shorter than an even share of the work over the CTAs that exist
+            assert pick["path"] >= -(-total // max(units, t["ctas"]))
+            if not causal and t["under_occupied"]:
+                whole = next(r for r in rows if r["mode"] == "whole_tiles")
+                assert whole["eligible"] and t["cost_steps"] <= steps + desc["ovh_whole_tile"]
+            # floors on what one CTA gets, and the room for what it receives
+            if pick["mode"] == "cluster":
+                k = pick["k"]
+                assert tiles * k <= units and desc["max_clusters"][k - 1] >= tiles
+                assert (-(-steps // k) if causal else steps // k) >= 2
+                if k > 2:
+                    assert -(-(4 * t["n_q"]) // k) * (k - 1) * (32 * 4 * d + 256) <= t["ring_bytes"]
+            if pick["mode"] == "workspace":
+                assert pick["k"] >= 2 and steps // pick["k"] >= 4 and tiles * pick["k"] <= units
+            if pick["mode"] == "ranges" and not causal:
+                assert tiles < t["ctas"] <= units and total // t["ctas"] >= 4
+            if pick["mode"] == "persistent":
+                heads = min(B * H, units)
+                assert t["ctas"] == units and 3 * heads * 2 * L * d * 2 <= 2 * desc["cache_bytes"]
+
+
+def test_candidate_paths_equal_the_brute_force_shares():
+    """The `path` column against the shares counted CTA by CTA: equal ranges [c*T/G, (c+1)*T/G) of the unit line,
+    equal shares [p*s/k, (p+1)*s/k) of a tile's steps; causal tiles have min(steps, (q+1)*ratio) steps."""
+    for desc in (B200, dict(B200, num_units=40, max_clusters=[40, 20, 13, 10, 8, 6, 5, 5])):
+        for (B, H, L, d), causal in itertools.product([(1, 1, 1024, 128), (1, 3, 1500, 128), (2, 2, 2048, 64),
+                                                       (1, 5, 768, 64), (1, 1, 4096, 128), (1, 9, 640, 128)], [False, True]):
+            t = po.derive_tiles_tmem_machine(desc, B, H, L, d, causal=causal)
+            steps, q_tiles, ratio = t["steps"], -(-L // t["tile_q"]), t["tile_q"] // t["tile_kv"]
+            per_tile = [min(steps, (q + 1) * ratio) if causal else steps for q in range(q_tiles)] * (B * H)
+            assert sum(per_tile) == (B * H * po.causal_head_units(q_tiles, steps, ratio) if causal else t["tiles"] * steps)
+            for r in t["candidates"]:
+                if r["mode"] == "ranges":
+                    T = sum(per_tile) + (3 * len(per_tile) if causal else 0)     # causal: 3 cost units lead every tile
+                    G = r["ctas"]
+                    assert r["path"] == max((c + 1) * T // G - c * T // G for c in range(G))
+                elif r["mode"] in ("cluster", "workspace") and r["k"] >= 1:
+                    k = r["k"]
+                    share = lambda s: max((p + 1) * s // min(k, s) - p * s // min(k, s) for p in range(min(k, s)))
+                    assert r["path"] == max(share(s) for s in per_tile)
+                    assert r["ctas"] == k * len(per_tile)
+                elif r["mode"] == "persistent":
+                    T, G = sum(per_tile), r["ctas"]
+                    assert r["path"] == max((c + 1) * T // G - c * T // G for c in range(G))
+
+
+def test_cost_constants_steer_the_choice():
+    """A way of sharing out the keys that is made expensive in the descriptor is no longer chosen, and with every
+    cost constant zero the choice is a candidate of the shortest path."""
+    t = po.derive_tiles_tmem_machine(B200, 1, 8, 2048, 128)
+    assert t["mode"] == "cluster" and t["k"] == 2
+    assert po.derive_tiles_tmem_machine(dict(B200, ovh_cluster=40), 1, 8, 2048, 128)["mode"] != "cluster"
+    t = po.derive_tiles_tmem_machine(B200, 1, 1, 16384, 128)
+    assert t["mode"] == "ranges" and t["ctas"] == 148
+    t = po.derive_tiles_tmem_machine(dict(B200, ovh_ranges=14), 1, 1, 16384, 128)
+    assert (t["mode"], t["k"], t["ctas"]) == ("cluster", 2, 128)
+    free = dict(B200, **{k: 0 for k in B200 if k.startswith("ovh_")})
+    for B, H, L, d in _SHAPES:
+        t = po.derive_tiles_tmem_machine(free, B, H, L, d)
+        assert t["cost_steps"] == min(r["path"] for r in t["candidates"] if r["eligible"])
