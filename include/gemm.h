@@ -37,8 +37,12 @@ typedef struct gemm_tiles {
   int32_t tiles;        /* batch * ceil(M / tile_m) * ceil(N / tile_n)                           */
   int32_t ctas;         /* persistent grid: min(num_units, tiles)                                */
   int32_t feasible;     /* 1 if the kernel's tile shape fits this descriptor                     */
-  float wave_efficiency;/* tiles / (ceil(tiles / ctas) * ctas)                                   */
+  float wave_efficiency;/* tiles / (ceil(tiles / ctas) * ctas); per pair of CTAs if cta_pair == 2 */
   int32_t binding_constraint; /* attn_binding: what fixed the tile (tensor memory or ring depth) */
+  int32_t cta_pair;     /* CTAs that share one matrix instruction: 1, or 2 (a cluster of two CTAs owns a
+                           tile_m x tile_n tile, each holding half of its rows and half of B's columns)  */
+  int32_t acc_buffers;  /* accumulators that fit tensor memory: with more than one the epilogue of a tile
+                           runs under the products of the next                                        */
 } gemm_tiles;
 
 /*
@@ -47,9 +51,14 @@ typedef struct gemm_tiles {
  * n_sub = min(2, acc_mem_columns / atom_n_max), reduced to 1 if two-sub-tile blocks
  * would be fewer than the compute units (occupancy);
  * tile_k = 128 bytes / elem_bytes; stages = min(8, (local_mem - staging - 1024)
- * / ((tile_m + tile_n) * tile_k * elem_bytes)), at least 2.  Pure host
- * arithmetic.  Returns ATTN_OK (then check out->feasible) or
- * ATTN_ERR_INVALID_ARG.
+ * / ((tile_m + tile_n) * tile_k * elem_bytes)), at least 2.
+ * CTA pairs: taken when the descriptor says pairs can run (max_clusters[1] > 0), tensor memory holds two
+ * accumulators (acc_mem_columns >= 2 atom_n_max), M > atom_m, N > atom_n_max / 2 and
+ * the pairs, P = min(max_clusters[1], num_units / 2, tiles), occupy at least as many CTAs as the lone-CTA tiling
+ * above would (the paper's occupancy step).  A pair owns a 2 atom_m x atom_n_max tile; every CTA stages its own
+ * atom_m rows of A and atom_n_max / 2 columns of B, so stages = min(8, (local_mem - 4 atom_m 128 - 1024) /
+ * ((atom_m + atom_n_max / 2) * tile_k * elem_bytes)); acc_buffers = acc_mem_columns / atom_n_max; ctas = 2 P.
+ * Pure host arithmetic.  Returns ATTN_OK (then check out->feasible) or ATTN_ERR_INVALID_ARG.
  */
 int gemm_plan(const attn_hw_desc *desc, int batch, int M, int N, int K, gemm_tiles *out);
 
@@ -64,6 +73,12 @@ int gemm_plan(const attn_hw_desc *desc, int batch, int M, int N, int K, gemm_til
  */
 int gemm_forward(const void *a, const void *b, void *c, int batch, int M, int N, int K, int b_layout,
                  void *cuda_stream);
+
+/* Same with tile fields overridden (tile sweep only; 0 keeps the closed-form value): cta_pair = 1 runs the
+ * lone-CTA tiling where the closed form takes pairs, cta_pair = 2 insists on pairs; tile_n (128 | 256) narrows a
+ * pair's tile.  ATTN_ERR_BAD_TILES if the combination was not compiled or does not fit. */
+int gemm_forward_tiles(const void *a, const void *b, void *c, int batch, int M, int N, int K, int b_layout,
+                       const gemm_tiles *override_tiles, void *cuda_stream);
 
 /*
  * p[r][:] = softmax(scale * s[r][:]) for `rows` rows of `cols` bf16 values

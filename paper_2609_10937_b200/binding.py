@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = (
     "attn_set_workspace", "attn_workspace_init", "attn_forward_ws", "attn_status_read", "attn_forward", "attn_forward_causal", "attn_forward_tiles", "attn_forward_simple", "attn_forward_host", "attn_forward_host_workspace_bytes", "attn_forward_static_scratch", "attn_forward_desc", "attn_plan_qk", "attn_forward_qk",
     "attn_last_device_status", "attn_selftest_wait_expiry", "attn_selftest_wait_expiry_to",
     "attn_last_launch_count", "attn_last_cluster_size", "attn_status_string", "attn_last_cuda_error",
-    "gemm_plan", "gemm_forward", "softmax_rows_forward", "attn_forward_unfused",
+    "gemm_plan", "gemm_forward", "gemm_forward_tiles", "softmax_rows_forward", "attn_forward_unfused",
 )
 
 
@@ -54,7 +54,8 @@ class AttnTiles(ctypes.Structure):
 class GemmTiles(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "tile_m", "tile_n", "tile_k", "n_sub", "stages", "smem_bytes", "tmem_columns", "tiles", "ctas", "feasible",
-    )] + [("wave_efficiency", ctypes.c_float), ("binding_constraint", ctypes.c_int32)]
+    )] + [("wave_efficiency", ctypes.c_float), ("binding_constraint", ctypes.c_int32), ("cta_pair", ctypes.c_int32),
+          ("acc_buffers", ctypes.c_int32)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -114,6 +115,7 @@ def lib() -> ctypes.CDLL:
         L.attn_last_cuda_error.restype = ctypes.c_char_p
         L.gemm_plan.argtypes = [ctypes.POINTER(AttnHwDesc), i32, i32, i32, i32, ctypes.POINTER(GemmTiles)]
         L.gemm_forward.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
+        L.gemm_forward_tiles.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, ctypes.POINTER(GemmTiles), vp]
         L.softmax_rows_forward.argtypes = [vp, vp, ctypes.c_longlong, i32, ctypes.c_float, vp]
         L.attn_forward_unfused.argtypes = [vp, vp, vp, vp, vp, ctypes.c_size_t, i32, i32, i32, i32, vp]
         for name in EXPORTED_SYMBOLS:
@@ -415,8 +417,10 @@ def _mat(x, name):
     return x if x.dim() == 3 else x.unsqueeze(0)
 
 
-def gemm(a, b, c=None, *, b_layout="kn"):
-    """C = A B ("kn": b is [.., K, N]) or C = A B^T ("nk": b is [.., N, K]); bf16 in and out, fp32 accumulation."""
+def gemm(a, b, c=None, *, b_layout="kn", cta_pair=0, tile_n=0):
+    """C = A B ("kn": b is [.., K, N]) or C = A B^T ("nk": b is [.., N, K]); bf16 in and out, fp32 accumulation.
+
+    cta_pair (1 | 2) and tile_n (128 | 256) override the closed-form tiles (tile sweep only; 0 keeps them)."""
     import torch
 
     a3, b3 = _mat(a, "a"), _mat(b, "b")
@@ -436,8 +440,14 @@ def gemm(a, b, c=None, *, b_layout="kn"):
     dev = a.device.index if a.device.index is not None else torch.cuda.current_device()
     with torch.cuda.device(dev):
         stream = torch.cuda.current_stream(a.device).cuda_stream
-        _check(lib().gemm_forward(a.data_ptr(), b.data_ptr(), c.data_ptr(), batch, M, N, K,
-                                  0 if b_layout == "kn" else 1, stream), "gemm_forward")
+        if cta_pair or tile_n:
+            ov = GemmTiles()
+            ov.cta_pair, ov.tile_n = int(cta_pair), int(tile_n)
+            _check(lib().gemm_forward_tiles(a.data_ptr(), b.data_ptr(), c.data_ptr(), batch, M, N, K,
+                                            0 if b_layout == "kn" else 1, ctypes.byref(ov), stream), "gemm_forward_tiles")
+        else:
+            _check(lib().gemm_forward(a.data_ptr(), b.data_ptr(), c.data_ptr(), batch, M, N, K,
+                                      0 if b_layout == "kn" else 1, stream), "gemm_forward")
     return c
 
 

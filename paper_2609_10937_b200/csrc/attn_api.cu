@@ -785,7 +785,8 @@ int make_tmap_mat(CUtensorMap* m, const void* base, int batch, int rows, int col
   return make_tmap(m, base, batch, rows, cols, box_rows);
 }
 
-int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, int K, int b_layout, cudaStream_t stream) {
+int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, int K, int b_layout, cudaStream_t stream,
+                const gemm_tiles* ovr = nullptr) {
   if (!a || !b || !c || batch <= 0 || M <= 0 || N <= 0 || K <= 0) return ATTN_ERR_INVALID_ARG;
   if (b_layout != 0 && b_layout != 1) return ATTN_ERR_INVALID_ARG;
   if ((K & 7) || (N & 7)) return ATTN_ERR_UNSUPPORTED_SHAPE;
@@ -796,18 +797,37 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
   int rc = device_state(&st);
   if (rc != ATTN_OK) return rc;
   gemm_tiles t;
-  if ((rc = gemm_plan(&st->desc, batch, M, N, K, &t)) != ATTN_OK) return rc;
-  // the kernel is compiled for exactly the tile shape the derivation gives on this architecture
+  if (ovr) {
+    // tile sweep: the derivation re-run with pairs switched off (cta_pair 1) or with the other tile width
+    attn_hw_desc d2 = st->desc;
+    if (ovr->cta_pair == 1) d2.max_clusters[1] = 0;
+    if ((rc = gemm_plan(&d2, batch, M, N, K, &t)) != ATTN_OK) return rc;
+    if (ovr->cta_pair == 2 && t.cta_pair != 2) return ATTN_ERR_BAD_TILES;
+    if (ovr->tile_n > 0 && ovr->tile_n != t.tile_n) {
+      if (t.cta_pair != 2 || (ovr->tile_n != 128 && ovr->tile_n != 256)) return ATTN_ERR_BAD_TILES;
+      t.tile_n = ovr->tile_n;
+      const int stage = gemm::pair_stage_bytes(t.tile_n);
+      t.stages = std::min(gemm::kMaxStages, (st->desc.local_mem_bytes - gemm::kPairOutBytes - gemm::kMiscBytes) / stage);
+      t.tiles = batch * ((M + 255) / 256) * ((N + t.tile_n - 1) / t.tile_n);
+      t.ctas = 2 * std::min(t.tiles, std::min(st->desc.max_clusters[1], st->desc.num_units / 2));
+      t.acc_buffers = 512 / t.tile_n;
+    }
+  } else if ((rc = gemm_plan(&st->desc, batch, M, N, K, &t)) != ATTN_OK) {
+    return rc;
+  }
+  // the kernels are compiled for exactly the tile shapes the derivation gives on this architecture
   if (!t.feasible || (t.n_sub != 1 && t.n_sub != 2) || t.tile_m != t.n_sub * attn::kSub || (t.tile_n != 128 && t.tile_n != 256) ||
-      t.tile_k != gemm::kTileK ||
-      t.stages > gemm::kMaxStages)
+      t.tile_k != gemm::kTileK || t.stages > gemm::kMaxStages || t.stages < 2)
     return ATTN_ERR_INFEASIBLE_PLAN;
   CUtensorMap ta, tb, tc;
+  const bool pair = t.cta_pair == 2;
+  // a CTA of a pair stages its own 128 rows of A and tile_n / 2 columns (rows, for [N][K]) of B
   if ((rc = make_tmap_mat(&ta, a, batch, M, K, attn::kSub)) != ATTN_OK) return rc;
   if (b_layout == 0) rc = make_tmap_mat(&tb, b, batch, K, N, gemm::kTileK);    // [K][N]: box 64 columns x 64 k-rows
-  else rc = make_tmap_mat(&tb, b, batch, N, K, t.tile_n);                      // [N][K]: box 64 k-columns x tile_n rows
+  else rc = make_tmap_mat(&tb, b, batch, N, K, pair ? t.tile_n / 2 : t.tile_n);   // [N][K]: box 64 k-columns x rows of B
   if (rc != ATTN_OK) return rc;
-  if ((rc = make_tmap_mat(&tc, c, batch, M, N, attn::kSub)) != ATTN_OK) return rc;
+  // (a pair's epilogue warps each store their own 32 rows)
+  if ((rc = make_tmap_mat(&tc, c, batch, M, N, pair ? 32 : attn::kSub)) != ATTN_OK) return rc;
   gemm::GemmParams p;
   p.M = M; p.N = N; p.K = K; p.batch = batch;
   p.n_sub = t.n_sub;
@@ -815,14 +835,37 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
   p.n_tiles = (N + t.tile_n - 1) / t.tile_n;
   p.k_steps = (K + gemm::kTileK - 1) / gemm::kTileK;
   p.stages = t.stages;
-  const int smem = gemm::smem_total(t.stages, t.tile_n);
-  auto launch = [&](auto kernel) -> int {
-    ATTN_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kernel<<<t.ctas, gemm::kThreads, smem, stream>>>(ta, tb, tc, p);
-    return ATTN_OK;
-  };
-  if (t.tile_n == 256) rc = (b_layout == 0) ? launch(gemm::gemm_kernel<true, 256>) : launch(gemm::gemm_kernel<false, 256>);
-  else rc = (b_layout == 0) ? launch(gemm::gemm_kernel<true, 128>) : launch(gemm::gemm_kernel<false, 128>);
+  if (pair) {
+    const int smem = gemm::pair_smem_total(t.stages, t.tile_n);
+    auto launch_pair = [&](auto kernel) -> int {
+      ATTN_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)t.ctas);
+      cfg.blockDim = dim3(gemm::kPairThreads);
+      cfg.dynamicSmemBytes = smem;
+      cfg.stream = stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      ATTN_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ta, tb, tc, p));
+      return ATTN_OK;
+    };
+    if (t.tile_n == 256) rc = (b_layout == 0) ? launch_pair(gemm::gemm_pair_kernel<true, 256>) : launch_pair(gemm::gemm_pair_kernel<false, 256>);
+    else rc = (b_layout == 0) ? launch_pair(gemm::gemm_pair_kernel<true, 128>) : launch_pair(gemm::gemm_pair_kernel<false, 128>);
+  } else {
+    const int smem = gemm::smem_total(t.stages, t.tile_n);
+    auto launch = [&](auto kernel) -> int {
+      ATTN_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+      kernel<<<t.ctas, gemm::kThreads, smem, stream>>>(ta, tb, tc, p);
+      return ATTN_OK;
+    };
+    if (t.tile_n == 256) rc = (b_layout == 0) ? launch(gemm::gemm_kernel<true, 256>) : launch(gemm::gemm_kernel<false, 256>);
+    else rc = (b_layout == 0) ? launch(gemm::gemm_kernel<true, 128>) : launch(gemm::gemm_kernel<false, 128>);
+  }
   if (rc != ATTN_OK) return rc;
   ATTN_CUDA_TRY(cudaGetLastError());
   ++t_launch_count;
@@ -864,6 +907,12 @@ extern "C" int gemm_forward(const void* a, const void* b, void* c, int batch, in
                             void* cuda_stream) {
   t_launch_count = 0;
   return gemm_launch(a, b, c, batch, M, N, K, b_layout, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int gemm_forward_tiles(const void* a, const void* b, void* c, int batch, int M, int N, int K, int b_layout,
+                                  const gemm_tiles* override_tiles, void* cuda_stream) {
+  t_launch_count = 0;
+  return gemm_launch(a, b, c, batch, M, N, K, b_layout, static_cast<cudaStream_t>(cuda_stream), override_tiles);
 }
 
 extern "C" int softmax_rows_forward(const void* s, void* p, long long rows, int cols, float scale, void* cuda_stream) {

@@ -364,6 +364,42 @@ extern "C" int gemm_plan(const attn_hw_desc* desc, int batch, int M, int N, int 
   int stages = (h.local_mem_bytes - staging - 1024) / stage;
   if (stages > 8) stages = 8;
   if (stages < 2) { out->binding_constraint = ATTN_BIND_SMEM; return ATTN_OK; }
+  // CTA pairs: two CTAs as one 2 atom_m-row matrix unit, each staging its own rows of A and half of B's columns, with
+  // as many accumulators as tensor memory holds so that a tile's epilogue runs under the next tile's products.
+  // Taken when the machine can run pairs, tensor memory holds two accumulators, the output is wider than half the
+  // atom's N, and the pairs occupy at least as many CTAs as the lone-CTA tiling would (the occupancy step).
+  {
+    const int pairs_max = h.max_clusters[1] < h.num_units / 2 ? h.max_clusters[1] : h.num_units / 2;
+    const int pn = h.atom_n_max;
+    const long long pt = (long long)batch * ceil_div(M, 2 * h.atom_m) * ceil_div(N, pn);
+    const long long lone = (long long)batch * ceil_div(M, tile_m) * ceil_div(N, tile_n);
+    const long long lone_ctas = lone < h.num_units ? lone : h.num_units;
+    const long long pairs = pt < pairs_max ? pt : pairs_max;
+    if (pairs_max > 0 && M > h.atom_m && N > pn / 2 && h.acc_mem_columns >= 2 * pn && 2 * pairs >= lone_ctas &&
+        pt <= 0x3FFFFFFFLL) {
+      const int pstage = (h.atom_m + pn / 2) * tile_k * h.elem_bytes;
+      const int pstaging = 4 * h.atom_m * 128;    // per epilogue warp (4 lane quarters x 2 column halves) two 32-row chunks
+      int pstages = (h.local_mem_bytes - pstaging - 1024) / pstage;
+      if (pstages > 8) pstages = 8;
+      if (pstages >= 2) {
+        out->tile_m = 2 * h.atom_m;
+        out->tile_n = pn;
+        out->tile_k = tile_k;
+        out->n_sub = 2;
+        out->stages = pstages;
+        out->smem_bytes = pstages * pstage + pstaging + 1024;
+        out->tmem_columns = pow2_ceil((h.acc_mem_columns / pn) * pn);
+        out->tiles = (int)pt;
+        out->ctas = (int)(2 * pairs);
+        const long long pwaves = (pt + pairs - 1) / pairs;
+        out->wave_efficiency = (float)((double)pt / ((double)pwaves * pairs));
+        out->cta_pair = 2;
+        out->acc_buffers = h.acc_mem_columns / pn;
+        out->feasible = 1;
+        return ATTN_OK;
+      }
+    }
+  }
   const long long tiles = (long long)batch * ceil_div(M, tile_m) * ceil_div(N, tile_n);
   if (tiles > 0x3FFFFFFFLL) return ATTN_OK;
   out->tile_m = tile_m;
@@ -377,6 +413,8 @@ extern "C" int gemm_plan(const attn_hw_desc* desc, int batch, int M, int N, int 
   out->ctas = tiles < h.num_units ? (int)tiles : h.num_units;
   const long long waves = (tiles + out->ctas - 1) / out->ctas;
   out->wave_efficiency = (float)((double)tiles / ((double)waves * out->ctas));
+  out->cta_pair = 1;
+  out->acc_buffers = 1;
   out->feasible = 1;
   return ATTN_OK;
 }

@@ -227,6 +227,232 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
 }
 
 // ---------------------------------------------------------------------------
+// gemm_pair_kernel: the same product with two CTAs per matrix instruction (cta_group::2).
+//
+// A cluster of two CTAs owns a 256 x kPairN output tile.  CTA r of the pair holds rows [128 r, 128 r + 128) of the A
+// tile and columns [r kPairN / 2, (r + 1) kPairN / 2) of the B tile in its shared memory -- every byte of B is
+// fetched and stored once per pair, so a CTA's ring stage is half as large as for a lone CTA working on 256 rows --
+// and the 128 x kPairN fp32 accumulator of its rows in its tensor memory.  One thread of the even CTA issues
+// tcgen05.mma.cta_group::2 for both; its completion releases the ring stage in both CTAs (a commit multicast to
+// the two CTAs' barriers).  An accumulator takes kPairN of the 512 tensor-memory columns, so there are 512 / kPairN
+// of them and the epilogue of tile i (tensor memory -> bf16 -> staging -> TMA store, per CTA for its own rows) runs
+// under the products of tile i + 1.  Barriers: full[s] of the even CTA counts the bytes of both CTAs' loads (the
+// odd CTA's copies name that barrier; no load is multicast); empty[s] and acc_full[b] exist in both CTAs;
+// acc_empty[b] of the even CTA counts one arrival per epilogue warp of both CTAs.
+// ---------------------------------------------------------------------------
+constexpr int kPairEpiWarps = 8;           // four lane quarters x two column halves of the accumulator
+constexpr int kPairThreads = 64 + 32 * kPairEpiWarps;   // producer warp, MMA warp, epilogue warps
+constexpr int kPairStageA = kSub * kTileK * 2;
+__host__ __device__ constexpr int pair_stage_bytes(int pair_n) { return kPairStageA + (pair_n / 2) * kTileK * 2; }
+constexpr int kPairOutBytes = kPairEpiWarps * 2 * 4096;  // per epilogue warp two [32 rows][64 columns] bf16 staging chunks
+__host__ __device__ constexpr int pair_smem_total(int stages, int pair_n) {
+  return stages * pair_stage_bytes(pair_n) + kPairOutBytes + kMiscBytes;
+}
+
+struct GemmPairMisc {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t acc_full[4];
+  uint64_t acc_empty[4];
+  attn::AbortCell abort;
+  uint32_t tmem_slot;
+};
+static_assert(sizeof(GemmPairMisc) <= kMiscBytes, "misc region too large");
+
+template <bool B_KN, int kPairN>
+__global__ void __launch_bounds__(kPairThreads, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                 const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
+  static_assert(kPairN == 128 || kPairN == 256, "pair tile N");
+  constexpr int kStageBytes = pair_stage_bytes(kPairN);
+  constexpr int kHalfN = kPairN / 2;                 // B columns held by one CTA
+  constexpr int kBufs = 512 / kPairN;                // accumulators in tensor memory
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = smem_u32(smem_raw);
+  const uint32_t out_smem = smem_base + p.stages * kStageBytes;
+  GemmPairMisc* misc = reinterpret_cast<GemmPairMisc*>(smem_raw + p.stages * kStageBytes + kPairOutBytes);
+  volatile int* abort_flag = &misc->abort.flag;
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();           // 0: issues the matrix instructions of the pair
+  const long long pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    attn::abort_cell_init(&misc->abort, nullptr);
+    if (smem_base & 1023u) {
+      attn::report_timeout(attn::wait_info(kRoleGemmLoad, 0, 0xFFFF), abort_flag);
+      misc->abort.flag = 1;
+    }
+    for (int s = 0; s < kMaxStages; ++s) {
+      mbar_init(smem_u32(&misc->full[s]), 1);
+      mbar_init(smem_u32(&misc->empty[s]), 1);
+    }
+    for (int b = 0; b < 4; ++b) {
+      mbar_init(smem_u32(&misc->acc_full[b]), 1);
+      mbar_init(smem_u32(&misc->acc_empty[b]), 2 * kPairEpiWarps);   // the epilogue warps of both CTAs of the pair
+    }
+    fence_mbar_init();
+    prefetch_tmap(&tm_a);
+    prefetch_tmap(&tm_b);
+    prefetch_tmap(&tm_c);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(&misc->tmem_slot), 512);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  // the peer's barriers must exist before this CTA's copies or commits touch them
+  cluster_arrive();
+  cluster_wait();
+  tc_fence_after();
+  const uint32_t tmem_base = misc->tmem_slot;
+  const long long tiles = (long long)p.batch * p.m_tiles * p.n_tiles;
+  const bool run = (*abort_flag == 0);
+
+  if (warp == 0) {
+    // ========================================================== TMA producer (both CTAs, each for what it holds)
+    if (run && elect_one()) {
+      int stage = 0, issued = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (long long t = pair; ok && t < tiles; t += n_pairs) {
+        const int nt = (int)(t % p.n_tiles), mt = (int)((t / p.n_tiles) % p.m_tiles), b = (int)(t / ((long long)p.n_tiles * p.m_tiles));
+        const int row0 = mt * kTileM + (int)rank * kSub, col0 = nt * kPairN + (int)rank * kHalfN;
+        for (int ks = 0; ks < p.k_steps; ++ks) {
+          if (!attn::wait_bar(smem_u32(&misc->empty[stage]), phase ^ 1u, abort_flag, attn::wait_info(kRoleGemmLoad, 1, ks))) { ok = false; break; }
+          // the even CTA's barrier counts the bytes of both CTAs' copies of this stage
+          const uint32_t bar = map_to_cta(smem_u32(&misc->full[stage]), 0);
+          const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kPairStageA;
+          if (rank == 0) mbar_arrive_expect_tx(smem_u32(&misc->full[stage]), 2 * kStageBytes);
+          tma_load_3d_pair(a_dst, &tm_a, ks * kTileK, row0, b, bar);
+          if (B_KN) {
+#pragma unroll
+            for (int c = 0; c < kHalfN / 64; ++c)
+              tma_load_3d_pair(b_dst + c * (kTileK * 128), &tm_b, col0 + c * 64, ks * kTileK, b, bar);
+          } else {
+            tma_load_3d_pair(b_dst, &tm_b, ks * kTileK, col0, b, bar);
+          }
+          ++issued;
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // Drain: a copy this thread started must land before the CTA may exit.  The bytes are counted on the even
+        // CTA's barrier; the odd CTA cannot poll it, so it waits out the time a copy can take instead.
+        if (rank == 0) {
+          const int first = issued > p.stages ? issued - p.stages : 0;
+          for (int t = first; t < issued; ++t) {
+            const long long t0 = clock64();
+            while (!mbar_try_wait(smem_u32(&misc->full[t % p.stages]), (uint32_t)(t / p.stages) & 1u) &&
+                   clock64() - t0 < attn::kWaitLimitCycles) {}
+          }
+        } else {
+          const long long t0 = clock64();
+          while (clock64() - t0 < 2000000LL) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ============================================================ MMA issuer (even CTA only)
+    bool ok = run && rank == 0;
+    int stage = 0;
+    uint32_t phase = 0, tile_ctr = 0;
+    constexpr uint32_t idesc = make_idesc_bf16(2 * kSub, kPairN, B_KN);
+    constexpr uint32_t hi_k = attn::desc_hi_sw128(1024);
+    for (long long t = pair; ok && t < tiles; t += n_pairs, ++tile_ctr) {
+      const uint32_t buf = tile_ctr % kBufs, use = tile_ctr / kBufs;
+      if (use > 0) {
+        ok = attn::wait_bar_warp(smem_u32(&misc->acc_empty[buf]), (use - 1) & 1, abort_flag, attn::wait_info(kRoleGemmMma, 2, tile_ctr));
+        if (!ok) break;
+        tc_fence_after();
+      }
+      for (int ks = 0; ok && ks < p.k_steps; ++ks) {
+        if (!attn::wait_bar_warp(smem_u32(&misc->full[stage]), phase, abort_flag, attn::wait_info(kRoleGemmMma, 1, ks))) { ok = false; break; }
+        tc_fence_after();
+        if (elect_one()) {
+          const uint32_t a_smem = smem_base + stage * kStageBytes, b_smem = a_smem + kPairStageA;
+          const uint32_t a_lo = attn::desc_lo(a_smem, 16);
+          const uint32_t b_lo = B_KN ? attn::desc_lo(b_smem, kTileK * 128) : attn::desc_lo(b_smem, 16);
+#pragma unroll
+          for (int k16 = 0; k16 < kTileK / 16; ++k16) {
+            const uint64_t a = attn::desc_from_words(a_lo + ((k16 * 32) >> 4), hi_k);
+            const uint64_t b = attn::desc_from_words(b_lo + ((B_KN ? k16 * 2048 : k16 * 32) >> 4), hi_k);
+            umma_ss_pair(tmem_base + buf * kPairN, a, b, idesc, (ks > 0 || k16 > 0) ? 1u : 0u);
+          }
+          umma_commit_pair(smem_u32(&misc->empty[stage]), 3);
+          if (ks == p.k_steps - 1) umma_commit_pair(smem_u32(&misc->acc_full[buf]), 3);
+        }
+        __syncwarp();
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else {
+    // ============================================================== epilogue (both CTAs, each its own 128 rows)
+    // Eight warps, none of which meets another: warp w reads lanes 32 (w mod 4) .. + 31 (its rows) of one column
+    // half of the accumulator, 64 columns at a time, and sends them off through two staging chunks of its own
+    // (tensor memory -> bf16 -> swizzled [32 rows][64 columns] chunk -> TMA store of a 32-row box), the store of
+    // one chunk running under the conversion of the next.
+    const int ew = warp - 2;
+    const int half = ew >> 2;                                 // column half of the accumulator
+    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t stage_w = out_smem + ew * 8192;
+    constexpr int kChunks = kPairN / 128;                     // 64-column chunks per warp and tile
+    uint32_t tile_ctr = 0, chunk_ctr = 0;
+    bool ok = run;
+    for (long long t = pair; ok && t < tiles; t += n_pairs, ++tile_ctr) {
+      const int nt = (int)(t % p.n_tiles), mt = (int)((t / p.n_tiles) % p.m_tiles), b = (int)(t / ((long long)p.n_tiles * p.m_tiles));
+      const uint32_t buf = tile_ctr % kBufs, use = tile_ctr / kBufs;
+      ok = attn::wait_bar_warp(smem_u32(&misc->acc_full[buf]), use & 1, abort_flag, attn::wait_info(kRoleGemmEpi, 2, tile_ctr));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t acc = lane_base + buf * kPairN + half * (kPairN / 2);
+      const int row0 = mt * kTileM + (int)rank * kSub + (warp & 3) * 32;
+#pragma unroll 1
+      for (int c = 0; c < kChunks; ++c, ++chunk_ctr) {
+        uint32_t r0[32], r1[32];
+        tmem_ld32_nowait(acc + c * 64, r0);
+        tmem_ld32_nowait(acc + c * 64 + 32, r1);
+        tmem_ld_fence(r0);
+        tmem_ld_fence(r1);
+        if (c == kChunks - 1) {
+          // this warp has read its part of the accumulator: one arrival per warp on the even CTA's barrier
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_peer(map_to_cta(smem_u32(&misc->acc_empty[buf]), 0));
+        }
+        const uint32_t dst = stage_w + (chunk_ctr & 1) * 4096;
+        // the store that last read this chunk (two chunks ago) must have finished reading it
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        __syncwarp();
+        float v0[32], v1[32];
+#pragma unroll
+        for (int k = 0; k < 32; ++k) { v0[k] = __uint_as_float(r0[k]); v1[k] = __uint_as_float(r1[k]); }
+        attn::stage_row_chunk(dst, 0, lane, v0);
+        attn::stage_row_chunk(dst, 1, lane, v1);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_3d(&tm_c, dst, nt * kPairN + half * (kPairN / 2) + c * 64, row0, b);
+          tma_store_commit();
+        }
+      }
+    }
+    if (lane == 0) tma_store_wait_read();                    // shared memory is read by the stores until here
+    __syncwarp();
+  }
+  tc_fence_before();
+  __syncthreads();
+  // no CTA leaves while its peer may still read its shared memory, signal its barriers or use its tensor memory
+  cluster_arrive();
+  cluster_wait();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------
 // Row softmax of scale * S, bf16 in and out (in place allowed).  One CTA of THREADS threads per row; thread t
 // holds VPT vectors of 8 consecutive columns (vector v covers columns (v * THREADS + t) * 8 ...).  Each thread keeps
 // the running statistics (m, d) of its columns; partials are merged with

@@ -28,12 +28,12 @@ def _rand_bits(rng, shape, sigma=1.0):
     return synth.f32_to_bf16_bits((rng.standard_normal(shape) * sigma).astype(np.float32))
 
 
-def _check_product(env, batch, M, N, K, layout, seed, rows_per_batch=None):
+def _check_product(env, batch, M, N, K, layout, seed, rows_per_batch=None, **tiles):
     torch, go, binding = env
     rng = np.random.default_rng([seed, M, N, K])
     a = _rand_bits(rng, (batch, M, K))
     b = _rand_bits(rng, (batch, K, N) if layout == "kn" else (batch, N, K))
-    c = binding.gemm(to_cuda_bf16(a), to_cuda_bf16(b), b_layout=layout)
+    c = binding.gemm(to_cuda_bf16(a), to_cuda_bf16(b), b_layout=layout, **tiles)
     torch.cuda.synchronize()
     assert binding.last_device_status()[0] == 0
     got = to_host_f64(c).reshape(batch, M, N)
@@ -53,6 +53,29 @@ def _check_product(env, batch, M, N, K, layout, seed, rows_per_batch=None):
     (1, 1000, 1000, 1000), (1, 2048, 128, 2048)])
 def test_matrix_product_matches_oracle(env, layout, batch, M, N, K):
     _check_product(env, batch, M, N, K, layout, seed=1)
+
+
+@pytest.mark.parametrize("layout", ["kn", "nk"])
+@pytest.mark.parametrize("batch,M,N,K", [
+    (1, 512, 512, 64), (1, 520, 264, 72), (2, 300, 1000, 200), (1, 129, 136, 8), (1, 4096, 768, 320), (5, 257, 257 + 7, 1024),
+    (1, 2560, 2304, 64)])
+def test_cta_pairs_and_lone_ctas_agree_with_the_oracle_and_each_other(env, layout, batch, M, N, K):
+    """The two tilings of the same product: CTA pairs (one matrix instruction over two CTAs, two accumulators in tensor
+    memory, per-warp stores) and lone CTAs.  Ragged M, N and K, several tiles per pair (more than the accumulators,
+    so that buffers are reused), batches.  Both sum the K products of an element in the same order: same bits."""
+    torch, go, binding = env
+    desc = binding.hw_desc_query(0)
+    assert binding.gemm_plan(desc, batch, M, N, K).cta_pair == 2
+    _check_product(env, batch, M, N, K, layout, seed=4, rows_per_batch=300)                 # closed-form default: pairs
+    _check_product(env, batch, M, N, K, layout, seed=4, rows_per_batch=300, cta_pair=1)
+    _check_product(env, batch, M, N, K, layout, seed=4, rows_per_batch=300, cta_pair=2, tile_n=128)
+    rng = np.random.default_rng([9, M, N, K])
+    a = to_cuda_bf16(_rand_bits(rng, (batch, M, K)))
+    b = to_cuda_bf16(_rand_bits(rng, (batch, K, N) if layout == "kn" else (batch, N, K)))
+    pair, lone = binding.gemm(a, b, b_layout=layout), binding.gemm(a, b, b_layout=layout, cta_pair=1)
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0
+    assert torch.equal(pair.view(torch.int16), lone.view(torch.int16))
 
 
 @pytest.mark.parametrize("layout", ["kn", "nk"])

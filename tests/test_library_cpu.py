@@ -45,19 +45,32 @@ def test_gemm_plan_closed_form(binding):
     with the B200 constants, and its reaction to a changed descriptor."""
     desc = binding.hw_desc_b200()
     t = binding.gemm_plan(desc, 1, 4096, 4096, 4096)
-    # 512 accumulator columns / 256 = 2 sub-tiles; stage = (256 + 256) * 64 * 2 = 65536; staging 2 * 128 * 128
-    assert (t.tile_m, t.tile_n, t.tile_k, t.n_sub) == (256, 256, 64, 2)
+    # CTA pairs: a pair owns 256 x 256; per CTA a stage is (128 + 128) * 64 * 2 = 32768 bytes, staging 8 warps x 2 x 4096
+    assert (t.tile_m, t.tile_n, t.tile_k, t.n_sub, t.cta_pair, t.acc_buffers) == (256, 256, 64, 2, 2, 2)
+    assert t.stages == (232448 - 65536 - 1024) // 32768 == 5 and t.smem_bytes == 5 * 32768 + 65536 + 1024
+    assert (t.tiles, t.ctas, t.feasible, t.tmem_columns) == (256, 148, 1, 512)
+    assert t.wave_efficiency == pytest.approx(256 / (4 * 74))
+    # pairs occupy as many CTAs as lone 128-row tiles would (3 * 4 * 3 = 36 pairs against 3 * 8 * 3 = 72 CTAs)
+    t = binding.gemm_plan(desc, 3, 1000, 520, 64)
+    assert (t.cta_pair, t.tile_m, t.tiles, t.ctas) == (2, 256, 36, 72)
+    # an output no wider than half the atom's N stays with lone CTAs (P V of the unfused path: 64 blocks -> 128)
+    t = binding.gemm_plan(desc, 1, 16384, 128, 16384)
+    assert (t.cta_pair, t.n_sub, t.tile_n, t.tiles, t.ctas) == (1, 1, 128, 128, 128)
+    # a machine that cannot run pairs: the lone-CTA derivation (two sub-tiles share every B tile)
+    desc.max_clusters[1] = 0
+    t = binding.gemm_plan(desc, 1, 4096, 4096, 4096)
+    assert (t.tile_m, t.tile_n, t.tile_k, t.n_sub, t.cta_pair, t.acc_buffers) == (256, 256, 64, 2, 1, 1)
+    # stage = (256 + 256) * 64 * 2 = 65536; staging 2 * 128 * 128
     assert t.stages == (232448 - 32768 - 1024) // 65536 == 3 and t.smem_bytes == 3 * 65536 + 32768 + 1024
     assert (t.tiles, t.ctas, t.feasible, t.tmem_columns) == (256, 148, 1, 512)
     assert t.wave_efficiency == pytest.approx(256 / (2 * 148))
     # fewer two-sub-tile blocks than SMs (3 * 4 * 3 = 36 < 148): one sub-tile per block, twice as many blocks
     t = binding.gemm_plan(desc, 3, 1000, 520, 64)
     assert (t.n_sub, t.tile_m, t.tiles, t.ctas) == (1, 128, 3 * 8 * 3, 72)
-    t = binding.gemm_plan(desc, 1, 16384, 128, 16384)        # P V of the unfused path: 64 blocks -> 128
-    assert (t.n_sub, t.tile_n, t.tiles, t.ctas) == (1, 128, 128, 128)
-    desc.acc_mem_columns = 256                      # half the tensor memory: one sub-tile
+    desc = binding.hw_desc_b200()
+    desc.acc_mem_columns = 256                      # half the tensor memory: no second accumulator, one sub-tile
     t = binding.gemm_plan(desc, 1, 4096, 4096, 4096)
-    assert (t.n_sub, t.tile_m, t.stages) == (1, 128, (232448 - 16384 - 1024) // 49152)
+    assert (t.cta_pair, t.n_sub, t.tile_m, t.stages) == (1, 1, 128, (232448 - 16384 - 1024) // 49152)
     desc.local_mem_bytes = 101376                   # a small shared memory: the ring no longer fits twice
     t = binding.gemm_plan(desc, 1, 4096, 4096, 4096)
     assert t.feasible == 0 or t.stages >= 2

@@ -247,3 +247,29 @@ def test_cost_constants_steer_the_choice():
     for B, H, L, d in _SHAPES:
         t = po.derive_tiles_tmem_machine(free, B, H, L, d)
         assert t["cost_steps"] == min(r["path"] for r in t["candidates"] if r["eligible"])
+
+
+def test_closed_form_grid_is_the_measured_fastest():
+    """The B200 cost constants against measurements: for every shape of the grid sweep kept under profiles/ (times of
+    all candidate grids on a B200), the grid the C planner derives from the built-in descriptor must be within 5 % of
+    the fastest measured one.  A wrong constant or tie-break moves some pick to a measurably slower grid."""
+    import os
+
+    from paper_2609_10937_b200 import binding, build
+    from tests.conftest import ROOT
+
+    build.build()
+    desc = binding.hw_desc_b200()
+    shapes = {}
+    with open(os.path.join(ROOT, "profiles", "grid_sweep_b200.txt")) as fh:
+        for line in fh:
+            if line.startswith("#") or not line.strip():
+                continue
+            B, H, L, d, q_tiles, steps, ctas, k, cluster, us, picked = line.split()
+            shapes.setdefault((int(B), int(H), int(L), int(d)), {})[int(ctas)] = float(us)
+    assert len(shapes) >= 18
+    for (B, H, L, d), times in shapes.items():
+        assert len(times) >= 2
+        pick = binding.plan(desc, B, H, L, d).ctas
+        assert pick in times, f"{(B, H, L, d)}: the closed form picks {pick} CTAs, which the sweep did not measure"
+        assert times[pick] <= 1.05 * min(times.values()), (B, H, L, d, pick, times)
