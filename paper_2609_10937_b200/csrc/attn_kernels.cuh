@@ -590,12 +590,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           // complete on the wrong 128 / 256 arrivals.  Here every arrival of step g comes after P V(g-1) has
           // finished, hence after every thread's arrivals of step g-1.  (The segment's first step is covered by
           // the wait for the last P V at the end of the previous segment.)
+          misc->alpha[i][g & 1][row] = alpha;
           if (g != g_seg0) {
             if (!wait_bar_warp(smem_u32(&misc->o_full[i]), (g - 1) & 1, abort_flag, wait_info(kRoleSoftmax, kBarOFull, 0x4000 | g))) return false;
             tc_fence_after();
           }
+        } else {
+          misc->alpha[i][g & 1][row] = alpha;
         }
-        misc->alpha[i][g & 1][row] = alpha;
         mbar_arrive(bar_a);
         const uint64_t neg_m2 = pack_f32x2(-m_new, -m_new);
         uint64_t sum_a = 0ull, sum_b = 0ull;               // packed (0.f, 0.f)
