@@ -835,7 +835,13 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
   p.n_tiles = (N + t.tile_n - 1) / t.tile_n;
   p.k_steps = (K + gemm::kTileK - 1) / gemm::kTileK;
   p.stages = t.stages;
+  p.group_m = 1;
   if (pair) {
+    // bands of about sqrt(pairs) tile rows: the tiles in flight then share the fewest operand panels
+    const int pairs = t.ctas / 2;
+    int gm = 1;
+    while ((gm + 1) * (gm + 1) <= pairs) ++gm;
+    p.group_m = gm;
     const int smem = gemm::pair_smem_total(t.stages, t.tile_n);
     auto launch_pair = [&](auto kernel) -> int {
       ATTN_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));

@@ -39,7 +39,24 @@ struct GemmParams {
   int m_tiles, n_tiles;   // ceil(M / (128 n_sub)), ceil(N / tile_n)
   int k_steps;            // ceil(K / 64)
   int stages;
+  int group_m;            // pair kernel: tiles are walked in bands of this many tile rows (see tile_coords)
 };
+
+// Order in which the persistent grid walks the output tiles.  Tiles that run at the same time should share operand
+// panels in the cache: with P tiles in flight, a band of `group_m` tile rows walked column by column keeps
+// group_m row panels of A and about P / group_m column panels of B live -- (group_m + P / group_m) panels, least for
+// group_m ~ sqrt(P) -- where walking whole tile rows would stream all of B for every wave.
+__device__ __forceinline__ void tile_coords(long long t, int m_tiles, int n_tiles, int group_m, int& mt, int& nt, int& b) {
+  const long long per_batch = (long long)m_tiles * n_tiles;
+  b = (int)(t / per_batch);
+  const int r = (int)(t - (long long)b * per_batch);
+  const int band = r / (group_m * n_tiles);
+  const int first = band * group_m;
+  const int rows = (m_tiles - first) < group_m ? (m_tiles - first) : group_m;
+  const int in = r - band * group_m * n_tiles;
+  mt = first + in % rows;
+  nt = in / rows;
+}
 
 struct GemmMisc {
   uint64_t full[kMaxStages];
@@ -317,7 +334,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       uint32_t phase = 0;
       bool ok = true;
       for (long long t = pair; ok && t < tiles; t += n_pairs) {
-        const int nt = (int)(t % p.n_tiles), mt = (int)((t / p.n_tiles) % p.m_tiles), b = (int)(t / ((long long)p.n_tiles * p.m_tiles));
+        int nt, mt, b;
+      tile_coords(t, p.m_tiles, p.n_tiles, p.group_m, mt, nt, b);
         const int row0 = mt * kTileM + (int)rank * kSub, col0 = nt * kPairN + (int)rank * kHalfN;
         for (int ks = 0; ks < p.k_steps; ++ks) {
           if (!attn::wait_bar(smem_u32(&misc->empty[stage]), phase ^ 1u, abort_flag, attn::wait_info(kRoleGemmLoad, 1, ks))) { ok = false; break; }
@@ -401,7 +419,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     uint32_t tile_ctr = 0, chunk_ctr = 0;
     bool ok = run;
     for (long long t = pair; ok && t < tiles; t += n_pairs, ++tile_ctr) {
-      const int nt = (int)(t % p.n_tiles), mt = (int)((t / p.n_tiles) % p.m_tiles), b = (int)(t / ((long long)p.n_tiles * p.m_tiles));
+      int nt, mt, b;
+      tile_coords(t, p.m_tiles, p.n_tiles, p.group_m, mt, nt, b);
       const uint32_t buf = tile_ctr % kBufs, use = tile_ctr / kBufs;
       ok = attn::wait_bar_warp(smem_u32(&misc->acc_full[buf]), use & 1, abort_flag, attn::wait_info(kRoleGemmEpi, 2, tile_ctr));
       if (!ok) break;
