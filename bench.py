@@ -306,11 +306,14 @@ def measure_config(gpu, name, peaks, iters=None, oracle=True):
     plan = binding.plan(gpu.desc, case.B, case.H, case.L, case.d)
     if iters is None:
         iters = 100 if case.flops < 1e9 else 30 if case.flops < 5e11 else 10
-    ms, per, _, _ = gpu.timed(lambda: binding.forward(dq, dk, dv, do), iters, 5)
+    ms_mean, per, _, _ = gpu.timed(lambda: binding.forward(dq, dk, dv, do), iters, 5)
     cluster = binding.last_cluster_size()
     gpu.check_status()
+    # the median of the per-launch times: one launch delayed on the host side (the events bracket the launch call)
+    # would otherwise carry into a mean over few launches
+    ms = statistics.median(per)
     tf = case.flops / (ms * 1e-3) / 1e12
-    out = {"shape": [case.B, case.H, case.L, case.d], "ms": ms, "ms_min": min(per), "tflops": tf,
+    out = {"shape": [case.B, case.H, case.L, case.d], "ms": ms, "ms_mean": ms_mean, "ms_min": min(per), "tflops": tf,
            "frac_of_measured_burst_peak": tf / peaks["bf16_tflops"], "launches_timed": iters,
            "tiles": {"tile_q": plan.tile_q, "tile_kv": plan.tile_kv, "kv_stages": plan.kv_stages, "q_tiles": plan.tiles,
                      "ctas": plan.ctas, "cluster": cluster, "cost_steps": plan.cost_steps},
