@@ -43,6 +43,8 @@ typedef struct gemm_tiles {
                            tile_m x tile_n tile, each holding half of its rows and half of B's columns)  */
   int32_t acc_buffers;  /* accumulators that fit tensor memory: with more than one the epilogue of a tile
                            runs under the products of the next                                        */
+  int32_t tail_split;   /* CTA pairs: the last this-many tiles -- those that would form a partly empty last wave,
+                           if they are no more than half the pairs -- run as two half-width work items each      */
 } gemm_tiles;
 
 /*
@@ -58,6 +60,9 @@ typedef struct gemm_tiles {
  * above would (the paper's occupancy step).  A pair owns a 2 atom_m x atom_n_max tile; every CTA stages its own
  * atom_m rows of A and atom_n_max / 2 columns of B, so stages = min(8, (local_mem - 4 atom_m 128 - 1024) /
  * ((atom_m + atom_n_max / 2) * tile_k * elem_bytes)); acc_buffers = acc_mem_columns / atom_n_max; ctas = 2 P.
+ * Last wave: r = tiles mod P tiles remain after the whole waves; if 0 < 2 r <= P they are executed as 2 r work items
+ * of half the width (tail_split = r), which keeps twice as many pairs busy for the shorter last wave; wave_efficiency
+ * then counts a half-width item as 0.64 of a tile (measured on B200: the narrow instruction runs at 0.78 of the rate).
  * Pure host arithmetic.  Returns ATTN_OK (then check out->feasible) or ATTN_ERR_INVALID_ARG.
  */
 int gemm_plan(const attn_hw_desc *desc, int batch, int M, int N, int K, gemm_tiles *out);
@@ -76,7 +81,7 @@ int gemm_forward(const void *a, const void *b, void *c, int batch, int M, int N,
 
 /* Same with tile fields overridden (tile sweep only; 0 keeps the closed-form value): cta_pair = 1 runs the
  * lone-CTA tiling where the closed form takes pairs, cta_pair = 2 insists on pairs; tile_n (128 | 256) narrows a
- * pair's tile.  ATTN_ERR_BAD_TILES if the combination was not compiled or does not fit. */
+ * pair's tile; tail_split < 0 keeps whole tiles in the last wave.  ATTN_ERR_BAD_TILES if the combination was not compiled or does not fit. */
 int gemm_forward_tiles(const void *a, const void *b, void *c, int batch, int M, int N, int K, int b_layout,
                        const gemm_tiles *override_tiles, void *cuda_stream);
 

@@ -55,7 +55,7 @@ class GemmTiles(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "tile_m", "tile_n", "tile_k", "n_sub", "stages", "smem_bytes", "tmem_columns", "tiles", "ctas", "feasible",
     )] + [("wave_efficiency", ctypes.c_float), ("binding_constraint", ctypes.c_int32), ("cta_pair", ctypes.c_int32),
-          ("acc_buffers", ctypes.c_int32)]
+          ("acc_buffers", ctypes.c_int32), ("tail_split", ctypes.c_int32)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -417,10 +417,11 @@ def _mat(x, name):
     return x if x.dim() == 3 else x.unsqueeze(0)
 
 
-def gemm(a, b, c=None, *, b_layout="kn", cta_pair=0, tile_n=0):
+def gemm(a, b, c=None, *, b_layout="kn", cta_pair=0, tile_n=0, tail_split=0):
     """C = A B ("kn": b is [.., K, N]) or C = A B^T ("nk": b is [.., N, K]); bf16 in and out, fp32 accumulation.
 
-    cta_pair (1 | 2) and tile_n (128 | 256) override the closed-form tiles (tile sweep only; 0 keeps them)."""
+    cta_pair (1 | 2), tile_n (128 | 256) and tail_split (-1: whole tiles in the last wave) override the closed-form
+    tiles (tile sweep only; 0 keeps them)."""
     import torch
 
     a3, b3 = _mat(a, "a"), _mat(b, "b")
@@ -440,9 +441,9 @@ def gemm(a, b, c=None, *, b_layout="kn", cta_pair=0, tile_n=0):
     dev = a.device.index if a.device.index is not None else torch.cuda.current_device()
     with torch.cuda.device(dev):
         stream = torch.cuda.current_stream(a.device).cuda_stream
-        if cta_pair or tile_n:
+        if cta_pair or tile_n or tail_split:
             ov = GemmTiles()
-            ov.cta_pair, ov.tile_n = int(cta_pair), int(tile_n)
+            ov.cta_pair, ov.tile_n, ov.tail_split = int(cta_pair), int(tile_n), int(tail_split)
             _check(lib().gemm_forward_tiles(a.data_ptr(), b.data_ptr(), c.data_ptr(), batch, M, N, K,
                                             0 if b_layout == "kn" else 1, ctypes.byref(ov), stream), "gemm_forward_tiles")
         else:

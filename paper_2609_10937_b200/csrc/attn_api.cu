@@ -811,7 +811,9 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
       t.tiles = batch * ((M + 255) / 256) * ((N + t.tile_n - 1) / t.tile_n);
       t.ctas = 2 * std::min(t.tiles, std::min(st->desc.max_clusters[1], st->desc.num_units / 2));
       t.acc_buffers = 512 / t.tile_n;
+      t.tail_split = 0;
     }
+    if (ovr->tail_split < 0) t.tail_split = 0;                 // (sweep: whole tiles in the last wave too)
   } else if ((rc = gemm_plan(&st->desc, batch, M, N, K, &t)) != ATTN_OK) {
     return rc;
   }
@@ -836,12 +838,14 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
   p.k_steps = (K + gemm::kTileK - 1) / gemm::kTileK;
   p.stages = t.stages;
   p.group_m = 1;
+  p.tail_tiles = 0;
   if (pair) {
     // bands of about sqrt(pairs) tile rows: the tiles in flight then share the fewest operand panels
     const int pairs = t.ctas / 2;
     int gm = 1;
     while ((gm + 1) * (gm + 1) <= pairs) ++gm;
     p.group_m = gm;
+    p.tail_tiles = t.tail_split;
     const int smem = gemm::pair_smem_total(t.stages, t.tile_n);
     auto launch_pair = [&](auto kernel) -> int {
       ATTN_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));

@@ -392,7 +392,12 @@ extern "C" int gemm_plan(const attn_hw_desc* desc, int batch, int M, int N, int 
         out->tiles = (int)pt;
         out->ctas = (int)(2 * pairs);
         const long long pwaves = (pt + pairs - 1) / pairs;
-        out->wave_efficiency = (float)((double)pt / ((double)pwaves * pairs));
+        // Last wave: the r tiles left after the whole waves run as 2 r half-width items if those fit one wave of pairs.
+        const long long r = pt % pairs;
+        const bool split = r > 0 && 2 * r <= pairs;
+        out->tail_split = split ? (int32_t)r : 0;
+        const double waves_eff = split ? (double)(pwaves - 1) + 0.64 : (double)pwaves;   // a half-width item: 0.64 of a tile
+        out->wave_efficiency = (float)((double)pt / (waves_eff * pairs));
         out->cta_pair = 2;
         out->acc_buffers = h.acc_mem_columns / pn;
         out->feasible = 1;

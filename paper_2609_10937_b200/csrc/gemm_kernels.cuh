@@ -40,6 +40,7 @@ struct GemmParams {
   int k_steps;            // ceil(K / 64)
   int stages;
   int group_m;            // pair kernel: tiles are walked in bands of this many tile rows (see tile_coords)
+  int tail_tiles;         // pair kernel: the last this-many tiles are executed as two half-width work items each
 };
 
 // Order in which the persistent grid walks the output tiles.  Tiles that run at the same time should share operand
@@ -326,6 +327,16 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   const uint32_t tmem_base = misc->tmem_slot;
   const long long tiles = (long long)p.batch * p.m_tiles * p.n_tiles;
   const bool run = (*abort_flag == 0);
+  // Work items.  The tiles that would make up a last, partly empty wave (p.tail_tiles of them, fewer than half the
+  // pairs) are executed as two items of half the width each, so that the last wave keeps twice as many pairs busy for
+  // about 0.6 of a tile's time (a 128-wide instruction of a pair runs at about 0.8 of the rate of a 256-wide one).
+  const long long full_tiles = tiles - (kPairN == 256 ? p.tail_tiles : 0);
+  const long long items = full_tiles + 2 * (tiles - full_tiles);
+  auto item_of = [&](long long t, int& mt, int& nt, int& b, int& narrow, int& hcol) {
+    narrow = t >= full_tiles ? 1 : 0;
+    hcol = narrow ? (int)((t - full_tiles) & 1) : 0;
+    tile_coords(narrow ? full_tiles + ((t - full_tiles) >> 1) : t, p.m_tiles, p.n_tiles, p.group_m, mt, nt, b);
+  };
 
   if (warp == 0) {
     // ========================================================== TMA producer (both CTAs, each for what it holds)
@@ -333,20 +344,24 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (long long t = pair; ok && t < tiles; t += n_pairs) {
-        int nt, mt, b;
-      tile_coords(t, p.m_tiles, p.n_tiles, p.group_m, mt, nt, b);
-        const int row0 = mt * kTileM + (int)rank * kSub, col0 = nt * kPairN + (int)rank * kHalfN;
+      for (long long t = pair; ok && t < items; t += n_pairs) {
+        int nt, mt, b, narrow, hcol;
+        item_of(t, mt, nt, b, narrow, hcol);
+        // a half-width item: this CTA holds 64 of its 128 columns (the [N][K] box still brings 128 rows: the matrix
+        // instruction reads the first 64)
+        const int row0 = mt * kTileM + (int)rank * kSub;
+        const int col0 = nt * kPairN + (narrow ? hcol * (kPairN / 2) + (int)rank * (kHalfN / 2) : (int)rank * kHalfN);
+        const int b_chunks = narrow ? kHalfN / 128 : kHalfN / 64;
+        const uint32_t tx = (B_KN && narrow) ? 2u * (kPairStageA + (kHalfN / 2) * kTileK * 2) : 2u * kStageBytes;
         for (int ks = 0; ks < p.k_steps; ++ks) {
           if (!attn::wait_bar(smem_u32(&misc->empty[stage]), phase ^ 1u, abort_flag, attn::wait_info(kRoleGemmLoad, 1, ks))) { ok = false; break; }
           // the even CTA's barrier counts the bytes of both CTAs' copies of this stage
           const uint32_t bar = map_to_cta(smem_u32(&misc->full[stage]), 0);
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kPairStageA;
-          if (rank == 0) mbar_arrive_expect_tx(smem_u32(&misc->full[stage]), 2 * kStageBytes);
+          if (rank == 0) mbar_arrive_expect_tx(smem_u32(&misc->full[stage]), tx);
           tma_load_3d_pair(a_dst, &tm_a, ks * kTileK, row0, b, bar);
           if (B_KN) {
-#pragma unroll
-            for (int c = 0; c < kHalfN / 64; ++c)
+            for (int c = 0; c < b_chunks; ++c)
               tma_load_3d_pair(b_dst + c * (kTileK * 128), &tm_b, col0 + c * 64, ks * kTileK, b, bar);
           } else {
             tma_load_3d_pair(b_dst, &tm_b, ks * kTileK, col0, b, bar);
@@ -376,10 +391,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     bool ok = run && rank == 0;
     int stage = 0;
     uint32_t phase = 0, tile_ctr = 0;
-    constexpr uint32_t idesc = make_idesc_bf16(2 * kSub, kPairN, B_KN);
+    constexpr uint32_t idesc_full = make_idesc_bf16(2 * kSub, kPairN, B_KN);
+    constexpr uint32_t idesc_narrow = make_idesc_bf16(2 * kSub, kPairN / 2, B_KN);
     constexpr uint32_t hi_k = attn::desc_hi_sw128(1024);
-    for (long long t = pair; ok && t < tiles; t += n_pairs, ++tile_ctr) {
+    for (long long t = pair; ok && t < items; t += n_pairs, ++tile_ctr) {
       const uint32_t buf = tile_ctr % kBufs, use = tile_ctr / kBufs;
+      const uint32_t idesc = t >= full_tiles ? idesc_narrow : idesc_full;
       if (use > 0) {
         ok = attn::wait_bar_warp(smem_u32(&misc->acc_empty[buf]), (use - 1) & 1, abort_flag, attn::wait_info(kRoleGemmMma, 2, tile_ctr));
         if (!ok) break;
@@ -415,18 +432,20 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     const int half = ew >> 2;                                 // column half of the accumulator
     const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t stage_w = out_smem + ew * 8192;
-    constexpr int kChunks = kPairN / 128;                     // 64-column chunks per warp and tile
     uint32_t tile_ctr = 0, chunk_ctr = 0;
     bool ok = run;
-    for (long long t = pair; ok && t < tiles; t += n_pairs, ++tile_ctr) {
-      int nt, mt, b;
-      tile_coords(t, p.m_tiles, p.n_tiles, p.group_m, mt, nt, b);
+    for (long long t = pair; ok && t < items; t += n_pairs, ++tile_ctr) {
+      int nt, mt, b, narrow, hcol;
+      item_of(t, mt, nt, b, narrow, hcol);
+      const int width = narrow ? kPairN / 2 : kPairN;           // columns of this item's accumulator
+      const int kChunks = width / 128;                          // 64-column chunks per warp and item
       const uint32_t buf = tile_ctr % kBufs, use = tile_ctr / kBufs;
       ok = attn::wait_bar_warp(smem_u32(&misc->acc_full[buf]), use & 1, abort_flag, attn::wait_info(kRoleGemmEpi, 2, tile_ctr));
       if (!ok) break;
       tc_fence_after();
-      const uint32_t acc = lane_base + buf * kPairN + half * (kPairN / 2);
+      const uint32_t acc = lane_base + buf * kPairN + half * (width / 2);
       const int row0 = mt * kTileM + (int)rank * kSub + (warp & 3) * 32;
+      const int col_w = nt * kPairN + hcol * (kPairN / 2) + half * (width / 2);   // first column of this warp's part
 #pragma unroll 1
       for (int c = 0; c < kChunks; ++c, ++chunk_ctr) {
         uint32_t r0[32], r1[32];
@@ -452,7 +471,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_3d(&tm_c, dst, nt * kPairN + half * (kPairN / 2) + c * 64, row0, b);
+          tma_store_3d(&tm_c, dst, col_w + c * 64, row0, b);
           tma_store_commit();
         }
       }

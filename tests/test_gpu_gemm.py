@@ -58,17 +58,21 @@ def test_matrix_product_matches_oracle(env, layout, batch, M, N, K):
 @pytest.mark.parametrize("layout", ["kn", "nk"])
 @pytest.mark.parametrize("batch,M,N,K", [
     (1, 512, 512, 64), (1, 520, 264, 72), (2, 300, 1000, 200), (1, 129, 136, 8), (1, 4096, 768, 320), (5, 257, 257 + 7, 1024),
-    (1, 2560, 2304, 64)])
+    (1, 2560, 2304, 64), (1, 4000, 4096 - 56, 72), (1, 1280, 4096 - 8, 200)])
 def test_cta_pairs_and_lone_ctas_agree_with_the_oracle_and_each_other(env, layout, batch, M, N, K):
     """The two tilings of the same product: CTA pairs (one matrix instruction over two CTAs, two accumulators in tensor
     memory, per-warp stores) and lone CTAs.  Ragged M, N and K, several tiles per pair (more than the accumulators,
-    so that buffers are reused), batches.  Both sum the K products of an element in the same order: same bits."""
+    so that buffers are reused), batches, and shapes whose last wave runs as half-width work items (the last two: 256 and
+    80 tiles on 74 pairs leave 34 and 6).  All sum the K products of an element in the same order: same bits."""
     torch, go, binding = env
     desc = binding.hw_desc_query(0)
     assert binding.gemm_plan(desc, batch, M, N, K).cta_pair == 2
+    if M >= 1280 and N > 4000:
+        assert binding.gemm_plan(desc, batch, M, N, K).tail_split > 0
     _check_product(env, batch, M, N, K, layout, seed=4, rows_per_batch=300)                 # closed-form default: pairs
     _check_product(env, batch, M, N, K, layout, seed=4, rows_per_batch=300, cta_pair=1)
     _check_product(env, batch, M, N, K, layout, seed=4, rows_per_batch=300, cta_pair=2, tile_n=128)
+    _check_product(env, batch, M, N, K, layout, seed=4, rows_per_batch=300, tail_split=-1)   # whole tiles in the last wave
     rng = np.random.default_rng([9, M, N, K])
     a = to_cuda_bf16(_rand_bits(rng, (batch, M, K)))
     b = to_cuda_bf16(_rand_bits(rng, (batch, K, N) if layout == "kn" else (batch, N, K)))

@@ -49,7 +49,10 @@ def test_gemm_plan_closed_form(binding):
     assert (t.tile_m, t.tile_n, t.tile_k, t.n_sub, t.cta_pair, t.acc_buffers) == (256, 256, 64, 2, 2, 2)
     assert t.stages == (232448 - 65536 - 1024) // 32768 == 5 and t.smem_bytes == 5 * 32768 + 65536 + 1024
     assert (t.tiles, t.ctas, t.feasible, t.tmem_columns) == (256, 148, 1, 512)
-    assert t.wave_efficiency == pytest.approx(256 / (4 * 74))
+    # last wave: 256 = 3 * 74 + 34 tiles, 2 * 34 <= 74: the 34 run as 68 half-width items (0.64 of a tile's time each)
+    assert t.tail_split == 34 and t.wave_efficiency == pytest.approx(256 / ((3 + 0.64) * 74))
+    t8 = binding.gemm_plan(desc, 1, 8192, 8192, 8192)          # 1024 = 13 * 74 + 62 tiles: 124 halves do not fit one wave
+    assert t8.tail_split == 0 and t8.wave_efficiency == pytest.approx(1024 / (14 * 74))
     # pairs occupy as many CTAs as lone 128-row tiles would (3 * 4 * 3 = 36 pairs against 3 * 8 * 3 = 72 CTAs)
     t = binding.gemm_plan(desc, 3, 1000, 520, 64)
     assert (t.cta_pair, t.tile_m, t.tiles, t.ctas) == (2, 256, 36, 72)
