@@ -632,6 +632,30 @@ def test_bounded_wait_expiry_is_recorded_in_the_callers_status_words(env):
     assert torch.equal(out.view(torch.int16), want.view(torch.int16))
 
 
+@pytest.mark.parametrize("B,H,L,d,causal", [(2, 40, 2048, 64, False), (4, 32, 8192, 64, False), (1, 8, 2048, 64, False),
+                                            (2, 40, 2048, 128, False), (2, 40, 2048, 64, True)])
+def test_many_launches_no_wait_expires_and_the_bits_repeat(env, B, H, L, d, causal):
+    """Launch-to-launch repeatability under many launches.  At d = 64 the next step's scores are produced before this
+    step's P V is issued; arrivals on the per-step barriers are anonymous, so a protocol that lets a fast warp arrive
+    for step g+1 before a slow warp has arrived for step g fails once in ~10^4 launches of the large prefill shape (an
+    expired wait, or a product issued before its rows were rescaled).  Every launch must leave the device status clean
+    and reproduce the first launch's output bits."""
+    torch, _, binding = env
+    case = _case("many", B, H, L, d, cfg_id=88)
+    q, k, v = (to_cuda_bf16(x) for x in synth.make_qkv(case, 0))
+    first = binding.forward(q, k, v, causal=causal).clone()
+    torch.cuda.synchronize()
+    assert binding.last_device_status()[0] == 0
+    out = torch.empty_like(q)
+    launches = 300 if case.flops > 1e12 else 3000
+    for it in range(launches):
+        binding.forward(q, k, v, out, causal=causal)
+        if it % 50 == 49 or it == launches - 1:
+            code, detail = binding.last_device_status()
+            assert code == 0, (it, detail)
+            assert torch.equal(out.view(torch.int16), first.view(torch.int16)), f"launch {it} differs from the first"
+
+
 def test_descriptor_of_a_larger_machine_is_refused(env):
     torch, _, binding = env
     desc = binding.hw_desc_query(0)
