@@ -840,10 +840,13 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
   p.group_m = 1;
   p.tail_tiles = 0;
   if (pair) {
-    // bands of about sqrt(pairs) tile rows: the tiles in flight then share the fewest operand panels
+    // Bands of about sqrt(pairs) tile rows: the tiles in flight then share the fewest operand panels.  Only when the
+    // operands of a tile outweigh its output eightfold (K >= 1024 for 256 x 256 tiles): below that the output
+    // dominates the traffic, and tile rows walked whole write whole rows of C (16384 x 16384 x 64: 141 against 156 us).
     const int pairs = t.ctas / 2;
     int gm = 1;
-    while ((gm + 1) * (gm + 1) <= pairs) ++gm;
+    if ((long long)(t.tile_m + t.tile_n) * K >= 8LL * t.tile_m * t.tile_n)
+      while ((gm + 1) * (gm + 1) <= pairs) ++gm;
     p.group_m = gm;
     p.tail_tiles = t.tail_split;
     const int smem = gemm::pair_smem_total(t.stages, t.tile_n);

@@ -57,8 +57,8 @@ def test_matrix_product_matches_oracle(env, layout, batch, M, N, K):
 
 @pytest.mark.parametrize("layout", ["kn", "nk"])
 @pytest.mark.parametrize("batch,M,N,K", [
-    (1, 512, 512, 64), (1, 520, 264, 72), (2, 300, 1000, 200), (1, 129, 136, 8), (1, 4096, 768, 320), (5, 257, 257 + 7, 1024),
-    (1, 2560, 2304, 64), (1, 4000, 4096 - 56, 72), (1, 1280, 4096 - 8, 200)])
+    (1, 512, 512, 256), (1, 520, 264, 264), (2, 300, 1000, 328), (1, 129, 136, 256), (1, 4096, 768, 320), (5, 257, 257 + 7, 1024),
+    (1, 2560, 2304, 256), (1, 4000, 4096 - 56, 264), (1, 1280, 4096 - 8, 1096)])
 def test_cta_pairs_and_lone_ctas_agree_with_the_oracle_and_each_other(env, layout, batch, M, N, K):
     """The two tilings of the same product: CTA pairs (one matrix instruction over two CTAs, two accumulators in tensor
     memory, per-warp stores) and lone CTAs.  Ragged M, N and K, several tiles per pair (more than the accumulators,

@@ -54,8 +54,11 @@ def test_gemm_plan_closed_form(binding):
     t8 = binding.gemm_plan(desc, 1, 8192, 8192, 8192)          # 1024 = 13 * 74 + 62 tiles: 124 halves do not fit one wave
     assert t8.tail_split == 0 and t8.wave_efficiency == pytest.approx(1024 / (14 * 74))
     # pairs occupy as many CTAs as lone 128-row tiles would (3 * 4 * 3 = 36 pairs against 3 * 8 * 3 = 72 CTAs)
-    t = binding.gemm_plan(desc, 3, 1000, 520, 64)
+    t = binding.gemm_plan(desc, 3, 1000, 520, 256)
     assert (t.cta_pair, t.tile_m, t.tiles, t.ctas) == (2, 256, 36, 72)
+    # fewer than four ring stages of products per tile: the hand-over inside a pair would not pay
+    t = binding.gemm_plan(desc, 3, 1000, 520, 64)
+    assert (t.cta_pair, t.n_sub, t.tile_m, t.tiles, t.ctas) == (1, 1, 128, 72, 72)
     # an output no wider than half the atom's N stays with lone CTAs (P V of the unfused path: 64 blocks -> 128)
     t = binding.gemm_plan(desc, 1, 16384, 128, 16384)
     assert (t.cta_pair, t.n_sub, t.tile_n, t.tiles, t.ctas) == (1, 1, 128, 128, 128)
