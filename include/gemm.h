@@ -55,9 +55,8 @@ typedef struct gemm_tiles {
  * tile_k = 128 bytes / elem_bytes; stages = min(8, (local_mem - staging - 1024)
  * / ((tile_m + tile_n) * tile_k * elem_bytes)), at least 2.
  * CTA pairs: taken when the descriptor says pairs can run (max_clusters[1] > 0), tensor memory holds two
- * accumulators (acc_mem_columns >= 2 atom_n_max), M > atom_m, N > atom_n_max / 2, K >= 4 tile_k (the hand-over between the
- * two CTAs of a pair costs about as much per tile as two ring stages of products: measured, 16384 x 16384 x K, pairs
- * 141 / 157 / 182 / 216 us against 120 / 147 / 181 / 252 us for lone CTAs at K = 64 / 128 / 256 / 512) and
+ * accumulators (acc_mem_columns >= 2 atom_n_max), M > atom_m, N > atom_n_max / 2 (any K: measured, 16384 x 16384 x K,
+ * pairs 100 / 98 / 131 / 198 us against 121 / 147 / 195 / 263 us for lone CTAs at K = 64 / 128 / 256 / 512) and
  * the pairs, P = min(max_clusters[1], num_units / 2, tiles), occupy at least as many CTAs as the lone-CTA tiling
  * above would (the paper's occupancy step).  A pair owns a 2 atom_m x atom_n_max tile; every CTA stages its own
  * atom_m rows of A and atom_n_max / 2 columns of B, so stages = min(8, (local_mem - 4 atom_m 128 - 1024) /

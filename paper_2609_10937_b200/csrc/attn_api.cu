@@ -839,6 +839,7 @@ int gemm_launch(const void* a, const void* b, void* c, int batch, int M, int N, 
   p.stages = t.stages;
   p.group_m = 1;
   p.tail_tiles = 0;
+  p.stream_c = (long long)batch * M * N * 2 > (long long)st->desc.cache_bytes ? 1 : 0;
   if (pair) {
     // Bands of about sqrt(pairs) tile rows: the tiles in flight then share the fewest operand panels.  Only when the
     // operands of a tile outweigh its output eightfold (K >= 1024 for 256 x 256 tiles): below that the output

@@ -375,9 +375,8 @@ extern "C" int gemm_plan(const attn_hw_desc* desc, int batch, int M, int N, int 
     const long long lone = (long long)batch * ceil_div(M, tile_m) * ceil_div(N, tile_n);
     const long long lone_ctas = lone < h.num_units ? lone : h.num_units;
     const long long pairs = pt < pairs_max ? pt : pairs_max;
-    // (a pair pays a hand-over between its two CTAs per tile: it needs a few ring stages of products per tile to win)
     if (pairs_max > 0 && M > h.atom_m && N > pn / 2 && h.acc_mem_columns >= 2 * pn && 2 * pairs >= lone_ctas &&
-        K >= 4 * tile_k && pt <= 0x3FFFFFFFLL) {
+        pt <= 0x3FFFFFFFLL) {
       const int pstage = (h.atom_m + pn / 2) * tile_k * h.elem_bytes;
       const int pstaging = 4 * h.atom_m * 128;    // per epilogue warp (4 lane quarters x 2 column halves) two 32-row chunks
       int pstages = (h.local_mem_bytes - pstaging - 1024) / pstage;

@@ -41,6 +41,7 @@ struct GemmParams {
   int stages;
   int group_m;            // pair kernel: tiles are walked in bands of this many tile rows (see tile_coords)
   int tail_tiles;         // pair kernel: the last this-many tiles are executed as two half-width work items each
+  int stream_c;           // pair kernel: C is larger than the cache and its stores carry the evict-first priority
 };
 
 // Order in which the persistent grid walks the output tiles.  Tiles that run at the same time should share operand
@@ -454,7 +455,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         tmem_ld_fence(r0);
         tmem_ld_fence(r1);
         if (c == kChunks - 1) {
-          // this warp has read its part of the accumulator: one arrival per warp on the even CTA's barrier
+          // this warp has read its part of the accumulator: one arrival per warp on the even CTA's barrier (the
+          // tensor-memory loads have completed and are fenced; no memory of this thread has to reach the peer)
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_peer(map_to_cta(smem_u32(&misc->acc_empty[buf]), 0));
@@ -471,7 +473,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_3d(&tm_c, dst, col_w + c * 64, row0, b);
+          if (p.stream_c) tma_store_3d_hint(&tm_c, dst, col_w + c * 64, row0, b, l2_policy_evict_first());
+          else tma_store_3d(&tm_c, dst, col_w + c * 64, row0, b);
           tma_store_commit();
         }
       }

@@ -77,6 +77,19 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, uint32_t src_
       ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src_smem), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
+// The same store with an L2 eviction priority: a stream of output much larger than the cache, marked evict-first,
+// leaves the cache as it arrives instead of piling up as dirty lines that later writes have to wait out.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_store_3d_hint(const CUtensorMap* m, uint32_t src_smem, int x, int y, int z, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3, %4}], [%1], %5;"
+      ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src_smem), "r"(x), "r"(y), "r"(z), "l"(policy)
+      : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() {
   asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -290,9 +303,13 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
   return r;
 }
-// One arrival on an mbarrier of another CTA of the cluster (release at cluster scope).
+// One arrival on an mbarrier of another CTA of the cluster, with release at CTA scope only: it tells the peer that
+// this CTA is done READING something (tensor memory after tcgen05.fence::before_thread_sync, or a shared-memory buffer
+// whose last reader -- a matrix instruction -- this thread has seen complete on an mbarrier), so that the peer may
+// overwrite it.  It publishes nothing this thread wrote; a release at cluster scope would, and costs the arriving
+// thread about a thousand cycles (measured: 950 cycles per tile in the pair matrix product).
 __device__ __forceinline__ void mbar_arrive_peer(uint32_t peer_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(peer_bar) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(peer_bar) : "memory");
 }
 // Asynchronous stores into another CTA's shared memory; the bytes are counted on that CTA's mbarrier
 // (complete_tx), whose waiter then sees the data -- the same contract as a bulk copy.

@@ -58,12 +58,15 @@ def test_matrix_product_matches_oracle(env, layout, batch, M, N, K):
 @pytest.mark.parametrize("layout", ["kn", "nk"])
 @pytest.mark.parametrize("batch,M,N,K", [
     (1, 512, 512, 256), (1, 520, 264, 264), (2, 300, 1000, 328), (1, 129, 136, 256), (1, 4096, 768, 320), (5, 257, 257 + 7, 1024),
-    (1, 2560, 2304, 256), (1, 4000, 4096 - 56, 264), (1, 1280, 4096 - 8, 1096)])
+    (1, 2560, 2304, 256), (1, 4000, 4096 - 56, 264), (1, 1280, 4096 - 8, 1096),
+    (1, 512, 520, 64), (2, 300, 1000, 72), (1, 2560, 2304, 128), (1, 384, 264, 8), (1, 8192, 8200, 64)])
 def test_cta_pairs_and_lone_ctas_agree_with_the_oracle_and_each_other(env, layout, batch, M, N, K):
     """The two tilings of the same product: CTA pairs (one matrix instruction over two CTAs, two accumulators in tensor
     memory, per-warp stores) and lone CTAs.  Ragged M, N and K, several tiles per pair (more than the accumulators,
     so that buffers are reused), batches, and shapes whose last wave runs as half-width work items (the last two: 256 and
-    80 tiles on 74 pairs leave 34 and 6).  All sum the K products of an element in the same order: same bits."""
+    80 tiles on 74 pairs leave 34 and 6), one or two ring stages of products per tile, and an output larger than the
+    cache (the last: its stores carry an eviction priority).  All sum the K products of an element in the same order:
+    same bits."""
     torch, go, binding = env
     desc = binding.hw_desc_query(0)
     assert binding.gemm_plan(desc, batch, M, N, K).cta_pair == 2

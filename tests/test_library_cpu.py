@@ -56,9 +56,12 @@ def test_gemm_plan_closed_form(binding):
     # pairs occupy as many CTAs as lone 128-row tiles would (3 * 4 * 3 = 36 pairs against 3 * 8 * 3 = 72 CTAs)
     t = binding.gemm_plan(desc, 3, 1000, 520, 256)
     assert (t.cta_pair, t.tile_m, t.tiles, t.ctas) == (2, 256, 36, 72)
-    # fewer than four ring stages of products per tile: the hand-over inside a pair would not pay
+    # ... whatever K is (one ring stage of products per tile: the scores of the unfused path at d = 64)
     t = binding.gemm_plan(desc, 3, 1000, 520, 64)
-    assert (t.cta_pair, t.n_sub, t.tile_m, t.tiles, t.ctas) == (1, 1, 128, 72, 72)
+    assert (t.cta_pair, t.tile_m, t.tiles, t.ctas) == (2, 256, 36, 72)
+    # M within one sub-tile: nothing for a second CTA to hold
+    t = binding.gemm_plan(desc, 3, 128, 520, 64)
+    assert (t.cta_pair, t.n_sub, t.tile_m, t.tiles) == (1, 1, 128, 9)
     # an output no wider than half the atom's N stays with lone CTAs (P V of the unfused path: 64 blocks -> 128)
     t = binding.gemm_plan(desc, 1, 16384, 128, 16384)
     assert (t.cta_pair, t.n_sub, t.tile_n, t.tiles, t.ctas) == (1, 1, 128, 128, 128)
