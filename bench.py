@@ -501,18 +501,20 @@ def run_ours(args):
 # ------------------------------------------------------------------------------------------------ other modes
 def run_case(args):
     """One named configuration, timed alone (few launches: the command profiler captures are taken on).  `gemmN` is
-    the N x N x N matrix product."""
+    the N x N x N matrix product, `gemmMxNxK` any other.  Beside it the library product on the same inputs."""
     gpu = Gpu(0)
     if args.case.startswith("gemm"):
-        n = int(args.case[4:])
+        dims = [int(x) for x in args.case[4:].split("x")]
+        m, n, k = dims if len(dims) == 3 else (dims[0],) * 3
         torch, binding = gpu.torch, gpu.binding
-        a = torch.randn(n, n, device="cuda").to(torch.bfloat16)
-        b = torch.randn(n, n, device="cuda").to(torch.bfloat16)
-        c = torch.empty(n, n, dtype=torch.bfloat16, device="cuda")
+        a = torch.randn(m, k, device="cuda").to(torch.bfloat16)
+        b = torch.randn(k, n, device="cuda").to(torch.bfloat16)
+        c = torch.empty(m, n, dtype=torch.bfloat16, device="cuda")
         ms, _, _, _ = gpu.timed(lambda: binding.gemm(a, b, c), args.steps, 3)
         ms_lib, _, _, _ = gpu.timed(lambda: torch.matmul(a, b, out=c), args.steps, 3)
-        print(json.dumps({"case": args.case, "ms": ms, "tflops": 2.0 * n ** 3 / ms / 1e9, "torch_matmul_ms": ms_lib,
-                          "tiles": binding.gemm_plan(gpu.desc, 1, n, n, n).as_dict()}), flush=True)
+        print(json.dumps({"case": args.case, "ms": ms, "tflops": 2.0 * m * n * k / ms / 1e9,
+                          "c_write_gbs": 2.0 * m * n / ms / 1e6, "torch_matmul_ms": ms_lib,
+                          "tiles": binding.gemm_plan(gpu.desc, 1, m, n, k).as_dict()}), flush=True)
         return 0
     out = measure_config(gpu, args.case, load_peaks(), iters=args.steps, oracle=False)
     print(json.dumps({"case": args.case, **out}), flush=True)
@@ -651,7 +653,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the unfused-path and matrix-product context numbers")
     ap.add_argument("--no-configs", action="store_true", help="skip the other benchmark configurations")
     ap.add_argument("--no-sustained", action="store_true", help="skip the seconds-long back-to-back leg")
-    ap.add_argument("--case", default=None, help="time one named configuration only (cfg1, cfg2, cfg4_L1024, ..., cfg5b, gemm4096)")
+    ap.add_argument("--case", default=None, help="time one named configuration only (cfg1, cfg2, cfg4_L1024, ..., cfg5b, gemm4096, gemm16384x16384x128)")
     ap.add_argument("--tile-sweep", default=None, metavar="NAME", help="tile sweep around the closed-form default")
     ap.add_argument("--grid-sweep", action="store_true", help="grid-size sweep over short and medium shapes")
     ap.add_argument("--unfused-sweep", action="store_true", help="fused against unfused over L; matrix product alone")
