@@ -629,7 +629,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mbar_arrive(bar_h);
               return true;
       };
-      for (int jj = 0; ok && jj < n; ++jj, ++g) {
+      // Causal: the steps before the sub-tile's diagonal (and before a ragged last key tile) need no mask and run in
+      // a loop of their own that holds nothing but the common step; the few masked steps of the segment follow.
+      int jj = 0;
+      if constexpr (CAUSAL && !CLUSTER) {
+        int first_masked = (q_row0 + i * kSub) / TKV;          // first step that reaches past the sub-tile's first row
+        if (kv_tail != 0 && p.n_steps - 1 < first_masked) first_masked = p.n_steps - 1;
+        int n_plain = first_masked - j0;
+        n_plain = n_plain < 0 ? 0 : (n_plain > n ? n : n_plain);
+        for (; ok && jj < n_plain; ++jj, ++g) ok = softmax_step(MaskTag<false>{}, TKV - 1);
+      }
+      for (; ok && jj < n; ++jj, ++g) {
         const int j = j0 + jj;
         const bool ragged = (kv_tail != 0) && (j == p.n_steps - 1);
         const bool diagonal = CAUSAL && ((j + 1) * TKV - 1 > q_row0 + i * kSub);   // warp-uniform
